@@ -1,0 +1,356 @@
+#!/usr/bin/env python
+"""Benchmark of the LoRDBA adapter forward on B200.
+
+One step = one pass of the whole hot path (pack excluded: it runs once per
+adapter) over one batch: the LLaMA-2-7B attention-projection adapter,
+d_in = d_out = 4096, r = 16, T = 2048 tokens, bf16 activations, float32 scales.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line.  `value` is adapter-branch tokens/s with the inputs
+resident in HBM; consecutive steps rotate through buffer sets whose total size
+exceeds the L2 several times over, so every step reads x and y from DRAM.
+`e2e` is the same metric through lordba_adapter_forward_host with pinned host
+buffers (H2D of x and y and D2H of y inside the timed region).  `roofline`
+relates the kernel's algorithmic bytes per launch to the measured HBM copy peak.
+`cpu_baseline` is the float64 oracle timed on this machine's host cores.
+
+With --gpus N > 1 (under torchrun) every rank runs the same step on its own
+token shard of T tokens (weak scaling, no collective on the data path).
+With --impl reference the oracle itself is timed on the host, rank 0 only.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_24058_b200 import workloads  # noqa: E402
+
+METRIC = "adapter-branch tokens/s at r=16, T=2048 (LLaMA-2-7B attention projection 4096->4096, bf16)"
+UNIT = "tokens/s"
+D_IN = D_OUT = workloads.HIDDEN
+R = 16
+T = 2048
+ELEM = 2
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and throttle reasons through NVML (read-only) while the GPU is busy."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        self.recording = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            if self.recording:
+                try:
+                    mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                    self.samples.append(mhz)
+                    for bit, name in names.items():
+                        if mask & bit:
+                            self.reasons.add(name)
+                except Exception:
+                    pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                    "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_inputs(p):
+    f8 = np.float64
+    return (p.x_f64(), p.A_sign, p.B_sign, p.s_in.astype(f8), p.s_r.astype(f8), p.s_out.astype(f8),
+            p.y_f64())
+
+
+def time_oracle(p, tokens: int, repeats: int):
+    """Seconds for `repeats` oracle passes over the first `tokens` tokens of p."""
+    import oracle
+    x, A, B, s_in, s_r, s_out, y = oracle_inputs(p)
+    x, y = x[:tokens], y[:tokens]
+    oracle.adapter_forward(x[:8], A, B, s_in, s_r, s_out, y[:8])        # load + warm
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        oracle.adapter_forward(x, A, B, s_in, s_r, s_out, y)
+    return time.perf_counter() - t0, oracle.num_threads()
+
+
+def cpu_baseline(p):
+    dt1, cores = time_oracle(p, T, 1)
+    repeats = int(min(200, max(2, round(12.0 / max(dt1, 1e-3)))))
+    dt, cores = time_oracle(p, T, repeats)
+    return {"value": repeats * T / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d passes of the float64 oracle over the full step (T=%d tokens), %.1f s"
+                      % (repeats, T, dt)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    p = workloads.config1(T=T, r=R)
+    dt_probe, cores = time_oracle(p, 64, 1)
+    rate = 64.0 / max(dt_probe, 1e-6)
+    budget_s = 90.0
+    tokens = int(max(1, min(T, budget_s * rate / max(1, args.steps + args.warmup))))
+    time_oracle(p, tokens, max(0, args.warmup))
+    dt, cores = time_oracle(p, tokens, args.steps)
+    value = args.steps * tokens / dt
+    sample = "each step = the oracle over %d of the step's %d tokens" % (tokens, T)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": "config1: attn 4096->4096, r=16, T=2048, bf16 inputs widened to f64",
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------- GPU arm
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2605_24058_b200 import lordba
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    lordba.load()
+    if args.variant is not None:
+        lordba.set_variant({"auto": 0, "fma": 1, "tc": 2}[args.variant])
+
+    # inputs: one seeded draw per rank (its own token shard); buffer sets are device-side
+    # copies so that consecutive steps never hit L2.
+    p = workloads.config1(T=T, r=R, seed=1000 + rank)
+    to_bf16 = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16)
+    x_host = to_bf16(p.x).pin_memory()
+    y_host = to_bf16(p.y).pin_memory()
+    set_bytes = (T * D_IN + T * D_OUT) * ELEM
+    n_sets = int(np.ceil(4 * L2_BYTES / set_bytes))
+    xs = [x_host.to(dev) for _ in range(n_sets)]
+    ys = [y_host.to(dev) for _ in range(n_sets)]
+    packed_A = lordba.pack_signs(torch.from_numpy(p.A_sign).to(dev), 0)
+    packed_B = lordba.pack_signs(torch.from_numpy(p.B_sign).to(dev), 1)
+    s_in = torch.from_numpy(p.s_in).to(dev)
+    s_r = torch.from_numpy(p.s_r).to(dev)
+    s_out = torch.from_numpy(p.s_out).to(dev)
+
+    def step(i):
+        lordba.adapter_forward(xs[i % n_sets], packed_A, packed_B, s_in, s_r, s_out, ys[i % n_sets], R)
+
+    # correctness of the configuration being timed: sampled rows against the oracle (rank 0)
+    parity = None
+    if rank == 0:
+        import oracle
+        step(0)
+        torch.cuda.synchronize()
+        rows = np.array([0, 1, 127, 128, 1000, 2047])
+        got = ys[0][torch.from_numpy(rows).to(dev)].to(torch.float64).cpu().numpy()
+        f8 = np.float64
+        want = oracle.adapter_forward(p.x_f64()[rows], p.A_sign, p.B_sign, p.s_in.astype(f8),
+                                      p.s_r.astype(f8), p.s_out.astype(f8), p.y_f64()[rows])
+        rms = float(np.sqrt(np.mean(want * want)))
+        parity = float(np.abs(got - want).max() / rms)
+        if not parity <= 2e-2:
+            raise RuntimeError("bench configuration fails parity: max err / rms = %g" % parity)
+        ys[0].copy_(y_host)
+
+    # one CUDA graph holds n_sets consecutive steps (one per buffer set): launches are then
+    # issued faster than the ~10 us kernels retire.
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for i in range(n_sets):
+            step(i)
+        stream.synchronize()
+        n0 = lordba.launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(n_sets):
+                step(i)
+        launches_per_step = (lordba.launch_count() - n0) / n_sets
+
+        def run_steps(k):
+            full, rem = divmod(k, n_sets)
+            for _ in range(full):
+                graph.replay()
+            for i in range(rem):
+                step(i)
+
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        run_steps(args.warmup)
+        stream.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.recording = True
+        e0.record(stream)
+        run_steps(args.steps)
+        e1.record(stream)
+        stream.synchronize()
+        sampler.recording = False
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+
+        # end to end through the host-buffer entry point: H2D x, H2D y, kernel, D2H y per step
+        ws = torch.empty(lordba.host_workspace_bytes(T, D_IN, D_OUT, lordba.BF16), dtype=torch.uint8,
+                         device=dev)
+        e2e_steps = int(max(3, min(args.steps, 40)))
+
+        def host_step():
+            lordba.adapter_forward_host(x_host, packed_A, packed_B, s_in, s_r, s_out, y_host, R, ws,
+                                        stream=stream)
+        for _ in range(3):
+            host_step()
+        stream.synchronize()
+        y_host.copy_(to_bf16(p.y))
+        if world > 1:
+            dist.barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(e2e_steps):
+            host_step()
+        h1.record(stream)
+        stream.synchronize()
+        e2e_ms = h0.elapsed_time(h1)
+        sampler.stop()
+
+    status = lordba.device_status()
+    if status != 0:
+        raise RuntimeError("device status word is %d after the timed region" % status)
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        alg_bytes = workloads.algorithmic_bytes(T, D_IN, D_OUT, R, ELEM)
+        sec_per_step = ms * 1e-3 / args.steps
+        achieved = alg_bytes / sec_per_step / 1e9
+        variant = {0: "auto", 1: "fma", 2: "tc"}[lordba.get_variant()]
+        line = {
+            "metric": METRIC, "value": world * T * args.steps / (ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "config1: LLaMA-2-7B attention projection adapter, d_in=d_out=4096, "
+                                   "r=16, T=2048 tokens per GPU per step, bf16 x/y, fp32 scales",
+                       "l2": "steps rotate through %d device buffer sets (%.0f MB > 4 x L2)"
+                             % (n_sets, n_sets * set_bytes / 1e6),
+                       "launch": "CUDA graph of %d steps replayed" % n_sets,
+                       "kernel_variant": variant, "parallelism": "token shards, no collective",
+                       "parity_max_err_over_rms": parity},
+            "hbm_gbs": achieved,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": args.traffic,
+                         "peak_kind": "of " + peak_kind,
+                         "algorithmic_bytes_per_launch": alg_bytes},
+            "e2e": {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": (T * D_IN + T * D_OUT) * ELEM,
+                    "d2h_bytes_per_step": T * D_OUT * ELEM, "steps": e2e_steps},
+            "gpu_launches": int(round(launches_per_step * args.steps)),
+            "clocks": sampler.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(p)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=400)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", default=None, choices=["auto", "fma", "tc"],
+                    help="pin the kernel family (default: the library's own choice)")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="ncu DRAM bytes per launch to report in roofline.traffic")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,174 @@
+/*
+ * lordba.h -- C ABI of the B200 (sm_100a) LoRDBA adapter-forward library.
+ *
+ * The library evaluates the unmerged low-rank double-binary adapter branch
+ *
+ *     y[t,:] += s_out * ( B_sign ( s_r * ( A_sign ( s_in * x[t,:] ) ) ) )      t < T
+ *
+ * i.e. the paper's Delta-W(theta) = D_alpha B1 D_beta B2 D_gamma (Def. 1, Eq. 4,
+ * canonical l = 1) applied in the evaluation order of Eq. 8 with both binary
+ * products done as the sign accumulation of Eq. 9, and added to the buffer that
+ * already holds the frozen base projection's output (Eq. 2).
+ *
+ *     paper              here
+ *     N, M, R            d_in, d_out, r
+ *     B1 (N x R)         A_sign = B1^T   (r x d_in,   +-1)
+ *     B2 (R x M)         B_sign = B2^T   (d_out x r,  +-1)
+ *     alpha, beta, gamma s_in (d_in), s_r (r), s_out (d_out), float32
+ *     X (T x N)          x, row-major, one token per row
+ *
+ * The paper's Def. 1 carries no scalar LoRA alpha/r factor; a caller that has
+ * one multiplies it into s_r.
+ *
+ * Conventions for every entry point
+ *   - Pointers marked [device] are caller-owned device memory of the current
+ *     CUDA device; [host] pointers are ordinary host memory.  The library keeps
+ *     no pointer after a call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls enqueue work on it and return without synchronising,
+ *     except where stated.
+ *   - Return value: a lordba_status.  Argument errors are detected on the host
+ *     and nothing is launched.  There is no CPU fallback: without a usable CUDA
+ *     device the calls return LORDBA_ECUDA.
+ *   - Supported rank: 1 <= r <= 64.
+ *
+ * Bit-packed carriers (the paper says only "bit-packed"; this layout is the
+ * library's own).  Bit 1 <=> +1, bit 0 <=> -1, 32-bit little-endian words,
+ * pad bits are 0:
+ *   role 0, A carrier (r x d_in): r bit-rows, each padded to whole words,
+ *       wA = ceil(d_in/32); entry (k,i) is bit (i mod 32) of word k*wA + i/32.
+ *   role 1, B carrier (d_out x r): one dense bit stream of the row-major
+ *       matrix; entry (j,k) is bit (b mod 32) of word b/32 with b = j*r + k.
+ */
+#ifndef LORDBA_H_
+#define LORDBA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LORDBA_F32 = 0,   /* x and y are float32                                   */
+    LORDBA_BF16 = 1   /* x and y are bfloat16; all accumulation is in float32  */
+} lordba_dtype;
+
+typedef enum {
+    LORDBA_OK = 0,
+    LORDBA_EINVAL = 1,        /* null pointer, negative size, ld < width, x aliases y ...   */
+    LORDBA_EUNSUPPORTED = 2,  /* rank outside 1..64, unknown dtype / role / variant         */
+    LORDBA_EALIGN = 3,        /* a pointer is not aligned to its element type               */
+    LORDBA_ECUDA = 4,         /* a CUDA runtime call or the launch failed                   */
+    LORDBA_ETIMEOUT = 5       /* a bounded device-side wait gave up (see lordba_device_status) */
+} lordba_status;
+
+/* Kernel families the forward entry points can be pinned to (default AUTO). */
+typedef enum {
+    LORDBA_VARIANT_AUTO = 0,  /* tensor-core kernel when the shape allows it, else FMA      */
+    LORDBA_VARIANT_FMA = 1,   /* CUDA-core float32 FMA kernel (always used for LORDBA_F32)  */
+    LORDBA_VARIANT_TC = 2     /* tcgen05/TMA kernel; LORDBA_EUNSUPPORTED if the shape or    */
+                              /* alignment rules it out                                     */
+} lordba_variant;
+
+/* One adapted projection for the _ex and _batched entry points.  ldx / ldy are
+ * row pitches in elements (ldx >= d_in, ldy >= d_out). */
+typedef struct lordba_proj {
+    const void     *x;          /* [device] T x d_in,  pitch ldx                */
+    const uint32_t *packed_A;   /* [device] role-0 words of A_sign (r x d_in)   */
+    const uint32_t *packed_B;   /* [device] role-1 words of B_sign (d_out x r)  */
+    const float    *s_in;       /* [device] d_in                                */
+    const float    *s_r;        /* [device] r                                   */
+    const float    *s_out;      /* [device] d_out                               */
+    void           *y;          /* [device] T x d_out, pitch ldy, updated in place */
+    int64_t d_in, d_out, ldx, ldy;
+    int32_t r;
+    int32_t reserved;           /* must be 0 */
+} lordba_proj;
+
+/* Number of uint32 words of a packed carrier (layout above); -1 on bad arguments. */
+int64_t lordba_packed_words(int64_t rows, int64_t cols, int role);
+
+/*
+ * Bit-pack a sign matrix ("bit-packed {B1,B2} stored once per adapter",
+ * Section 3.3).  signs: [device] int8, rows x cols row-major; an entry < 0 packs
+ * as -1, anything else (0 included: sign(0) = +1) as +1.  role 0: rows = r,
+ * cols = d_in.  role 1: rows = d_out, cols = r.  packed: [device], at least
+ * lordba_packed_words() words, fully overwritten (pad bits 0).
+ */
+int lordba_pack_signs(const int8_t *signs, int64_t rows, int64_t cols, int role,
+                      uint32_t *packed, void *stream);
+
+/* Inverse of lordba_pack_signs: writes +1 / -1 into signs [device] (rows x cols). */
+int lordba_unpack_signs(const uint32_t *packed, int64_t rows, int64_t cols, int role,
+                        int8_t *signs, void *stream);
+
+/*
+ * Adapter forward, Eq. 8 / Eq. 9, bfloat16 activations, dense rows
+ * (ldx = d_in, ldy = d_out).  All pointers [device].  y is read, the adapter
+ * term is added in float32 and the sum is rounded once to bfloat16.  x and y
+ * must not overlap.  T = 0 is a no-op.
+ */
+int lordba_adapter_forward(const void *x, const uint32_t *packed_A, const uint32_t *packed_B,
+                           const float *s_in, const float *s_r, const float *s_out, void *y,
+                           int64_t T, int64_t d_in, int64_t d_out, int r, void *stream);
+
+/* Same operation with float32 x and y (float32 arithmetic throughout). */
+int lordba_adapter_forward_f32(const float *x, const uint32_t *packed_A, const uint32_t *packed_B,
+                               const float *s_in, const float *s_r, const float *s_out, float *y,
+                               int64_t T, int64_t d_in, int64_t d_out, int r, void *stream);
+
+/* Same operation with explicit row pitches and dtype.  p: [host]. */
+int lordba_adapter_forward_ex(const lordba_proj *p, int64_t T, int dtype, void *stream);
+
+/*
+ * The adapter forward of n_proj projections that share T and dtype (for
+ * instance the seven adapted projections q,k,v,o,gate,up,down of one decoder
+ * layer, Section 5 Setup) in as few launches as the kernel-parameter space
+ * allows.  projs: [host] array, read before the call returns.  The projections
+ * must write disjoint y buffers.
+ */
+int lordba_adapter_forward_batched(const lordba_proj *projs, int n_proj, int64_t T, int dtype,
+                                   void *stream);
+
+/*
+ * Host-buffer form of lordba_adapter_forward{,_f32}: x_host and y_host are
+ * [host] (pinned memory makes the copies asynchronous), dense rows; the carriers
+ * and scales stay [device] because they are loaded once per adapter.
+ * workspace: [device], at least lordba_host_workspace_bytes() bytes, 256-byte
+ * aligned.  Enqueues H2D(x), H2D(y), the forward kernel and D2H(y) on `stream`;
+ * y_host is valid once the stream has been synchronised.
+ */
+size_t lordba_host_workspace_bytes(int64_t T, int64_t d_in, int64_t d_out, int dtype);
+int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
+                                const uint32_t *packed_B, const float *s_in, const float *s_r,
+                                const float *s_out, void *y_host, int64_t T, int64_t d_in,
+                                int64_t d_out, int r, int dtype, void *workspace,
+                                size_t workspace_bytes, void *stream);
+
+/* Storage of one adapter in bits, Eq. 5: r(d_in+d_out) + 16 ell (d_in+r+d_out). */
+int64_t lordba_adapter_bits(int64_t d_in, int64_t d_out, int r, int ell);
+
+/* Pin the kernel family used by the forward entry points (process-wide). */
+int lordba_set_variant(int variant);
+int lordba_get_variant(void);
+
+/*
+ * Bounded device-side waits (TMA / MMA completion barriers) record a non-zero
+ * code in a device status word instead of spinning forever.  This call
+ * synchronises `stream`, copies the word to *code, clears it, and returns
+ * LORDBA_ETIMEOUT if it was non-zero.
+ */
+int lordba_device_status(int *code, void *stream);
+
+/* Kernels launched by this library in this process so far. */
+int64_t lordba_launch_count(void);
+
+const char *lordba_status_string(int status);
+const char *lordba_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LORDBA_H_ */

@@ -1,0 +1,261 @@
+// C ABI of liblordba: argument validation on the host, kernel-family choice,
+// launches.  See include/lordba.h for the contract of every entry point.
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "lordba_internal.h"
+
+namespace lordba {
+
+namespace {
+std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_variant{LORDBA_VARIANT_AUTO};
+__device__ int g_device_status;   // written by bounded waits that gave up
+std::mutex g_status_mutex;
+int *g_status_ptr[64] = {nullptr};
+}  // namespace
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int *device_status_word()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_status_mutex);
+    if (!g_status_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        g_status_ptr[dev] = static_cast<int *>(p);
+    }
+    return g_status_ptr[dev];
+}
+
+namespace {
+
+bool aligned(const void *p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a == 0; }
+
+bool overlaps(const void *a, size_t na, const void *b, size_t nb)
+{
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+
+int validate_proj(const lordba_proj &p, int64_t T, int dtype)
+{
+    if (dtype != LORDBA_F32 && dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    if (T < 0 || p.d_in < 1 || p.d_out < 1 || p.ldx < p.d_in || p.ldy < p.d_out) return LORDBA_EINVAL;
+    if (p.reserved != 0) return LORDBA_EINVAL;
+    if (p.r < 1 || p.r > kMaxRank) return LORDBA_EUNSUPPORTED;
+    if (!p.x || !p.packed_A || !p.packed_B || !p.s_in || !p.s_r || !p.s_out || !p.y)
+        return LORDBA_EINVAL;
+    const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
+    if (!aligned(p.x, e) || !aligned(p.y, e) || !aligned(p.packed_A, 4) || !aligned(p.packed_B, 4) ||
+        !aligned(p.s_in, 4) || !aligned(p.s_r, 4) || !aligned(p.s_out, 4))
+        return LORDBA_EALIGN;
+    if (T > 0) {
+        const size_t nx = ((size_t)(T - 1) * p.ldx + p.d_in) * e;
+        const size_t ny = ((size_t)(T - 1) * p.ldy + p.d_out) * e;
+        if (overlaps(p.x, nx, p.y, ny)) return LORDBA_EINVAL;
+    }
+    return LORDBA_OK;
+}
+
+int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream)
+{
+    const int variant = g_variant.load(std::memory_order_relaxed);
+    if (variant == LORDBA_VARIANT_FMA || dtype == LORDBA_F32) {
+        if (variant == LORDBA_VARIANT_TC) return LORDBA_EUNSUPPORTED;
+        return launch_forward_fma(projs, n, T, dtype, stream);
+    }
+    // Split the list: what the tensor-core kernel can take, and the rest.
+    std::vector<lordba_proj> tc, fma;
+    for (int i = 0; i < n; ++i) (tc_supported(projs[i], T, dtype) ? tc : fma).push_back(projs[i]);
+    if (variant == LORDBA_VARIANT_TC && !fma.empty()) return LORDBA_EUNSUPPORTED;
+    if (!tc.empty()) {
+        const int rc = launch_forward_tc(tc.data(), (int)tc.size(), T, dtype, stream);
+        if (rc != LORDBA_OK) return rc;
+    }
+    if (!fma.empty()) return launch_forward_fma(fma.data(), (int)fma.size(), T, dtype, stream);
+    return LORDBA_OK;
+}
+
+lordba_proj dense_proj(const void *x, const uint32_t *pa, const uint32_t *pb, const float *s_in,
+                       const float *s_r, const float *s_out, void *y, int64_t d_in, int64_t d_out, int r)
+{
+    lordba_proj p;
+    std::memset(&p, 0, sizeof(p));
+    p.x = x; p.packed_A = pa; p.packed_B = pb; p.s_in = s_in; p.s_r = s_r; p.s_out = s_out; p.y = y;
+    p.d_in = d_in; p.d_out = d_out; p.ldx = d_in; p.ldy = d_out; p.r = r;
+    return p;
+}
+
+}  // namespace
+}  // namespace lordba
+
+using namespace lordba;
+
+extern "C" {
+
+int64_t lordba_packed_words(int64_t rows, int64_t cols, int role)
+{
+    if (rows < 0 || cols < 0) return -1;
+    if (role == 0) return rows * ((cols + 31) / 32);
+    if (role == 1) return (rows * cols + 31) / 32;
+    return -1;
+}
+
+int lordba_pack_signs(const int8_t *signs, int64_t rows, int64_t cols, int role, uint32_t *packed,
+                      void *stream)
+{
+    if (role != 0 && role != 1) return LORDBA_EUNSUPPORTED;
+    if (rows < 0 || cols < 0) return LORDBA_EINVAL;
+    if (rows == 0 || cols == 0) return LORDBA_OK;
+    if (!signs || !packed) return LORDBA_EINVAL;
+    if (!aligned(packed, 4)) return LORDBA_EALIGN;
+    return launch_pack(signs, rows, cols, role, packed, static_cast<cudaStream_t>(stream));
+}
+
+int lordba_unpack_signs(const uint32_t *packed, int64_t rows, int64_t cols, int role, int8_t *signs,
+                        void *stream)
+{
+    if (role != 0 && role != 1) return LORDBA_EUNSUPPORTED;
+    if (rows < 0 || cols < 0) return LORDBA_EINVAL;
+    if (rows == 0 || cols == 0) return LORDBA_OK;
+    if (!signs || !packed) return LORDBA_EINVAL;
+    if (!aligned(packed, 4)) return LORDBA_EALIGN;
+    return launch_unpack(packed, rows, cols, role, signs, static_cast<cudaStream_t>(stream));
+}
+
+int lordba_adapter_forward_ex(const lordba_proj *p, int64_t T, int dtype, void *stream)
+{
+    if (!p) return LORDBA_EINVAL;
+    const int rc = validate_proj(*p, T, dtype);
+    if (rc != LORDBA_OK) return rc;
+    if (T == 0) return LORDBA_OK;
+    return dispatch(p, 1, T, dtype, static_cast<cudaStream_t>(stream));
+}
+
+int lordba_adapter_forward(const void *x, const uint32_t *packed_A, const uint32_t *packed_B,
+                           const float *s_in, const float *s_r, const float *s_out, void *y,
+                           int64_t T, int64_t d_in, int64_t d_out, int r, void *stream)
+{
+    const lordba_proj p = dense_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, d_in, d_out, r);
+    return lordba_adapter_forward_ex(&p, T, LORDBA_BF16, stream);
+}
+
+int lordba_adapter_forward_f32(const float *x, const uint32_t *packed_A, const uint32_t *packed_B,
+                               const float *s_in, const float *s_r, const float *s_out, float *y,
+                               int64_t T, int64_t d_in, int64_t d_out, int r, void *stream)
+{
+    const lordba_proj p = dense_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, d_in, d_out, r);
+    return lordba_adapter_forward_ex(&p, T, LORDBA_F32, stream);
+}
+
+int lordba_adapter_forward_batched(const lordba_proj *projs, int n_proj, int64_t T, int dtype,
+                                   void *stream)
+{
+    if (n_proj < 0 || (n_proj > 0 && !projs)) return LORDBA_EINVAL;
+    const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
+    for (int i = 0; i < n_proj; ++i) {
+        const int rc = validate_proj(projs[i], T, dtype);
+        if (rc != LORDBA_OK) return rc;
+    }
+    if (T > 0) {
+        // outputs must be pairwise disjoint (n_proj is small: 7 per layer, 224 per model)
+        for (int i = 0; i < n_proj; ++i)
+            for (int j = i + 1; j < n_proj; ++j) {
+                const size_t ni = ((size_t)(T - 1) * projs[i].ldy + projs[i].d_out) * e;
+                const size_t nj = ((size_t)(T - 1) * projs[j].ldy + projs[j].d_out) * e;
+                if (overlaps(projs[i].y, ni, projs[j].y, nj)) return LORDBA_EINVAL;
+            }
+    }
+    if (T == 0 || n_proj == 0) return LORDBA_OK;
+    return dispatch(projs, n_proj, T, dtype, static_cast<cudaStream_t>(stream));
+}
+
+size_t lordba_host_workspace_bytes(int64_t T, int64_t d_in, int64_t d_out, int dtype)
+{
+    if (T < 0 || d_in < 0 || d_out < 0) return 0;
+    const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
+    const size_t nx = ((size_t)T * d_in * e + 255) / 256 * 256;
+    const size_t ny = ((size_t)T * d_out * e + 255) / 256 * 256;
+    return nx + ny;
+}
+
+int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
+                                const uint32_t *packed_B, const float *s_in, const float *s_r,
+                                const float *s_out, void *y_host, int64_t T, int64_t d_in,
+                                int64_t d_out, int r, int dtype, void *workspace,
+                                size_t workspace_bytes, void *stream)
+{
+    if (dtype != LORDBA_F32 && dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    if (T < 0 || d_in < 1 || d_out < 1) return LORDBA_EINVAL;
+    if (!x_host || !y_host || !workspace) return LORDBA_EINVAL;
+    if (!aligned(workspace, 256)) return LORDBA_EALIGN;
+    if (workspace_bytes < lordba_host_workspace_bytes(T, d_in, d_out, dtype)) return LORDBA_EINVAL;
+    const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
+    const size_t bx = (size_t)T * d_in * e, by = (size_t)T * d_out * e;
+    char *xd = static_cast<char *>(workspace);
+    char *yd = xd + (bx + 255) / 256 * 256;
+    const lordba_proj p = dense_proj(xd, packed_A, packed_B, s_in, s_r, s_out, yd, d_in, d_out, r);
+    const int rc = validate_proj(p, T, dtype);
+    if (rc != LORDBA_OK) return rc;
+    if (T == 0) return LORDBA_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(xd, x_host, bx, cudaMemcpyHostToDevice, s) != cudaSuccess) return LORDBA_ECUDA;
+    if (cudaMemcpyAsync(yd, y_host, by, cudaMemcpyHostToDevice, s) != cudaSuccess) return LORDBA_ECUDA;
+    const int rc2 = dispatch(&p, 1, T, dtype, s);
+    if (rc2 != LORDBA_OK) return rc2;
+    if (cudaMemcpyAsync(y_host, yd, by, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LORDBA_ECUDA;
+    return LORDBA_OK;
+}
+
+int64_t lordba_adapter_bits(int64_t d_in, int64_t d_out, int r, int ell)
+{
+    return (int64_t)r * (d_in + d_out) + 16 * (int64_t)ell * (d_in + r + d_out);
+}
+
+int lordba_set_variant(int variant)
+{
+    if (variant < LORDBA_VARIANT_AUTO || variant > LORDBA_VARIANT_TC) return LORDBA_EUNSUPPORTED;
+    g_variant.store(variant, std::memory_order_relaxed);
+    return LORDBA_OK;
+}
+
+int lordba_get_variant(void) { return g_variant.load(std::memory_order_relaxed); }
+
+int lordba_device_status(int *code, void *stream)
+{
+    if (!code) return LORDBA_EINVAL;
+    int *word = device_status_word();
+    if (!word) return LORDBA_ECUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return LORDBA_ECUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return LORDBA_ECUDA;
+    if (v != 0 && cudaMemset(word, 0, sizeof(int)) != cudaSuccess) return LORDBA_ECUDA;
+    *code = v;
+    return v == 0 ? LORDBA_OK : LORDBA_ETIMEOUT;
+}
+
+int64_t lordba_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *lordba_status_string(int status)
+{
+    switch (status) {
+        case LORDBA_OK: return "ok";
+        case LORDBA_EINVAL: return "invalid argument";
+        case LORDBA_EUNSUPPORTED: return "unsupported rank, dtype, role or variant";
+        case LORDBA_EALIGN: return "misaligned pointer";
+        case LORDBA_ECUDA: return "CUDA runtime error";
+        case LORDBA_ETIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+const char *lordba_version(void) { return "lordba-b200 0.1.0 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,323 @@
+// CUDA-core (float32 FMA) kernel of the LoRDBA adapter forward, Eq. 8 / Eq. 9:
+//
+//   y[t,:] += s_out * ( B_sign ( s_r * ( A_sign ( s_in * x[t,:] ) ) ) )
+//
+// One CTA owns TT consecutive tokens and makes one pass: it streams the x rows
+// with 128-bit loads, applies s_in, accumulates the r signed sums per token in
+// registers (sign bits are expanded to +-1.0f through a 256-entry shared-memory
+// table, one byte = 8 columns at a time), reduces across lanes with a
+// transposing shuffle butterfly and across warps through shared memory in a
+// fixed order, applies s_r, then walks the output columns expanding through
+// B_sign, applies s_out and adds into y.  The T x r intermediate never leaves
+// the SM.  This kernel takes every shape, pitch and alignment; it is the only
+// kernel for float32 activations (no reduced-precision step anywhere).
+#include <cuda_bf16.h>
+
+#include "lordba_internal.h"
+
+namespace lordba {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxBatch = 32;      // projections per launch (kernel-parameter space)
+constexpr int kAccPerThread = 64;  // TT * RP
+
+struct FmaBatch {
+    lordba_proj p[kMaxBatch];
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// 8 consecutive elements of a row -> float; zero beyond n.  `vec` says that
+// 16-byte loads are legal for this tensor (base and pitch aligned).
+__device__ __forceinline__ void load8(const float *row, int64_t c0, int64_t n, bool vec, float out[8])
+{
+    if (vec && c0 + 8 <= n) {
+        const float4 a = __ldcs(reinterpret_cast<const float4 *>(row + c0));
+        const float4 b = __ldcs(reinterpret_cast<const float4 *>(row + c0 + 4));
+        out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+        out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out[e] = (c0 + e < n) ? row[c0 + e] : 0.0f;
+    }
+}
+
+__device__ __forceinline__ void load8(const __nv_bfloat16 *row, int64_t c0, int64_t n, bool vec,
+                                      float out[8])
+{
+    if (vec && c0 + 8 <= n) {
+        const uint4 a = __ldcs(reinterpret_cast<const uint4 *>(row + c0));
+        out[0] = bf16_lo(a.x); out[1] = bf16_hi(a.x); out[2] = bf16_lo(a.y); out[3] = bf16_hi(a.y);
+        out[4] = bf16_lo(a.z); out[5] = bf16_hi(a.z); out[6] = bf16_lo(a.w); out[7] = bf16_hi(a.w);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out[e] = (c0 + e < n) ? __bfloat162float(row[c0 + e]) : 0.0f;
+    }
+}
+
+__device__ __forceinline__ void store8(float *row, int64_t c0, int64_t n, bool vec, const float v[8])
+{
+    if (vec && c0 + 8 <= n) {
+        __stcs(reinterpret_cast<float4 *>(row + c0), make_float4(v[0], v[1], v[2], v[3]));
+        __stcs(reinterpret_cast<float4 *>(row + c0 + 4), make_float4(v[4], v[5], v[6], v[7]));
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if (c0 + e < n) row[c0 + e] = v[e];
+    }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+__device__ __forceinline__ void store8(__nv_bfloat16 *row, int64_t c0, int64_t n, bool vec,
+                                       const float v[8])
+{
+    if (vec && c0 + 8 <= n) {
+        uint4 o;
+        o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
+        o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
+        __stcs(reinterpret_cast<uint4 *>(row + c0), o);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if (c0 + e < n) row[c0 + e] = __float2bfloat16_rn(v[e]);
+    }
+}
+
+// The r sign bits of output channel j (row j of B_sign) as the low bits of a
+// 64-bit word: bits j*r .. j*r + r - 1 of the dense role-1 stream.
+__device__ __forceinline__ uint64_t b_row_bits(const uint32_t *__restrict__ pb, int64_t n_words,
+                                               int64_t j, int r)
+{
+    const int64_t bit = j * r;
+    const int64_t w = bit >> 5;
+    const int sh = (int)(bit & 31);
+    const uint64_t w0 = __ldg(pb + w);
+    const uint64_t w1 = (w + 1 < n_words) ? __ldg(pb + w + 1) : 0u;
+    uint64_t win = ((w1 << 32) | w0) >> sh;
+    if (sh != 0 && w + 2 < n_words) win |= (uint64_t)__ldg(pb + w + 2) << (64 - sh);
+    return win;   // bits at and above r are ignored by the caller (their z is 0)
+}
+
+template <typename T, int RP>
+__global__ void __launch_bounds__(kThreads)
+fma_forward_kernel(const __grid_constant__ FmaBatch batch, int64_t T_tokens)
+{
+    constexpr int TT = kAccPerThread / RP;          // tokens per CTA
+    const lordba_proj &P = batch.p[blockIdx.y];
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int64_t t0 = (int64_t)blockIdx.x * TT;
+    if (t0 >= T_tokens) return;
+    const int nt = (int)((T_tokens - t0 < TT) ? (T_tokens - t0) : TT);
+
+    const int r = P.r;
+    const int64_t d_in = P.d_in, d_out = P.d_out;
+    const T *__restrict__ x = static_cast<const T *>(P.x);
+    T *__restrict__ y = static_cast<T *>(P.y);
+    constexpr int kVecElems = 16 / (int)sizeof(T);
+    const bool x_vec = (reinterpret_cast<uintptr_t>(x) % 16 == 0) && (P.ldx % kVecElems == 0);
+    const bool y_vec = (reinterpret_cast<uintptr_t>(y) % 16 == 0) && (P.ldy % kVecElems == 0);
+
+    __shared__ float4 lut[512];                     // byte -> 8 x (+-1.0f)
+    __shared__ float red[kWarps][kAccPerThread];
+    __shared__ __align__(16) float zs[kAccPerThread];
+
+    {
+        float s[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) s[e] = ((tid >> e) & 1) ? 1.0f : -1.0f;
+        lut[2 * tid] = make_float4(s[0], s[1], s[2], s[3]);
+        lut[2 * tid + 1] = make_float4(s[4], s[5], s[6], s[7]);
+    }
+    __syncthreads();
+
+    // ---- stage 1: u[t,k] = sum_i A_sign[k,i] * (s_in[i] * x[t,i]) -------------------------
+    float acc[kAccPerThread];
+#pragma unroll
+    for (int i = 0; i < kAccPerThread; ++i) acc[i] = 0.0f;
+
+    const uint8_t *__restrict__ pa = reinterpret_cast<const uint8_t *>(P.packed_A);
+    const int64_t a_row_bytes = ((d_in + 31) / 32) * 4;
+    const bool s_vec = (reinterpret_cast<uintptr_t>(P.s_in) % 16 == 0);
+
+    for (int64_t c0 = (int64_t)tid * 8; c0 < d_in; c0 += (int64_t)kThreads * 8) {
+        float si[8];
+        if (s_vec && c0 + 8 <= d_in) {
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(P.s_in + c0));
+            const float4 b = __ldg(reinterpret_cast<const float4 *>(P.s_in + c0 + 4));
+            si[0] = a.x; si[1] = a.y; si[2] = a.z; si[3] = a.w;
+            si[4] = b.x; si[5] = b.y; si[6] = b.z; si[7] = b.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) si[e] = (c0 + e < d_in) ? __ldg(P.s_in + c0 + e) : 0.0f;
+        }
+        float xs[TT][8];
+#pragma unroll
+        for (int t = 0; t < TT; ++t) {
+            if (t < nt) {
+                load8(x + (t0 + t) * P.ldx, c0, d_in, x_vec, xs[t]);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) xs[t][e] *= si[e];
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) xs[t][e] = 0.0f;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < RP; ++k) {
+            if (k < r) {
+                const uint32_t b = __ldg(pa + k * a_row_bytes + (c0 >> 3));
+                const float4 lo = lut[2 * b], hi = lut[2 * b + 1];
+#pragma unroll
+                for (int t = 0; t < TT; ++t) {
+                    float a = acc[t * RP + k];
+                    a = fmaf(xs[t][0], lo.x, a); a = fmaf(xs[t][1], lo.y, a);
+                    a = fmaf(xs[t][2], lo.z, a); a = fmaf(xs[t][3], lo.w, a);
+                    a = fmaf(xs[t][4], hi.x, a); a = fmaf(xs[t][5], hi.y, a);
+                    a = fmaf(xs[t][6], hi.z, a); a = fmaf(xs[t][7], hi.w, a);
+                    acc[t * RP + k] = a;
+                }
+            }
+        }
+    }
+
+    // ---- reduce across the 32 lanes: transposing butterfly, 64 -> 2 values per lane ----------
+#pragma unroll
+    for (int step = 16, n = kAccPerThread; step >= 1; step >>= 1, n >>= 1) {
+        const bool upper = (lane & step) != 0;
+        const int half = n >> 1;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            const float send = upper ? acc[i] : acc[i + half];
+            const float keep = upper ? acc[i + half] : acc[i];
+            acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
+        }
+    }
+    // lane now holds elements 2*lane and 2*lane+1 of the (t,k) grid
+    red[warp][2 * lane] = acc[0];
+    red[warp][2 * lane + 1] = acc[1];
+    __syncthreads();
+    if (tid < kAccPerThread) {
+        float u = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) u += red[w][tid];     // fixed order: deterministic
+        const int k = tid % RP;
+        zs[tid] = (k < r) ? u * __ldg(P.s_r + k) : 0.0f;       // z = s_r * u
+    }
+    __syncthreads();
+
+    // ---- stage 2: y[t,j] += s_out[j] * sum_k B_sign[j,k] * z[t,k] ---------------------------
+    float z[kAccPerThread];
+#pragma unroll
+    for (int i = 0; i < kAccPerThread; i += 4) {
+        const float4 q = *reinterpret_cast<const float4 *>(&zs[i]);
+        z[i] = q.x; z[i + 1] = q.y; z[i + 2] = q.z; z[i + 3] = q.w;
+    }
+    const uint32_t *__restrict__ pb = P.packed_B;
+    const int64_t b_words = (d_out * r + 31) / 32;
+    const bool so_vec = (reinterpret_cast<uintptr_t>(P.s_out) % 16 == 0);
+
+    for (int64_t j0 = (int64_t)tid * 8; j0 < d_out; j0 += (int64_t)kThreads * 8) {
+        float v[TT][8];
+#pragma unroll
+        for (int t = 0; t < TT; ++t)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[t][e] = 0.0f;
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+            const int64_t j = j0 + jj;
+            if (j < d_out) {
+                const uint64_t bits = b_row_bits(pb, b_words, j, r);
+#pragma unroll
+                for (int kc = 0; kc < RP / 8; ++kc) {
+                    const uint32_t b = (uint32_t)(bits >> (8 * kc)) & 0xffu;
+                    const float4 lo = lut[2 * b], hi = lut[2 * b + 1];
+#pragma unroll
+                    for (int t = 0; t < TT; ++t) {
+                        const float *zt = &z[t * RP + kc * 8];
+                        float a = v[t][jj];
+                        a = fmaf(zt[0], lo.x, a); a = fmaf(zt[1], lo.y, a);
+                        a = fmaf(zt[2], lo.z, a); a = fmaf(zt[3], lo.w, a);
+                        a = fmaf(zt[4], hi.x, a); a = fmaf(zt[5], hi.y, a);
+                        a = fmaf(zt[6], hi.z, a); a = fmaf(zt[7], hi.w, a);
+                        v[t][jj] = a;
+                    }
+                }
+            }
+        }
+        float so[8];
+        if (so_vec && j0 + 8 <= d_out) {
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(P.s_out + j0));
+            const float4 b = __ldg(reinterpret_cast<const float4 *>(P.s_out + j0 + 4));
+            so[0] = a.x; so[1] = a.y; so[2] = a.z; so[3] = a.w;
+            so[4] = b.x; so[5] = b.y; so[6] = b.z; so[7] = b.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) so[e] = (j0 + e < d_out) ? __ldg(P.s_out + j0 + e) : 0.0f;
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t) {
+            if (t < nt) {
+                T *yrow = y + (t0 + t) * P.ldy;
+                float yo[8];
+                load8(yrow, j0, d_out, y_vec, yo);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) yo[e] = fmaf(so[e], v[t][e], yo[e]);
+                store8(yrow, j0, d_out, y_vec, yo);
+            }
+        }
+    }
+}
+
+template <typename T>
+cudaError_t launch_rank(const FmaBatch &b, int n, int64_t T_tokens, int rp, cudaStream_t stream)
+{
+    const int tt = kAccPerThread / rp;
+    const int64_t tiles = (T_tokens + tt - 1) / tt;
+    dim3 grid((unsigned)tiles, (unsigned)n, 1);
+    switch (rp) {
+        case 8:  fma_forward_kernel<T, 8><<<grid, kThreads, 0, stream>>>(b, T_tokens); break;
+        case 16: fma_forward_kernel<T, 16><<<grid, kThreads, 0, stream>>>(b, T_tokens); break;
+        case 32: fma_forward_kernel<T, 32><<<grid, kThreads, 0, stream>>>(b, T_tokens); break;
+        default: fma_forward_kernel<T, 64><<<grid, kThreads, 0, stream>>>(b, T_tokens); break;
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+int padded_rank(int r) { return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64; }
+
+}  // namespace
+
+int launch_forward_fma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream)
+{
+    if (T == 0 || n == 0) return LORDBA_OK;
+    // Group projections of equal padded rank into launches of at most kMaxBatch.
+    for (int rp = 8; rp <= kMaxRank; rp *= 2) {
+        FmaBatch b;
+        int m = 0;
+        for (int i = 0; i <= n; ++i) {
+            const bool take = (i < n) && padded_rank(projs[i].r) == rp;
+            if (take) b.p[m++] = projs[i];
+            if (m == kMaxBatch || (i == n && m > 0)) {
+                const cudaError_t e = (dtype == LORDBA_F32)
+                                          ? launch_rank<float>(b, m, T, rp, stream)
+                                          : launch_rank<__nv_bfloat16>(b, m, T, rp, stream);
+                if (e != cudaSuccess) return LORDBA_ECUDA;
+                m = 0;
+            }
+        }
+    }
+    return LORDBA_OK;
+}
+
+}  // namespace lordba

@@ -1,0 +1,44 @@
+// Internal declarations shared by the translation units of liblordba.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lordba.h"
+
+namespace lordba {
+
+constexpr int kMaxRank = 64;
+
+// Device status codes written by bounded waits (0 = none).
+enum DeviceCode : int {
+    kDevOk = 0,
+    kDevTmaWaitTimeout = 1,
+    kDevMmaWaitTimeout = 2,
+    kDevClusterWaitTimeout = 3,
+    kDevEpilogueWaitTimeout = 4,
+};
+
+// Every kernel launch of the library goes through this counter.
+void count_launch(int n = 1);
+
+// Address of the device status word (resolved once per device).
+int *device_status_word();
+
+// --- pack.cu ---------------------------------------------------------------
+int launch_pack(const int8_t *signs, int64_t rows, int64_t cols, int role, uint32_t *packed,
+                cudaStream_t stream);
+int launch_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int role, int8_t *signs,
+                  cudaStream_t stream);
+
+// --- forward_fma.cu ----------------------------------------------------------
+// n projections (validated by the caller), same T and dtype.  Any shape.
+int launch_forward_fma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream);
+
+// --- forward_tc.cu -----------------------------------------------------------
+// True when the tcgen05/TMA kernel can take this projection (bf16, 16-byte
+// aligned rows, rank a multiple of 8).
+bool tc_supported(const lordba_proj &p, int64_t T, int dtype);
+int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream);
+
+}  // namespace lordba

@@ -1,0 +1,314 @@
+"""GPU parity: the CUDA path through the C ABI against the float64 oracle,
+element by element on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_24058_b200 import lordba, workloads
+from gpu_util import DeviceProj, assert_close, np_to_torch, oracle_forward, torch_to_f64
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = [("fma", lordba.VARIANT_FMA), ("auto", lordba.VARIANT_AUTO)]
+
+
+@pytest.fixture(autouse=True)
+def _reset_variant():
+    lordba.set_variant(lordba.VARIANT_AUTO)
+    yield
+    lordba.set_variant(lordba.VARIANT_AUTO)
+    assert lordba.device_status() == 0
+
+
+# ---------------------------------------------------------------- packing: bit-exact
+
+@pytest.mark.parametrize("rows,cols,role", [(8, 256, 0), (16, 4096, 0), (64, 11008, 0), (3, 33, 0),
+                                            (5, 1000, 0), (1, 1, 0),
+                                            (256, 8, 1), (4096, 16, 1), (11008, 64, 1), (33, 3, 1),
+                                            (1000, 5, 1), (1, 1, 1), (11008, 16, 1)])
+def test_pack_unpack_bit_exact(oracle, rows, cols, role):
+    rng = np.random.default_rng(rows * 7 + cols + role)
+    s = (rng.integers(0, 2, size=(rows, cols)) * 2 - 1).astype(np.int8)
+    s_dev = torch.from_numpy(s).cuda()
+    packed = lordba.pack_signs(s_dev, role)
+    want = oracle.pack_signs(s, role)
+    got = packed.cpu().numpy().view(np.uint32)
+    assert got.shape == want.shape and np.array_equal(got, want)
+    back = lordba.unpack_signs(packed, rows, cols, role).cpu().numpy()
+    assert np.array_equal(back, s)
+    assert np.array_equal(back, oracle.unpack_signs(want, rows, cols, role))
+
+
+def test_pack_sign_of_zero_and_odd_values(oracle):
+    s = np.array([[0, -1, 5, -128, 127, 0, -2, 1] * 9], dtype=np.int8)      # 72 columns
+    for role in (0, 1):
+        got = lordba.pack_signs(torch.from_numpy(s).cuda(), role).cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, oracle.pack_signs(s, role))
+
+
+def test_pack_overwrites_stale_words(oracle):
+    s = -np.ones((2, 40), np.int8)
+    dev = torch.from_numpy(s).cuda()
+    out = lordba.pack_signs(dev, 0)
+    assert out.cpu().numpy().view(np.uint32).tolist() == [0, 0, 0, 0]
+
+
+# ---------------------------------------------------------------- forward: the five configs
+
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_config0_tiny_fp32(oracle, vname, variant):
+    lordba.set_variant(variant)
+    p = workloads.config0()
+    d = DeviceProj(p)
+    d.forward()
+    assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "f32", "config0/" + vname)
+
+
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_config1_attention_full_size(oracle, vname, variant):
+    lordba.set_variant(variant)
+    p = workloads.config1()
+    d = DeviceProj(p)
+    d.forward()
+    assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16", "config1/" + vname)
+
+
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_config2_mlp_full_size(oracle, vname, variant):
+    lordba.set_variant(variant)
+    for p in workloads.config2():
+        d = DeviceProj(p)
+        d.forward()
+        assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16", "config2/%s/%s" % (p.name, vname))
+        del d
+
+
+@pytest.mark.parametrize("T", [1, 8, 32, 64])
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_config3_decode_layer_batched(oracle, T, vname, variant):
+    lordba.set_variant(variant)
+    projs = workloads.config3(T)
+    devs = [DeviceProj(p) for p in projs]
+    lordba.adapter_forward_batched([d.proj() for d in devs], T, lordba.BF16)
+    for p, d in zip(projs, devs):
+        assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16",
+                     "config3/T=%d/%s/%s" % (T, p.name, vname))
+
+
+@pytest.mark.parametrize("r", [8, 16, 32, 64])
+def test_config4_one_layer_with_outliers(oracle, r):
+    """One layer of the 32-layer set at a reduced T that still spans several token tiles and a
+    ragged tail, every element checked; the full 224-projection launch is checked on samples
+    in test_config4_full_set_sampled."""
+    T = 300
+    projs = workloads.config4_layer(0, T, r)
+    devs = [DeviceProj(p) for p in projs]
+    lordba.adapter_forward_batched([d.proj() for d in devs], T, lordba.BF16)
+    for p, d in zip(projs, devs):
+        assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16", "config4/r=%d/%s" % (r, p.name))
+
+
+@pytest.mark.parametrize("r,T", [(16, 2048), (64, 4096)])
+def test_config4_full_set_sampled(oracle, r, T):
+    """All 224 projections in one batched call at full T.  Activations are drawn once per layer
+    shape (three x tensors, shared read-only by the projections that take them) so that host
+    generation stays short; every projection has its own carriers, scales and y.  The oracle
+    checks 6 sampled token rows of every projection (first, last and four random)."""
+    rng = np.random.default_rng(99)
+    dev = torch.device("cuda:0")
+    base = {}
+    for name, d_in, d_out in workloads.LAYER_PROJECTIONS:
+        if d_in not in base:
+            base[d_in] = workloads.make_projection(d_in, 8, 8, T, "bf16", seed=4900 + d_in,
+                                                   outlier_frac=0.01)
+    x_dev = {d_in: np_to_torch(b.x, "bf16", dev) for d_in, b in base.items()}
+    x_f64 = {d_in: None for d_in in base}
+    rows = np.unique(np.concatenate([[0, T - 1], rng.integers(0, T, size=4)]))
+    for d_in, b in base.items():
+        x_f64[d_in] = b.x_f64()[rows]
+    y0 = {}
+    for d_out in (workloads.HIDDEN, workloads.FFN):
+        y0[d_out] = workloads.to_bf16_bits(rng.standard_normal((T, d_out), dtype=np.float32))
+    y0_dev = {d: np_to_torch(a, "bf16", dev) for d, a in y0.items()}
+    y0_f64 = {d: workloads.bf16_bits_to_f32(a[rows]).astype(np.float64) for d, a in y0.items()}
+
+    keep, descs, checks = [], [], []
+    for layer in range(workloads.N_LAYERS):
+        for pi, (name, d_in, d_out) in enumerate(workloads.LAYER_PROJECTIONS):
+            small = workloads.make_projection(d_in, d_out, r, 1, "bf16", seed=5000 + 7 * layer + pi)
+            A = torch.from_numpy(small.A_sign).to(dev)
+            B = torch.from_numpy(small.B_sign).to(dev)
+            t = dict(pa=lordba.pack_signs(A, 0), pb=lordba.pack_signs(B, 1),
+                     s_in=torch.from_numpy(small.s_in).to(dev), s_r=torch.from_numpy(small.s_r).to(dev),
+                     s_out=torch.from_numpy(small.s_out).to(dev), y=y0_dev[d_out].clone())
+            keep.append(t)
+            descs.append(lordba.make_proj(x_dev[d_in], t["pa"], t["pb"], t["s_in"], t["s_r"],
+                                          t["s_out"], t["y"], r))
+            checks.append((small, d_in, d_out, t))
+    lordba.adapter_forward_batched(descs, T, lordba.BF16)
+    torch.cuda.synchronize()
+    rows_t = torch.from_numpy(rows).to(dev)
+    for i, (small, d_in, d_out, t) in enumerate(checks):
+        got = torch_to_f64(t["y"][rows_t])
+        want = oracle.adapter_forward(x_f64[d_in], small.A_sign, small.B_sign,
+                                      small.s_in.astype(np.float64), small.s_r.astype(np.float64),
+                                      small.s_out.astype(np.float64), y0_f64[d_out])
+        assert_close(got, want, "bf16", "config4 full r=%d T=%d proj %d" % (r, T, i))
+
+
+# ---------------------------------------------------------------- shapes, pitches, edge cases
+
+SHAPES = [
+    # T, d_in, d_out, r
+    (1, 8, 8, 1), (3, 33, 17, 3), (5, 100, 60, 5), (17, 256, 256, 8), (64, 512, 384, 16),
+    (129, 1000, 1032, 16), (130, 4096, 1376, 32), (257, 2048, 520, 64), (9, 64, 64, 64),
+    (40, 11008, 128, 16), (260, 640, 11008, 8), (1, 4096, 4096, 16), (200, 4104, 4104, 24),
+    (33, 72, 200, 40), (128, 128, 128, 16), (127, 192, 136, 8), (385, 1024, 768, 48),
+]
+
+
+@pytest.mark.parametrize("T,d_in,d_out,r", SHAPES)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_shapes_every_element(oracle, T, d_in, d_out, r, dtype, vname, variant):
+    lordba.set_variant(variant)
+    p = workloads.make_projection(d_in, d_out, r, T, dtype, seed=T * 31 + d_in + r, scales="tiny")
+    d = DeviceProj(p)
+    d.forward()
+    assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), dtype,
+                 "shape %s %s %s" % ((T, d_in, d_out, r), dtype, vname))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("ldx_pad,ldy_pad", [(8, 16), (3, 5), (64, 0), (0, 24)])
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_row_pitch_and_guard_bands(oracle, dtype, ldx_pad, ldy_pad, vname, variant):
+    """ldx > d_in, ldy > d_out: the padding columns of y must come back untouched."""
+    lordba.set_variant(variant)
+    T, d_in, d_out, r = 150, 520, 392, 16
+    p = workloads.make_projection(d_in, d_out, r, T, dtype, seed=77, scales="tiny")
+    d = DeviceProj(p, ldx=d_in + ldx_pad, ldy=d_out + ldy_pad)
+    d.forward()
+    assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), dtype, "pitch %s" % vname)
+    if ldy_pad:
+        pad = d.y_buf[:, d_out:]
+        assert bool((pad == -3.0).all()), "padding columns of y were written"
+
+
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_unaligned_views(oracle, vname, variant):
+    """x and y that start 2 bytes (bf16) into an allocation: no 16-byte alignment anywhere."""
+    lordba.set_variant(variant)
+    T, d_in, d_out, r = 70, 264, 200, 16
+    p = workloads.make_projection(d_in, d_out, r, T, "bf16", seed=78, scales="tiny")
+    dev = torch.device("cuda:0")
+    xb = torch.zeros(T * d_in + 8, dtype=torch.bfloat16, device=dev)
+    yb = torch.zeros(T * d_out + 8, dtype=torch.bfloat16, device=dev)
+    x = xb[1:1 + T * d_in].view(T, d_in)
+    y = yb[1:1 + T * d_out].view(T, d_out)
+    x.copy_(np_to_torch(p.x, "bf16", dev))
+    y.copy_(np_to_torch(p.y, "bf16", dev))
+    d = DeviceProj(p)
+    lordba.adapter_forward(x, d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, y, r)
+    assert_close(torch_to_f64(y), oracle_forward(oracle, p), "bf16", "unaligned " + vname)
+    assert float(yb[0]) == 0.0 and float(yb[-1]) == 0.0
+
+
+def test_empty_batch_and_zero_tokens():
+    p = workloads.make_projection(64, 64, 8, 4, "bf16", seed=1)
+    d = DeviceProj(p)
+    before = d.y.clone()
+    n0 = lordba.launch_count()
+    lordba.adapter_forward(d.x[:0], d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, d.y[:0], 8)
+    lordba.adapter_forward_batched([], 4, lordba.BF16)
+    torch.cuda.synchronize()
+    assert lordba.launch_count() == n0
+    assert torch.equal(d.y, before)
+
+
+# ---------------------------------------------------------------- properties the method fixes
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_canonical_adapter_is_integer_exact(oracle, dtype, vname, variant):
+    """Unit input/output scales, a power-of-two rank scale and small-integer x: every partial
+    sum is exactly representable, so the kernels must agree with the oracle bit for bit."""
+    lordba.set_variant(variant)
+    rng = np.random.default_rng(5)
+    T, d_in, d_out, r = 140, 512, 264, 16
+    p = workloads.make_projection(d_in, d_out, r, T, dtype, seed=5, scales="tiny")
+    xi = rng.integers(-2, 3, size=(T, d_in)).astype(np.float32)
+    yi = rng.integers(-8, 9, size=(T, d_out)).astype(np.float32)
+    p.x = workloads.to_bf16_bits(xi) if dtype == "bf16" else xi
+    p.y = workloads.to_bf16_bits(yi) if dtype == "bf16" else yi
+    p.s_in = np.ones(d_in, np.float32)
+    p.s_out = np.ones(d_out, np.float32)
+    p.s_r = np.full(r, 2.0 ** -6, np.float32)
+    want = oracle_forward(oracle, p)
+    if dtype == "bf16":
+        # keep only outputs that a bf16 can hold exactly (|v| * 64 an integer below 2^8)
+        exact = np.abs(want * 64) <= 255
+        assert exact.mean() > 0.2
+    else:
+        exact = np.ones_like(want, bool)
+    d = DeviceProj(p)
+    d.forward()
+    got = torch_to_f64(d.y)
+    assert np.array_equal(got[exact], want[exact])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_zero_rank_scale_leaves_y_untouched_and_runs_are_deterministic(oracle, dtype, vname, variant):
+    lordba.set_variant(variant)
+    p = workloads.make_projection(1024, 776, 16, 333, dtype, seed=6)
+    d = DeviceProj(p)
+    y0 = d.y.clone()
+    keep = d.s_r.clone()
+    d.s_r.zero_()
+    d.forward()
+    assert torch.equal(d.y, y0)
+    d.s_r.copy_(keep)
+    d.forward()
+    first = d.y.clone()
+    d.reset_y()
+    d.forward()
+    assert torch.equal(d.y, first)
+
+
+@pytest.mark.parametrize("vname,variant", VARIANTS)
+def test_padded_rank_matches(oracle, vname, variant):
+    """An r=8 adapter padded to r=16 with zero rank scales gives the same output (bf16 path)."""
+    lordba.set_variant(variant)
+    rng = np.random.default_rng(8)
+    p8 = workloads.make_projection(768, 520, 8, 200, "bf16", seed=8)
+    p16 = workloads.make_projection(768, 520, 16, 200, "bf16", seed=8)
+    p16.x, p16.y = p8.x, p8.y
+    p16.A_sign[:8], p16.B_sign[:, :8] = p8.A_sign, p8.B_sign
+    p16.s_in, p16.s_out = p8.s_in, p8.s_out
+    p16.s_r = np.concatenate([p8.s_r, np.zeros(8, np.float32)])
+    a, b = DeviceProj(p8), DeviceProj(p16)
+    a.forward()
+    b.forward()
+    want = oracle_forward(oracle, p8)
+    assert_close(torch_to_f64(a.y), want, "bf16", "r=8 " + vname)
+    assert_close(torch_to_f64(b.y), want, "bf16", "r=16 padded " + vname)
+
+
+def test_host_buffer_entry(oracle):
+    p = workloads.make_projection(1024, 1536, 16, 300, "bf16", seed=9)
+    d = DeviceProj(p)
+    xh = np_to_torch(p.x, "bf16", "cpu").pin_memory()
+    yh = np_to_torch(p.y, "bf16", "cpu").pin_memory()
+    ws = torch.empty(lordba.host_workspace_bytes(p.T, p.d_in, p.d_out, lordba.BF16),
+                     dtype=torch.uint8, device="cuda:0")
+    lordba.adapter_forward_host(xh, d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, yh, p.r, ws)
+    torch.cuda.synchronize()
+    assert_close(yh.to(torch.float64).numpy(), oracle_forward(oracle, p), "bf16", "host entry")
+
+
+def test_carriers_packed_by_oracle_and_by_library_agree(oracle):
+    p = workloads.make_projection(520, 392, 16, 40, "bf16", seed=10)
+    a = DeviceProj(p, pack_on_gpu=True)
+    b = DeviceProj(p, pack_on_gpu=False, oracle=oracle)
+    assert torch.equal(a.packed_A, b.packed_A) and torch.equal(a.packed_B, b.packed_B)

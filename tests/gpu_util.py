@@ -5,12 +5,18 @@ import torch
 
 from paper_2605_24058_b200 import lordba, workloads
 
-# Acceptance bounds: float32 I/O: max|err| <= 1e-5 * max|y'|;
-# bfloat16 I/O (float32 accumulation): max|err| <= 2e-2 * rms(y'); y' = oracle output.
+# Acceptance bounds (y' = oracle output, norms over the whole output tensor of the call):
+#   float32 I/O:  max|err| <= 1e-5 * max|y'|
+#   bfloat16 I/O: max|err| <= 2e-2 * rms(y'), float32 accumulation.
+# A bfloat16 output carries 8 significant bits, so storing even the exact result costs up to
+# 2^-8 |y'|; with the heavy-tailed s_out of the workloads some outputs exceed 5 rms(y') and
+# their correct rounding alone is larger than 2e-2 rms(y').  The 2e-2 rms bound is therefore
+# asserted as stated on every element with |y'| <= 5 rms(y') (2^-8 * 5 < 2e-2), and every
+# element, large ones included, is held to the tighter arithmetic bound below.
 F32_REL_INF = 1e-5
 BF16_REL_RMS = 2e-2
-# Tighter bound the bf16 kernels are also held to: half a bf16 ulp of the exact
-# result for the one final rounding (8 significant bits: at most 2^-8 |y'|) plus
+BF16_RAW_BOUND_REGION = 5.0
+# Half a bf16 ulp of the exact result for the one final rounding (at most 2^-8 |y'|) plus
 # 2^-12 rms(y') for everything before it (split bf16 operands, fp32 summation order).
 BF16_HALF_ULP = 2.0 ** -8
 BF16_PRE_ROUNDING = 2.0 ** -12
@@ -85,7 +91,10 @@ def assert_close(got: np.ndarray, want: np.ndarray, dtype: str, what: str = "", 
     else:
         rms = float(np.sqrt(np.mean(ref * ref)))
         bound = BF16_REL_RMS * rms
-        assert err.max() <= bound, "%s: max err %.3e > %.3e" % (what, err.max(), bound)
+        region = np.abs(want) <= BF16_RAW_BOUND_REGION * rms
+        if region.any():
+            worst = err[region].max()
+            assert worst <= bound, "%s: max err %.3e > %.3e" % (what, worst, bound)
         tight = BF16_HALF_ULP * np.abs(want) + BF16_PRE_ROUNDING * rms
         bad = err > tight
         assert not bad.any(), "%s: %d elements beyond the bf16 rounding bound, worst %.3e vs %.3e" % (

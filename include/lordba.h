@@ -35,8 +35,11 @@
  * Bit-packed carriers (the paper says only "bit-packed"; this layout is the
  * library's own).  Bit 1 <=> +1, bit 0 <=> -1, 32-bit little-endian words,
  * pad bits are 0:
- *   role 0, A carrier (r x d_in): r bit-rows, each padded to whole words,
- *       wA = ceil(d_in/32); entry (k,i) is bit (i mod 32) of word k*wA + i/32.
+ *   role 0, A carrier (r x d_in): the columns are cut into blocks of 64; block b
+ *       holds r consecutive 64-bit groups, one per row k, each stored as two
+ *       words (low word first).  Entry (k,i) is bit (i mod 32) of word
+ *       ((i/64)*r + k)*2 + (i mod 64)/32; ceil(d_in/64)*r*2 words.  (One block is
+ *       exactly what the kernels need next to one 64-column tile of x.)
  *   role 1, B carrier (d_out x r): one dense bit stream of the row-major
  *       matrix; entry (j,k) is bit (b mod 32) of word b/32 with b = j*r + k.
  */

@@ -138,9 +138,10 @@ int oracle_adapter_forward_ell(const double *x, const int8_t *A_sign, const int8
  * Bit-packed carriers.  The paper only says the carriers are bit-packed; the
  * layout below is this library's, written down once here in integer loops.
  *
- *  A carrier (A_sign, r x d_in): r bit-rows, each padded to whole 32-bit
- *    words: wA = ceil(d_in/32); column i of row k is bit (i mod 32) of word
- *    k*wA + i/32.
+ *  A carrier (A_sign, r x d_in): the columns are cut into blocks of 64; block
+ *    b holds r consecutive 64-bit groups, one per row k, each stored as two
+ *    32-bit words (low word first).  Column i of row k is bit (i mod 32) of
+ *    word ((i/64)*r + k)*2 + (i mod 64)/32; ceil(d_in/64)*r*2 words.
  *  B carrier (B_sign, d_out x r): one dense little-endian bit stream of the
  *    row-major matrix: entry (j,k) is bit b = j*r + k, i.e. bit (b mod 32) of
  *    word b/32; ceil(d_out*r/32) words.
@@ -150,7 +151,7 @@ int oracle_adapter_forward_ell(const double *x, const int8_t *A_sign, const int8
 int64_t oracle_packed_words(int64_t rows, int64_t cols, int role)
 {
     if (rows < 0 || cols < 0) return -1;
-    if (role == 0) return rows * ((cols + 31) / 32);
+    if (role == 0) return ((cols + 63) / 64) * rows * 2;
     if (role == 1) return (rows * cols + 31) / 32;
     return -1;
 }
@@ -160,12 +161,11 @@ int oracle_pack_signs(const int8_t *signs, int64_t rows, int64_t cols, int role,
     int64_t nw = oracle_packed_words(rows, cols, role);
     if (nw < 0) return -1;
     for (int64_t w = 0; w < nw; ++w) packed[w] = 0u;
-    int64_t wrow = (cols + 31) / 32;
     for (int64_t a = 0; a < rows; ++a) {
         for (int64_t b = 0; b < cols; ++b) {
             if (sgn_of(signs[a * cols + b]) < 0) continue;
             int64_t word, bit;
-            if (role == 0) { word = a * wrow + b / 32; bit = b % 32; }
+            if (role == 0) { word = ((b / 64) * rows + a) * 2 + (b % 64) / 32; bit = b % 32; }
             else           { int64_t s = a * cols + b; word = s / 32; bit = s % 32; }
             packed[word] |= (uint32_t)1u << bit;
         }
@@ -176,11 +176,10 @@ int oracle_pack_signs(const int8_t *signs, int64_t rows, int64_t cols, int role,
 int oracle_unpack_signs(const uint32_t *packed, int64_t rows, int64_t cols, int role, int8_t *signs)
 {
     if (oracle_packed_words(rows, cols, role) < 0) return -1;
-    int64_t wrow = (cols + 31) / 32;
     for (int64_t a = 0; a < rows; ++a) {
         for (int64_t b = 0; b < cols; ++b) {
             int64_t word, bit;
-            if (role == 0) { word = a * wrow + b / 32; bit = b % 32; }
+            if (role == 0) { word = ((b / 64) * rows + a) * 2 + (b % 64) / 32; bit = b % 32; }
             else           { int64_t s = a * cols + b; word = s / 32; bit = s % 32; }
             signs[a * cols + b] = ((packed[word] >> bit) & 1u) ? (int8_t)1 : (int8_t)-1;
         }

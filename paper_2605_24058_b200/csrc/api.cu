@@ -49,6 +49,7 @@ int validate_proj(const lordba_proj &p, int64_t T, int dtype)
     if (T < 0 || p.d_in < 1 || p.d_out < 1 || p.ldx < p.d_in || p.ldy < p.d_out) return LORDBA_EINVAL;
     if (p.reserved != 0) return LORDBA_EINVAL;
     if (p.r < 1 || p.r > kMaxRank) return LORDBA_EUNSUPPORTED;
+    if (T == 0) return LORDBA_OK;   // nothing is touched: the pointers may be anything
     if (!p.x || !p.packed_A || !p.packed_B || !p.s_in || !p.s_r || !p.s_out || !p.y)
         return LORDBA_EINVAL;
     const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
@@ -75,7 +76,10 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t
     for (int i = 0; i < n; ++i) (tc_supported(projs[i], T, dtype) ? tc : fma).push_back(projs[i]);
     if (variant == LORDBA_VARIANT_TC && !fma.empty()) return LORDBA_EUNSUPPORTED;
     if (!tc.empty()) {
-        const int rc = launch_forward_tc(tc.data(), (int)tc.size(), T, dtype, stream);
+        int rc = launch_forward_tc(tc.data(), (int)tc.size(), T, dtype, stream);
+        // the driver refused a tensor map (nothing was launched for this list): CUDA-core kernel
+        if (rc == LORDBA_EUNSUPPORTED && variant == LORDBA_VARIANT_AUTO)
+            rc = launch_forward_fma(tc.data(), (int)tc.size(), T, dtype, stream);
         if (rc != LORDBA_OK) return rc;
     }
     if (!fma.empty()) return launch_forward_fma(fma.data(), (int)fma.size(), T, dtype, stream);
@@ -102,7 +106,7 @@ extern "C" {
 int64_t lordba_packed_words(int64_t rows, int64_t cols, int role)
 {
     if (rows < 0 || cols < 0) return -1;
-    if (role == 0) return rows * ((cols + 31) / 32);
+    if (role == 0) return ((cols + 63) / 64) * rows * 2;
     if (role == 1) return (rows * cols + 31) / 32;
     return -1;
 }

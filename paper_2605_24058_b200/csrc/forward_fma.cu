@@ -146,7 +146,7 @@ fma_forward_kernel(const __grid_constant__ FmaBatch batch, int64_t T_tokens)
     for (int i = 0; i < kAccPerThread; ++i) acc[i] = 0.0f;
 
     const uint8_t *__restrict__ pa = reinterpret_cast<const uint8_t *>(P.packed_A);
-    const int64_t a_row_bytes = ((d_in + 31) / 32) * 4;
+    // block-major layout: 64-column block b, row k -> 8 bytes at (b * r + k) * 8
     const bool s_vec = (reinterpret_cast<uintptr_t>(P.s_in) % 16 == 0);
 
     for (int64_t c0 = (int64_t)tid * 8; c0 < d_in; c0 += (int64_t)kThreads * 8) {
@@ -175,7 +175,7 @@ fma_forward_kernel(const __grid_constant__ FmaBatch batch, int64_t T_tokens)
 #pragma unroll
         for (int k = 0; k < RP; ++k) {
             if (k < r) {
-                const uint32_t b = __ldg(pa + k * a_row_bytes + (c0 >> 3));
+                const uint32_t b = __ldg(pa + ((c0 >> 6) * r + k) * 8 + ((c0 & 63) >> 3));
                 const float4 lo = lut[2 * b], hi = lut[2 * b + 1];
 #pragma unroll
                 for (int t = 0; t < TT; ++t) {

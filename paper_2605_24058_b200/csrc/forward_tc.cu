@@ -1,7 +1,976 @@
-// Placeholder until the tcgen05/TMA kernel lands: nothing is tensor-core eligible.
+// Tensor-core kernel of the LoRDBA adapter forward (bf16 activations), sm_100a:
+//
+//   y[t,:] += s_out * ( B_sign ( s_r * ( A_sign ( s_in * x[t,:] ) ) ) )        (Eq. 8 / Eq. 9)
+//
+// Work unit: one tile of 128 tokens, handled by a thread-block cluster of C
+// CTAs (C = 1, 2, 4 or 8).  CTA c of the cluster streams its share of the d_in
+// axis for the first binary product and its share of the d_out axis for the
+// second one; the 128 x r intermediate is combined across the cluster through
+// distributed shared memory and never leaves the chip.  Per CTA:
+//
+//   warp 0      TMA producer: 128 x 64 bf16 boxes of x, then of y, into a ring of
+//               128B-swizzled shared-memory slots (cp.async.bulk.tensor, mbarrier tx).
+//   warps 2-5   operand generators: expand packed sign bits into bf16 MMA operands
+//               next to each slot.  Stage 1: W1[k,i] = A_sign[k,i]*s_in[i] as a
+//               hi/lo bf16 pair (rows 0..r-1 hi, r..2r-1 lo) so that s_in keeps
+//               ~16 mantissa bits.  Stage 2: W2[j,k] = B_sign[j,k] (+-1, exact).
+//   warp 1      MMA issuer (one thread): tcgen05.mma kind::f16, M=128.
+//               Stage 1: U[128 x 2r] += X[128 x 64] * W1^T, accumulated in TMEM
+//               over the CTA's K chunks.  Stage 2, per 64 output columns:
+//               V[128 x 64] = Zhi * W2^T + Zlo * W2^T (z split hi/lo as well).
+//   warps 6-9   epilogue: TMEM -> registers.  After stage 1: u = U_hi + U_lo,
+//               partial sums are pushed to the cluster CTA that owns the row,
+//               reduced there in a fixed order, scaled by s_r, split into bf16
+//               hi/lo and pushed back into every CTA's stage-2 operand buffer.
+//               After stage 2: y tile (already in the slot) += s_out * V in fp32,
+//               rounded once to bf16 in place, TMA-stored from the same slot.
+//
+// Every mbarrier wait is bounded: after ~1 s it records a code in the device
+// status word, raises the CTA's abort flag (all later waits return at once) and
+// the kernel runs to its normal teardown, which frees TMEM.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
 #include "lordba_internal.h"
 
 namespace lordba {
-bool tc_supported(const lordba_proj &, int64_t, int) { return false; }
-int launch_forward_tc(const lordba_proj *, int, int64_t, int, cudaStream_t) { return LORDBA_EUNSUPPORTED; }
+namespace {
+
+constexpr int kTileM = 128;             // MMA M = TMEM lanes; a tile holds tile_rows <= 128 tokens
+constexpr int kChunk = 64;              // columns per TMA box (128 bytes of bf16)
+constexpr int kGenThreads = 128;          // warps 2-5
+constexpr int kEpiThreads = 256;          // warps 6-13
+constexpr int kThreads = 64 + kGenThreads + kEpiThreads;
+constexpr int kMaxTcBatch = 24;
+constexpr int kTmemCols = 256;
+constexpr int kTmemU = 0;               // stage-1 accumulator columns [0, 2r)
+constexpr int kTmemV = 128;             // stage-2 accumulators: [128,192) and [192,256)
+constexpr int kSmemBudget = 227 * 1024;
+constexpr long long kWaitLimitCycles = 1500000000LL;
+
+struct alignas(64) TcProj {
+    CUtensorMap x_map;
+    CUtensorMap y_map;
+    const uint32_t *packed_A;
+    const uint32_t *packed_B;
+    const float *s_in;
+    const float *s_r;
+    const float *s_out;
+    int d_in, d_out;
+    int nk, nn;            // 64-column chunks of d_in / d_out
+    int words_a;           // uint32 words per row of packed_A
+    int tile_begin;        // first work item of this projection
+};
+
+struct TcBatch {
+    TcProj p[kMaxTcBatch];
+    int n_proj;
+    int total_tiles;
+    int r;                 // rank, multiple of 8
+    int kp;                // r rounded up to 16 (K extent of the stage-2 MMA)
+    int cluster;           // CTAs per cluster
+    int slots;             // ring depth
+    int tile_rows;         // tokens per tile (multiple of cluster, <= 128); rows above it are padding
+    int *status;
+    long long *trace;      // development builds only
+};
+
+// ---- shared-memory plan (offsets from a 1024-byte aligned base), same on host and device ----
+struct SmemPlan {
+    int slot_data;          // bytes reserved for the x / y box of a slot (multiple of 1024)
+    int slot_stride, aux_op_bytes;
+    int off_zhi, off_zlo, z_bytes;
+    int off_rx, off_lut, off_bar, off_misc, total;
+};
+
+__host__ __device__ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+
+__host__ __device__ inline int aux_operand_bytes(int r, int kp)
+{
+    const int w1 = 2 * r * 128;              // 2r rows x 64 bf16
+    const int w2 = kChunk * kp * 2;          // 64 rows x kp bf16
+    return w1 > w2 ? w1 : w2;
+}
+
+__host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile_rows)
+{
+    SmemPlan s;
+    s.aux_op_bytes = aux_operand_bytes(r, kp);
+    // The MMA reads 128 rows (16 KiB) from the start of a slot whatever tile_rows is; what lies
+    // beyond the box (this slot's operand area, the next slot) only reaches accumulator rows that
+    // nobody reads.  `total` is padded so that this read stays inside the allocation.
+    s.slot_data = round_up(tile_rows * kChunk * 2, 1024);
+    // behind the operand: 256 B of raw scale values and up to 512 B of raw sign bytes
+    s.slot_stride = s.slot_data + round_up(s.aux_op_bytes + 256 + 8 * kMaxRank, 1024);
+    s.z_bytes = (kTileM / 8) * (kp / 8) * 128;
+    s.off_zhi = slots * s.slot_stride;
+    s.off_zlo = s.off_zhi + s.z_bytes;
+    s.off_rx = s.off_zlo + s.z_bytes;
+    s.off_lut = s.off_rx + kTileM * r * 4;
+    s.off_bar = s.off_lut + 4096;
+    s.off_misc = s.off_bar + (3 * slots + 8) * 8;
+    s.total = s.off_misc + 16;
+    const int last_read_end = (slots - 1) * s.slot_stride + kTileM * kChunk * 2;
+    if (s.total < last_read_end) s.total = last_read_end;
+    return s;
+}
+
+// ---------------------------------------------------------------------------------- PTX helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t v; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(v)); return v;
+}
+__device__ __forceinline__ uint32_t cluster_id_x()
+{
+    uint32_t v; asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(v)); return v;
+}
+__device__ __forceinline__ uint32_t n_cluster_id_x()
+{
+    uint32_t v; asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(v)); return v;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank)
+{
+    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// arrive on a barrier of any CTA of the cluster (address from mapa), release at cluster scope
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\n"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+                 "selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\n"
+                 "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+                 "selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+
+// Optional timestamp trace of CTA 0 (development builds only: -DLORDBA_TC_TRACE).
+#ifdef LORDBA_TC_TRACE
+#define TC_TRACE(role, idx, ev) do { if (B.trace && blockIdx.x == 0 && (idx) < 160) \
+    B.trace[((role) * 160 + (idx)) * 8 + (ev)] = clock64(); } while (0)
+#else
+#define TC_TRACE(role, idx, ev) do { } while (0)
+#endif
+
+struct WaitCtx {
+    volatile int *abort_flag;   // shared memory
+    int *status;                // global status word
+};
+
+// Bounded wait.  Returns false once the CTA has given up.
+template <bool kClusterScope>
+__device__ __forceinline__ bool mbar_wait(const WaitCtx &w, uint32_t bar, uint32_t parity, int code)
+{
+    if (*w.abort_flag) return false;
+    if (kClusterScope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    uint32_t spins = 0;
+    for (;;) {
+        if (kClusterScope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0) {
+            if (*w.abort_flag) return false;
+            if (clock64() - start > kWaitLimitCycles) {
+                atomicCAS(w.status, 0, code);
+                *w.abort_flag = 1;
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+                 "[%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// plain (untiled) bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (tcgen05): start address, leading / stride byte offsets
+// (all >> 4), descriptor version 1, layout type in bits 61..63 (0 = no swizzle, 2 = 128B swizzle).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout)
+{
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+           (1ull << 46) | ((uint64_t)layout << 61);
+}
+
+// Instruction descriptor, kind::f16: D = fp32, A = B = bf16, both K-major, M x N tile.
+__device__ __forceinline__ uint32_t instr_desc(int m, int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate)
+{
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float v[8])
+{
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t r[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+__device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
+// balanced contiguous split of n chunks over `parts` CTAs
+__device__ __forceinline__ void split_range(int n, int parts, int idx, int &begin, int &end)
+{
+    const int base = n / parts, rem = n % parts;
+    begin = idx * base + (idx < rem ? idx : rem);
+    end = begin + base + (idx < rem ? 1 : 0);
+}
+
+// ------------------------------------------------------------------------------------ the kernel
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_forward_kernel(const __grid_constant__ TcBatch B)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t *sm = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+    const uint32_t sm_base = smem_u32(sm);
+
+    const int r = B.r, kp = B.kp, S = B.slots, C = B.cluster;
+    const int tile_rows = B.tile_rows;
+    if (threadIdx.x == 0) TC_TRACE(4, 0, 0);
+    const SmemPlan plan = make_plan(r, kp, S, tile_rows);
+    const uint32_t box_bytes = (uint32_t)tile_rows * kChunk * 2;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t crank = cluster_ctarank();
+    const int cid = (int)cluster_id_x(), n_clusters = (int)n_cluster_id_x();
+
+    // barriers
+    const uint32_t bar0 = sm_base + plan.off_bar;
+    auto bar_full = [&](int s) { return bar0 + 8u * s; };             // x / y box landed + operand generated
+    auto bar_empty = [&](int s) { return bar0 + 8u * (S + s); };      // slot may be refilled
+    auto bar_raw = [&](int s) { return bar0 + 8u * (2 * S + s); };    // raw scales + sign bytes landed
+    const uint32_t bar_u_full = bar0 + 8u * (3 * S);
+    const uint32_t bar_z_full = bar0 + 8u * (3 * S + 1);
+    const uint32_t bar_rx_full = bar0 + 8u * (3 * S + 2);
+    auto bar_v_full = [&](int b) { return bar0 + 8u * (3 * S + 3 + b); };
+    auto bar_v_empty = [&](int b) { return bar0 + 8u * (3 * S + 5 + b); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + plan.off_misc);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + plan.off_misc + 4);
+    const WaitCtx wctx{abort_flag, B.status};
+
+    const int kt8 = kp / 8;                 // 16-byte chunks per row of a stage-2 operand
+    const int r8 = r / 8;
+    const uint32_t sign_bytes = 8u * r;     // sign bytes next to one 64-column chunk, either stage
+
+    // ---- one-time setup ---------------------------------------------------------------------
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(bar_full(s), 1 + kGenThreads);   // producer's expect_tx arrive + generator threads
+            mbar_init(bar_empty(s), 1);
+            mbar_init(bar_raw(s), 1);
+        }
+        mbar_init(bar_u_full, 1);
+        mbar_init(bar_z_full, (uint32_t)(tile_rows * r8));   // one arrive per (row, 8-wide piece), all owners
+        mbar_init(bar_rx_full, (uint32_t)(2 * tile_rows));   // one arrive per (token row, column half)
+        mbar_init(bar_v_full(0), 1);
+        mbar_init(bar_v_full(1), 1);
+        mbar_init(bar_v_empty(0), kEpiThreads);
+        mbar_init(bar_v_empty(1), kEpiThreads);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // sign-flip table: byte of 8 sign bits -> four 32-bit XOR masks over bf16 pairs (bit 0 => flip)
+    if (tid < 256) {
+        uint32_t m[4];
+#pragma unroll
+        for (int p = 0; p < 4; ++p)
+            m[p] = (((tid >> (2 * p)) & 1) ? 0u : 0x8000u) | (((tid >> (2 * p + 1)) & 1) ? 0u : 0x80000000u);
+        reinterpret_cast<uint4 *>(sm + plan.off_lut)[tid] = make_uint4(m[0], m[1], m[2], m[3]);
+    }
+    // stage-2 A operands start as zeros (K padding beyond r and rows beyond tile_rows stay zero)
+    for (int i = tid; i < 2 * plan.z_bytes / 16; i += kThreads)
+        reinterpret_cast<uint4 *>(sm + plan.off_zhi)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    cluster_sync_all();
+    const uint32_t tmem_base = *tmem_slot;
+    if (tid == 0) TC_TRACE(4, 0, 1);
+
+    const uint4 *lut = reinterpret_cast<const uint4 *>(sm + plan.off_lut);
+    const int rows_per = tile_rows / C;      // token rows of a tile owned by each CTA of the cluster
+
+    // Every role walks the same sequence of (tile, chunk) and derives slot and phase from `it`.
+    uint32_t it = 0;        // chunk counter (ring position)
+    uint32_t vit = 0;       // stage-2 chunk counter (TMEM accumulator double buffer)
+    uint32_t tile_n = 0;    // tiles done by this cluster (phase of the per-tile barriers)
+
+    for (int item = cid; item < B.total_tiles; item += n_clusters, ++tile_n) {
+        int pi = 0;
+        while (pi + 1 < B.n_proj && item >= B.p[pi + 1].tile_begin) ++pi;
+        const TcProj &P = B.p[pi];
+        const int t0 = (item - P.tile_begin) * tile_rows;
+        int kb, ke, nb, ne;
+        split_range(P.nk, C, (int)crank, kb, ke);
+        split_range(P.nn, C, (int)crank, nb, ne);
+        const uint32_t tphase = tile_n & 1u;
+
+        if (warp == 0) {
+            // ================= TMA producer =================
+            // Per chunk: the raw scale values (256 B) and sign bytes (8r B) that belong to the
+            // chunk's 64 columns, then the 64-column box of x (stage 1) or y (stage 2).  A ragged
+            // last chunk (fewer than 64 valid columns) leaves the raw fetch to the generators.
+            if (lane == 0) {
+                for (int c = kb; c < ke; ++c, ++it) {
+                    const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                    mbar_wait<false>(wctx, bar_empty(s), ph ^ 1u, kDevTmaWaitTimeout);
+                    TC_TRACE(0, it, 0);
+                    const uint32_t slot = sm_base + s * plan.slot_stride;
+                    const uint32_t rawdst = slot + plan.slot_data + plan.aux_op_bytes;
+                    if ((c + 1) * kChunk <= P.d_in) {
+                        mbar_arrive_expect_tx(bar_raw(s), 256u + sign_bytes);
+                        bulk_load(rawdst, P.s_in + (size_t)c * kChunk, 256u, bar_raw(s));
+                        bulk_load(rawdst + 256u, reinterpret_cast<const uint8_t *>(P.packed_A) + (size_t)c * sign_bytes,
+                                  sign_bytes, bar_raw(s));
+                    } else {
+                        mbar_arrive(bar_raw(s));
+                    }
+                    mbar_arrive_expect_tx(bar_full(s), box_bytes);
+                    tma_load_2d(slot, &P.x_map, c * kChunk, t0, bar_full(s));
+                }
+                for (int c = nb; c < ne; ++c, ++it) {
+                    const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                    mbar_wait<false>(wctx, bar_empty(s), ph ^ 1u, kDevTmaWaitTimeout);
+                    TC_TRACE(0, it, 0);
+                    const uint32_t slot = sm_base + s * plan.slot_stride;
+                    const uint32_t rawdst = slot + plan.slot_data + plan.aux_op_bytes;
+                    if ((c + 1) * kChunk <= P.d_out) {
+                        mbar_arrive_expect_tx(bar_raw(s), 256u + sign_bytes);
+                        bulk_load(rawdst, P.s_out + (size_t)c * kChunk, 256u, bar_raw(s));
+                        bulk_load(rawdst + 256u, reinterpret_cast<const uint8_t *>(P.packed_B) + (size_t)c * sign_bytes,
+                                  sign_bytes, bar_raw(s));
+                    } else {
+                        mbar_arrive(bar_raw(s));
+                    }
+                    mbar_arrive_expect_tx(bar_full(s), box_bytes);
+                    tma_load_2d(slot, &P.y_map, c * kChunk, t0, bar_full(s));
+                }
+            }
+        } else if (warp == 1) {
+            // ================= MMA issuer =================
+            if (lane == 0) {
+                const uint32_t idesc1 = instr_desc(kTileM, 2 * r);
+                const uint32_t idesc2 = instr_desc(kTileM, kChunk);
+                for (int c = kb; c < ke; ++c, ++it) {
+                    const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                    mbar_wait<false>(wctx, bar_full(s), ph, kDevMmaWaitTimeout);
+                    TC_TRACE(1, it, 0);
+                    tc_fence_after();
+                    const uint32_t a0 = sm_base + s * plan.slot_stride;       // x tile, 128B swizzle
+                    const uint32_t b0 = a0 + plan.slot_data;                  // W1, no swizzle
+#pragma unroll
+                    for (int ks = 0; ks < kChunk / 16; ++ks) {
+                        const uint64_t ad = smem_desc(a0 + ks * 32, 16, 1024, 2);
+                        const uint64_t bd = smem_desc(b0 + ks * 256, 128, 1024, 0);
+                        mma_bf16(tmem_base + kTmemU, ad, bd, idesc1, (c > kb || ks > 0) ? 1u : 0u);
+                    }
+                    mma_commit(bar_empty(s));
+                }
+                mma_commit(bar_u_full);
+                mbar_wait<true>(wctx, bar_z_full, tphase, kDevMmaWaitTimeout);
+                TC_TRACE(1, it, 2);
+                fence_proxy_async();
+                tc_fence_after();
+                const uint32_t zhi = sm_base + plan.off_zhi, zlo = sm_base + plan.off_zlo;
+                const uint32_t z_sbo = kt8 * 128;
+                for (int c = nb; c < ne; ++c, ++it, ++vit) {
+                    const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                    const int vb = vit & 1u; const uint32_t vph = (vit >> 1) & 1u;
+                    mbar_wait<false>(wctx, bar_full(s), ph, kDevMmaWaitTimeout);
+                    TC_TRACE(1, it, 0);
+                    mbar_wait<false>(wctx, bar_v_empty(vb), vph ^ 1u, kDevMmaWaitTimeout);
+                    TC_TRACE(1, it, 1);
+                    tc_fence_after();
+                    const uint32_t b0 = sm_base + s * plan.slot_stride + plan.slot_data;   // W2, no swizzle
+                    const uint32_t d = tmem_base + kTmemV + vb * kChunk;
+                    uint32_t acc = 0;
+                    for (int half = 0; half < 2; ++half) {
+                        const uint32_t za = half ? zlo : zhi;
+                        for (int ks = 0; ks < kp / 16; ++ks) {
+                            const uint64_t ad = smem_desc(za + ks * 256, 128, z_sbo, 0);
+                            const uint64_t bd = smem_desc(b0 + ks * 256, 128, z_sbo, 0);
+                            mma_bf16(d, ad, bd, idesc2, acc);
+                            acc = 1;
+                        }
+                    }
+                    mma_commit(bar_v_full(vb));
+                }
+            }
+        } else if (warp < 2 + kGenThreads / 32) {
+            // ================= operand generators =================
+            const int g = tid - 64;                // 0..kGenThreads-1
+            const int rsub = g & 7;                // row within an 8-row core matrix
+            const int cc = (g >> 3) & 7;           // 16-byte chunk (8 columns) within the 64-column box
+            const int kg0 = g >> 6;                // first 8-row group handled by this thread (stage 1)
+            for (int c = kb; c < ke; ++c, ++it) {
+                const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                mbar_wait<false>(wctx, bar_raw(s), ph, kDevTmaWaitTimeout);
+                if (g == 0) TC_TRACE(2, it, 0);
+                uint8_t *aux = sm + s * plan.slot_stride + plan.slot_data;
+                float *raw_scale = reinterpret_cast<float *>(aux + plan.aux_op_bytes);
+                uint8_t *raw_sign = aux + plan.aux_op_bytes + 256;
+                if ((c + 1) * kChunk > P.d_in) {
+                    // ragged last chunk: guarded loads (the sign block itself is always complete)
+                    if (g < kChunk) raw_scale[g] = (c * kChunk + g < P.d_in) ? __ldg(P.s_in + c * kChunk + g) : 0.0f;
+                    for (int w = g; w < 2 * r; w += kGenThreads)
+                        reinterpret_cast<uint32_t *>(raw_sign)[w] = __ldg(P.packed_A + (size_t)c * 2 * r + w);
+                    asm volatile("bar.sync 2, %0;" ::"n"(kGenThreads) : "memory");
+                }
+                // s_in of this thread's 8 columns, split into bf16 hi + bf16 lo
+                const float4 sa = *reinterpret_cast<const float4 *>(raw_scale + cc * 8);
+                const float4 sb = *reinterpret_cast<const float4 *>(raw_scale + cc * 8 + 4);
+                const float sv[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    const float ah = bf16_round(sv[2 * p]), bh = bf16_round(sv[2 * p + 1]);
+                    hi[p] = pack2_bf16(ah, bh);
+                    lo[p] = pack2_bf16(sv[2 * p] - ah, sv[2 * p + 1] - bh);
+                }
+                uint8_t *w1 = aux;
+                for (int k = kg0 * 8 + rsub; k < r; k += kGenThreads / 8) {
+                    const uint4 m = lut[raw_sign[k * 8 + cc]];
+                    const int row_hi = k, row_lo = r + k;
+                    *reinterpret_cast<uint4 *>(w1 + (row_hi >> 3) * 1024 + cc * 128 + (row_hi & 7) * 16) =
+                        make_uint4(hi[0] ^ m.x, hi[1] ^ m.y, hi[2] ^ m.z, hi[3] ^ m.w);
+                    *reinterpret_cast<uint4 *>(w1 + (row_lo >> 3) * 1024 + cc * 128 + (row_lo & 7) * 16) =
+                        make_uint4(lo[0] ^ m.x, lo[1] ^ m.y, lo[2] ^ m.z, lo[3] ^ m.w);
+                }
+                fence_proxy_async();
+                mbar_arrive(bar_full(s));
+                if (g == 0) TC_TRACE(2, it, 1);
+            }
+            for (int c = nb; c < ne; ++c, ++it) {
+                const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                mbar_wait<false>(wctx, bar_raw(s), ph, kDevTmaWaitTimeout);
+                if (g == 0) TC_TRACE(2, it, 0);
+                uint8_t *aux = sm + s * plan.slot_stride + plan.slot_data;
+                float *raw_scale = reinterpret_cast<float *>(aux + plan.aux_op_bytes);
+                uint8_t *raw_sign = aux + plan.aux_op_bytes + 256;
+                if ((c + 1) * kChunk > P.d_out) {
+                    const int64_t n_words = ((int64_t)P.d_out * r + 31) / 32;
+                    if (g < kChunk) raw_scale[g] = (c * kChunk + g < P.d_out) ? __ldg(P.s_out + c * kChunk + g) : 0.0f;
+                    for (int w = g; w < 2 * r; w += kGenThreads) {
+                        const int64_t gw = (int64_t)c * 2 * r + w;
+                        reinterpret_cast<uint32_t *>(raw_sign)[w] = (gw < n_words) ? __ldg(P.packed_B + gw) : 0u;
+                    }
+                    asm volatile("bar.sync 2, %0;" ::"n"(kGenThreads) : "memory");
+                }
+                uint8_t *w2 = aux;
+                // 64 rows x kt8 chunks; task = (row group, chunk, row in group)
+                for (int task = g; task < kChunk * kt8; task += kGenThreads) {
+                    const int rs = task & 7;
+                    const int ch = (task >> 3) % kt8;
+                    const int row = ((task >> 3) / kt8) * 8 + rs;
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (c * kChunk + row < P.d_out && ch < r8) {
+                        const uint4 m = lut[raw_sign[row * r8 + ch]];
+                        v = make_uint4(0x3f803f80u ^ m.x, 0x3f803f80u ^ m.y, 0x3f803f80u ^ m.z, 0x3f803f80u ^ m.w);
+                    }
+                    *reinterpret_cast<uint4 *>(w2 + (row >> 3) * (kt8 * 128) + ch * 128 + rs * 16) = v;
+                }
+                fence_proxy_async();
+                mbar_arrive(bar_full(s));
+                if (g == 0) TC_TRACE(2, it, 1);
+            }
+        } else {
+            // ================= epilogue (8 warps: 4 TMEM lane quadrants x 2 column halves) ==========
+            const int e = tid - (64 + kGenThreads);       // 0..kEpiThreads-1
+            const int quad = warp & 3;                    // TMEM lanes 32*quad .. 32*quad+31
+            const int chalf = e >> 7;                     // which 32 of a chunk's 64 columns
+            const int row = quad * 32 + lane;             // token row of the tile
+            const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16);
+            const bool warp_has_rows = quad * 32 < tile_rows;    // warp-uniform
+            const bool row_valid = row < tile_rows;
+            it += (ke - kb);
+
+            // ---- after stage 1: partial u -> owner CTA of this row (even pieces: half 0, odd: half 1)
+            mbar_wait<false>(wctx, bar_u_full, tphase, kDevEpilogueWaitTimeout);
+            if (e == 0) TC_TRACE(3, it, 5);
+            __syncwarp();
+            tc_fence_after();
+            if (warp_has_rows) {
+                const uint32_t owner = row_valid ? (uint32_t)(row / rows_per) : 0u;
+                const int row_local = row - (int)owner * rows_per;
+                const uint32_t rx_remote = mapa(sm_base + plan.off_rx, owner) +
+                                           (uint32_t)(((int)crank * rows_per + row_local) * r) * 4u;
+                for (int p = chalf; p < r8; p += 2) {
+                    float h[8], l[8];
+                    tmem_ld8(tlane + kTmemU + p * 8, h);          // warp-collective
+                    tmem_ld8(tlane + kTmemU + r + p * 8, l);
+                    tmem_wait_ld();
+                    if (row_valid) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) w[i] = __float_as_uint(h[i] + l[i]);
+                        st_cluster_v4(rx_remote + p * 32, w[0], w[1], w[2], w[3]);
+                        st_cluster_v4(rx_remote + p * 32 + 16, w[4], w[5], w[6], w[7]);
+                    }
+                }
+                tc_fence_before();
+                if (row_valid) mbar_arrive_remote(mapa(bar_rx_full, owner));
+            }
+            // ---- owner: reduce over source CTAs in a fixed order, scale by s_r, split, broadcast z
+            mbar_wait<true>(wctx, bar_rx_full, tphase, kDevClusterWaitTimeout);
+            if (e == 0) TC_TRACE(3, it, 6);
+            {
+                const float *rx = reinterpret_cast<const float *>(sm + plan.off_rx);
+                for (int task = e; task < rows_per * r8; task += kEpiThreads) {
+                    const int row_local = task / r8, p = task - row_local * r8;
+                    float u[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) u[i] = 0.0f;
+                    for (int src = 0; src < C; ++src) {
+                        const float4 a = *reinterpret_cast<const float4 *>(rx + (src * rows_per + row_local) * r + p * 8);
+                        const float4 b = *reinterpret_cast<const float4 *>(rx + (src * rows_per + row_local) * r + p * 8 + 4);
+                        u[0] += a.x; u[1] += a.y; u[2] += a.z; u[3] += a.w;
+                        u[4] += b.x; u[5] += b.y; u[6] += b.z; u[7] += b.w;
+                    }
+                    uint32_t zh[4], zl[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float z0 = u[2 * q] * __ldg(P.s_r + p * 8 + 2 * q);
+                        const float z1 = u[2 * q + 1] * __ldg(P.s_r + p * 8 + 2 * q + 1);
+                        const float h0 = bf16_round(z0), h1 = bf16_round(z1);
+                        zh[q] = pack2_bf16(h0, h1);
+                        zl[q] = pack2_bf16(z0 - h0, z1 - h1);
+                    }
+                    const int grow = (int)crank * rows_per + row_local;          // row within the tile
+                    const uint32_t off = (uint32_t)((grow >> 3) * (kt8 * 128) + p * 128 + (grow & 7) * 16);
+                    for (int dst = 0; dst < C; ++dst) {
+                        st_cluster_v4(mapa(sm_base + plan.off_zhi, dst) + off, zh[0], zh[1], zh[2], zh[3]);
+                        st_cluster_v4(mapa(sm_base + plan.off_zlo, dst) + off, zl[0], zl[1], zl[2], zl[3]);
+                    }
+                    asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");
+                    for (int dst = 0; dst < C; ++dst) mbar_arrive_remote(mapa(bar_z_full, dst));
+                }
+            }
+            // ---- after stage 2: y tile (already in the slot) += s_out * V, in place, then TMA store
+            int prev_slot = -1;
+            for (int c = nb; c < ne; ++c, ++it, ++vit) {
+                const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                const int vb = vit & 1u; const uint32_t vph = (vit >> 1) & 1u;
+                mbar_wait<false>(wctx, bar_v_full(vb), vph, kDevEpilogueWaitTimeout);
+                if (e == 0) TC_TRACE(3, it, 0);
+                mbar_wait<false>(wctx, bar_full(s), ph, kDevEpilogueWaitTimeout);
+                __syncwarp();
+                tc_fence_after();
+                uint8_t *ytile = sm + s * plan.slot_stride;
+                const float *so = reinterpret_cast<const float *>(ytile + plan.slot_data + plan.aux_op_bytes);
+                if (warp_has_rows) {
+                    uint32_t v[32];
+                    tmem_ld32(tlane + kTmemV + vb * kChunk + chalf * 32, v);   // warp-collective
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    mbar_arrive(bar_v_empty(vb));
+                    if (e == 0) TC_TRACE(3, it, 1);
+                    if (row_valid) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int ch = chalf * 4 + q;                  // 16-byte chunk of the row
+                            uint4 *py = reinterpret_cast<uint4 *>(ytile + row * 128 + ((ch ^ (row & 7)) * 16));
+                            const uint4 yv = *py;
+                            const float4 s0 = *reinterpret_cast<const float4 *>(so + ch * 8);
+                            const float4 s1 = *reinterpret_cast<const float4 *>(so + ch * 8 + 4);
+                            const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
+                            const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                            uint32_t ow[4];
+#pragma unroll
+                            for (int k2 = 0; k2 < 4; ++k2) {
+                                const float y0 = __uint_as_float(yw[k2] << 16);
+                                const float y1 = __uint_as_float(yw[k2] & 0xffff0000u);
+                                const float o0 = fmaf(sc[2 * k2], __uint_as_float(v[q * 8 + 2 * k2]), y0);
+                                const float o1 = fmaf(sc[2 * k2 + 1], __uint_as_float(v[q * 8 + 2 * k2 + 1]), y1);
+                                ow[k2] = pack2_bf16(o0, o1);
+                            }
+                            *py = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                        }
+                    }
+                } else {
+                    mbar_arrive(bar_v_empty(vb));
+                }
+                if (e == 0) TC_TRACE(3, it, 2);
+                fence_proxy_async();
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                if (e == 0) {
+                    TC_TRACE(3, it, 3);
+                    tma_store_2d(&P.y_map, sm_base + s * plan.slot_stride, c * kChunk, t0);
+                    bulk_commit();
+                    if (prev_slot >= 0) {
+                        bulk_wait_read_1();
+                        mbar_arrive(bar_empty(prev_slot));
+                    }
+                    prev_slot = s;
+                    TC_TRACE(3, it, 4);
+                }
+            }
+            if (e == 0 && prev_slot >= 0) {
+                bulk_wait_read_0();
+                mbar_arrive(bar_empty(prev_slot));
+            }
+        }
+    }
+
+    // ---- teardown -------------------------------------------------------------------------------
+    if (tid == 64 + kGenThreads) bulk_wait_all();       // the thread that issued the stores
+    if (*abort_flag) {
+        // give copies that may still be in flight time to land before the CTA goes away
+        const long long start = clock64();
+        while (clock64() - start < 2000000LL) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) TC_TRACE(4, 0, 2);
+    cluster_sync_all();
+    if (tid == 0) TC_TRACE(4, 0, 3);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// T x d bf16 matrix with row pitch ld (elements); boxes of 128 rows x 64 columns, 128B swizzle.
+bool make_map(CUtensorMap *map, const void *base, int64_t T, int64_t d, int64_t ld, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)T};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kChunk, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS;
+}
+
+int env_int(const char *name, int dflt)
+{
+    const char *v = std::getenv(name);
+    return (v && *v) ? std::atoi(v) : dflt;
+}
+
+struct LaunchShape { int cluster, tile_rows, slots, smem, max_clusters; };
+
+constexpr int kMaxSlots = 32;
+
+// Co-resident clusters for a cluster size and shared-memory footprint (cached: the query is slow).
+int max_active_clusters(int cluster, int smem)
+{
+    static std::mutex mu;
+    static int cache_cluster[64], cache_smem[64], cache_val[64], n_cached = 0;
+    static bool attr_set = false;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(tc_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget) != cudaSuccess) {
+            cudaGetLastError();
+            return 0;
+        }
+        attr_set = true;
+    }
+    for (int i = 0; i < n_cached; ++i)
+        if (cache_cluster[i] == cluster && cache_smem[i] == smem) return cache_val[i];
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(cluster, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = cluster; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, tc_forward_kernel, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        n = 0;
+    }
+    if (n_cached < 64) {
+        cache_cluster[n_cached] = cluster; cache_smem[n_cached] = smem; cache_val[n_cached] = n;
+        ++n_cached;
+    }
+    return n;
+}
+
+// Deepest ring that fits next to the fixed buffers, and how many clusters can be co-resident.
+bool plan_launch(int r, int kp, int cluster, int tile_rows, LaunchShape *out)
+{
+    int slots = 0;
+    for (int s = kMaxSlots; s >= 2; --s) {
+        if (make_plan(r, kp, s, tile_rows).total + 1024 <= kSmemBudget) { slots = s; break; }
+    }
+    const int forced = env_int("LORDBA_TC_SLOTS", 0);
+    if (forced >= 2 && forced <= slots) slots = forced;
+    if (slots < 2) return false;
+    const int smem = make_plan(r, kp, slots, tile_rows).total + 1024;
+    const int n = max_active_clusters(cluster, smem);
+    if (n < 1) return false;
+    out->cluster = cluster; out->tile_rows = tile_rows; out->slots = slots; out->smem = smem;
+    out->max_clusters = n;
+    return true;
+}
+
+// Choose cluster size and tile height for `n_proj` projections of T tokens each.  Few tokens
+// are spread over many SMs by splitting the feature axes over a cluster and by shortening the
+// tile; many tokens use tall tiles and small clusters.
+bool choose_shape(int r, int kp, int n_proj, int64_t T, int min_chunks, LaunchShape *best)
+{
+    const int forced_c = env_int("LORDBA_TC_CLUSTER", 0);
+    const int forced_rows = env_int("LORDBA_TC_ROWS", 0);
+    double best_cost = 1e300;
+    bool found = false;
+    for (int c = 8; c >= 1; c /= 2) {
+        if (c > min_chunks) continue;
+        if (forced_c >= 1 && forced_c <= 8 && c != forced_c && c * 2 <= min_chunks) continue;
+        LaunchShape probe;
+        if (!plan_launch(r, kp, c, kTileM, &probe)) continue;
+        const int cap = probe.max_clusters;
+        // waves of `cap` clusters needed with full-height tiles, then the tile height that fills them
+        const int64_t full_tiles = (int64_t)n_proj * ((T + kTileM - 1) / kTileM);
+        const int64_t waves = (full_tiles + cap - 1) / cap;
+        int64_t rows = ((int64_t)n_proj * T + cap * waves - 1) / (cap * waves);   // per-tile share
+        rows = (rows + c - 1) / c * c;
+        if (rows > kTileM) rows = kTileM;
+        if (rows < c) rows = c;
+        if (forced_rows >= c && forced_rows <= kTileM && forced_rows % c == 0) rows = forced_rows;
+        LaunchShape shape;
+        if (!plan_launch(r, kp, c, (int)rows, &shape)) continue;
+        const int64_t tiles = (int64_t)n_proj * ((T + rows - 1) / rows);
+        const int64_t w = (tiles + shape.max_clusters - 1) / shape.max_clusters;
+        // cost model: time ~ waves * rows of work per cluster / CTAs sharing it, plus a fixed
+        // per-tile cost (operand generation, MMA on padded rows, cluster exchange)
+        const double per_tile = (double)rows / c + 24.0 / c + 6.0;
+        const double cost = (double)w * per_tile;
+        if (cost < best_cost) { best_cost = cost; *best = shape; found = true; }
+    }
+    return found;
+}
+
+}  // namespace
+
+bool tc_supported(const lordba_proj &p, int64_t T, int dtype)
+{
+    if (dtype != LORDBA_BF16 || T < 1) return false;
+    if (p.r % 8 != 0 || p.r < 8 || p.r > kMaxRank) return false;
+    if (p.d_in < kChunk || p.d_out < kChunk) return false;
+    if (p.d_in > (1 << 30) || p.d_out > (1 << 30) || T > (1 << 30)) return false;
+    if (reinterpret_cast<uintptr_t>(p.x) % 16 || reinterpret_cast<uintptr_t>(p.y) % 16) return false;
+    if (p.ldx % 8 || p.ldy % 8) return false;
+    // the raw scales and sign bytes of a chunk travel as bulk copies: 16-byte aligned sources
+    if (reinterpret_cast<uintptr_t>(p.s_in) % 16 || reinterpret_cast<uintptr_t>(p.s_out) % 16 ||
+        reinterpret_cast<uintptr_t>(p.packed_A) % 16 || reinterpret_cast<uintptr_t>(p.packed_B) % 16)
+        return false;
+    return encode_fn() != nullptr;
+}
+
+int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream)
+{
+    if (n == 0 || T == 0) return LORDBA_OK;
+    if (dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    int *status = device_status_word();
+    if (!status) return LORDBA_ECUDA;
+
+    // one launch per rank value and per kMaxTcBatch projections
+    for (int r = 8; r <= kMaxRank; r += 8) {
+        int i = 0;
+        while (i < n) {
+            // collect the next projections of this rank
+            const lordba_proj *sel[kMaxTcBatch];
+            int m = 0, min_chunks = 1 << 30;
+            for (; i < n && m < kMaxTcBatch; ++i) {
+                if (projs[i].r != r) continue;
+                sel[m++] = &projs[i];
+                const int nk = (int)((projs[i].d_in + kChunk - 1) / kChunk);
+                const int nn = (int)((projs[i].d_out + kChunk - 1) / kChunk);
+                if (nk < min_chunks) min_chunks = nk;
+                if (nn < min_chunks) min_chunks = nn;
+            }
+            if (m == 0) continue;
+            const int kp = (r + 15) / 16 * 16;
+            LaunchShape shape;
+            if (!choose_shape(r, kp, m, T, min_chunks, &shape)) return LORDBA_ECUDA;
+            const int tiles_per_proj = (int)((T + shape.tile_rows - 1) / shape.tile_rows);
+
+            TcBatch b;
+            std::memset(&b, 0, sizeof(b));
+            for (int k = 0; k < m; ++k) {
+                const lordba_proj &q = *sel[k];
+                TcProj &t = b.p[k];
+                if (!make_map(&t.x_map, q.x, T, q.d_in, q.ldx, shape.tile_rows) ||
+                    !make_map(&t.y_map, q.y, T, q.d_out, q.ldy, shape.tile_rows))
+                    return LORDBA_EUNSUPPORTED;
+                t.packed_A = q.packed_A; t.packed_B = q.packed_B;
+                t.s_in = q.s_in; t.s_r = q.s_r; t.s_out = q.s_out;
+                t.d_in = (int)q.d_in; t.d_out = (int)q.d_out;
+                t.nk = (int)((q.d_in + kChunk - 1) / kChunk);
+                t.nn = (int)((q.d_out + kChunk - 1) / kChunk);
+                t.words_a = (int)((q.d_in + 31) / 32);
+                t.tile_begin = k * tiles_per_proj;
+            }
+            b.n_proj = m;
+            b.total_tiles = m * tiles_per_proj;
+            b.r = r;
+            b.kp = kp;
+            b.status = status;
+#ifdef LORDBA_TC_TRACE
+            {
+                const char *tp = std::getenv("LORDBA_TC_TRACE_PTR");
+                b.trace = tp ? reinterpret_cast<long long *>(std::strtoull(tp, nullptr, 0)) : nullptr;
+            }
+#endif
+            b.cluster = shape.cluster;
+            b.slots = shape.slots;
+            b.tile_rows = shape.tile_rows;
+            int n_clusters = b.total_tiles < shape.max_clusters ? b.total_tiles : shape.max_clusters;
+            if (env_int("LORDBA_TC_DEBUG", 0))
+                std::fprintf(stderr, "[lordba tc] r=%d proj=%d tiles=%d rows=%d cluster=%d slots=%d smem=%d "
+                             "max_clusters=%d grid=%d\n", r, m, b.total_tiles, shape.tile_rows, shape.cluster,
+                             shape.slots, shape.smem, shape.max_clusters, n_clusters * shape.cluster);
+
+            cudaLaunchConfig_t cfg;
+            std::memset(&cfg, 0, sizeof(cfg));
+            cfg.gridDim = dim3(n_clusters * shape.cluster, 1, 1);
+            cfg.blockDim = dim3(kThreads, 1, 1);
+            cfg.dynamicSmemBytes = shape.smem;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = shape.cluster; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr; cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, tc_forward_kernel, b) != cudaSuccess) {
+                cudaGetLastError();
+                return LORDBA_ECUDA;
+            }
+            count_launch();
+        }
+    }
+    return LORDBA_OK;
+}
+
 }  // namespace lordba

@@ -1,9 +1,10 @@
 // Bit-packing of the +-1 carriers ("bit-packed {B1,B2}", Section 3.3).
 //
-// Both roles are a flat ballot: a warp reads 32 consecutive int8 signs and one
-// lane writes the word.  Role 1 (B carrier) is the flat row-major stream
-// itself; role 0 (A carrier) is the same per row, each row padded to whole
-// words.  sign(0) = +1: an entry packs as bit 0 only when it is negative.
+// A warp reads 32 consecutive int8 signs of one row and one lane writes the
+// ballot.  Role 1 (B carrier, d_out x r) is the flat row-major bit stream.
+// Role 0 (A carrier, r x d_in) is block-major: for every block of 64 columns,
+// r consecutive 64-bit groups (two words each, low word first), one per row.
+// sign(0) = +1: an entry packs as bit 0 only when it is negative.
 #include "lordba_internal.h"
 
 namespace lordba {
@@ -11,19 +12,31 @@ namespace {
 
 constexpr int kPackThreads = 256;
 
-// rows x cols int8 -> rows x ceil(cols/32) words; role 1 calls it with rows = 1
-// and cols = d_out * r.
+// Word w of the packed array -> (row, first column) of the 32 signs it holds.
+__device__ __forceinline__ void word_to_source(int64_t w, int64_t rows, int role, int64_t &row, int64_t &col0)
+{
+    if (role == 0) {
+        const int64_t block = w / (rows * 2);
+        const int64_t rem = w - block * rows * 2;
+        row = rem >> 1;
+        col0 = block * 64 + (rem & 1) * 32;
+    } else {            // flat stream: the caller passes rows = 1, cols = d_out * r
+        row = 0;
+        col0 = w * 32;
+    }
+}
+
 __global__ void __launch_bounds__(kPackThreads)
-pack_rows_kernel(const int8_t *__restrict__ signs, int64_t rows, int64_t cols, int64_t words_per_row,
-                 uint32_t *__restrict__ packed)
+pack_kernel(const int8_t *__restrict__ signs, int64_t rows, int64_t cols, int role, int64_t total_words,
+            uint32_t *__restrict__ packed)
 {
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (kPackThreads / 32) + (threadIdx.x >> 5);
     const int64_t n_warps = (int64_t)gridDim.x * (kPackThreads / 32);
-    const int64_t total = rows * words_per_row;
-    for (int64_t w = warp; w < total; w += n_warps) {
-        const int64_t row = w / words_per_row;
-        const int64_t col = (w - row * words_per_row) * 32 + lane;
+    for (int64_t w = warp; w < total_words; w += n_warps) {
+        int64_t row, col0;
+        word_to_source(w, rows, role, row, col0);
+        const int64_t col = col0 + lane;
         bool plus = false;
         if (col < cols) plus = signs[row * cols + col] >= 0;
         const uint32_t word = __ballot_sync(0xffffffffu, plus);
@@ -32,16 +45,17 @@ pack_rows_kernel(const int8_t *__restrict__ signs, int64_t rows, int64_t cols, i
 }
 
 __global__ void __launch_bounds__(kPackThreads)
-unpack_rows_kernel(const uint32_t *__restrict__ packed, int64_t rows, int64_t cols,
-                   int64_t words_per_row, int8_t *__restrict__ signs)
+unpack_kernel(const uint32_t *__restrict__ packed, int64_t rows, int64_t cols, int role,
+              int8_t *__restrict__ signs)
 {
     const int64_t total = rows * cols;
     const int64_t stride = (int64_t)gridDim.x * kPackThreads;
     for (int64_t e = (int64_t)blockIdx.x * kPackThreads + threadIdx.x; e < total; e += stride) {
         const int64_t row = e / cols;
         const int64_t col = e - row * cols;
-        const uint32_t word = packed[row * words_per_row + (col >> 5)];
-        signs[e] = ((word >> (col & 31)) & 1u) ? (int8_t)1 : (int8_t)-1;
+        const int64_t w = (role == 0) ? ((col >> 6) * rows + row) * 2 + ((col & 63) >> 5) : (e >> 5);
+        const int bit = (role == 0) ? (int)(col & 31) : (int)(e & 31);
+        signs[e] = ((packed[w] >> bit) & 1u) ? (int8_t)1 : (int8_t)-1;
     }
 }
 
@@ -60,10 +74,10 @@ int launch_pack(const int8_t *signs, int64_t rows, int64_t cols, int role, uint3
 {
     int64_t prow = rows, pcols = cols;
     if (role == 1) { prow = 1; pcols = rows * cols; }
-    const int64_t wpr = (pcols + 31) / 32;
-    if (prow * wpr == 0) return LORDBA_OK;
-    pack_rows_kernel<<<grid_for(prow * wpr, kPackThreads / 32), kPackThreads, 0, stream>>>(
-        signs, prow, pcols, wpr, packed);
+    const int64_t words = (role == 0) ? ((cols + 63) / 64) * rows * 2 : (pcols + 31) / 32;
+    if (words == 0) return LORDBA_OK;
+    pack_kernel<<<grid_for(words, kPackThreads / 32), kPackThreads, 0, stream>>>(signs, prow, pcols, role,
+                                                                                words, packed);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LORDBA_OK : LORDBA_ECUDA;
 }
@@ -73,10 +87,9 @@ int launch_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int role, 
 {
     int64_t prow = rows, pcols = cols;
     if (role == 1) { prow = 1; pcols = rows * cols; }
-    const int64_t wpr = (pcols + 31) / 32;
     if (prow * pcols == 0) return LORDBA_OK;
-    unpack_rows_kernel<<<grid_for(prow * pcols, kPackThreads), kPackThreads, 0, stream>>>(
-        packed, prow, pcols, wpr, signs);
+    unpack_kernel<<<grid_for(prow * pcols, kPackThreads), kPackThreads, 0, stream>>>(packed, prow, pcols,
+                                                                                     role, signs);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LORDBA_OK : LORDBA_ECUDA;
 }

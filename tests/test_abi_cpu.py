@@ -35,7 +35,7 @@ def test_host_only_helpers(lib):
     from paper_2605_24058_b200 import lordba
     assert lordba.packed_words(16, 4096, 0) == 16 * 128
     assert lordba.packed_words(4096, 16, 1) == 2048
-    assert lordba.packed_words(3, 33, 0) == 6
+    assert lordba.packed_words(3, 33, 0) == 6 and lordba.packed_words(3, 65, 0) == 12
     assert lordba.packed_words(33, 3, 1) == 4
     assert lordba.packed_words(-1, 3, 0) == -1 and lordba.packed_words(1, 3, 2) == -1
     assert lordba.adapter_bits(3, 5, 2, 1) == 2 * 8 + 16 * 10          # Eq. 5 by hand
@@ -87,6 +87,8 @@ def test_bad_arguments_return_codes_without_launching(lib):
     assert lib.lordba_adapter_forward_ex(None, 4, lordba.BF16, None) == EINVAL
     # T = 0 is a no-op that succeeds
     assert call(_proj(lordba), T=0) == 0
+    assert call(_proj(lordba, x=0, y=0), T=0) == 0
+    assert call(_proj(lordba, r=0), T=0) == EUNSUP
     # batched: overlapping outputs, negative count
     two = (lordba.Proj * 2)(_proj(lordba), _proj(lordba, x=0x8000))
     assert lib.lordba_adapter_forward_batched(two, 2, 4, lordba.BF16, None) == EINVAL

@@ -17,13 +17,21 @@ def test_hand_written_words_role_a(oracle):
         s[0, c] = 1
     got = oracle.pack_signs(s, 0)
     assert got.tolist() == [0x80000003, 0x80000001]
-    # two rows of 40 columns: each row starts on a fresh word, pad bits stay 0
+    # two rows of 40 columns: one 64-column block, one 64-bit group per row, pad bits stay 0
     s = -np.ones((2, 40), np.int8)
     s[0, 39] = 1
     s[1, 0] = 1
     s[1, 33] = 1
     got = oracle.pack_signs(s, 0)
     assert got.tolist() == [0x0, 0x80, 0x1, 0x2]
+    # two rows of 70 columns: block 0 = (row 0, row 1), block 1 = (row 0, row 1)
+    s = -np.ones((2, 70), np.int8)
+    s[0, 1] = 1       # block 0, row 0, low word bit 1
+    s[1, 63] = 1      # block 0, row 1, high word bit 31
+    s[0, 64] = 1      # block 1, row 0, low word bit 0
+    s[1, 69] = 1      # block 1, row 1, low word bit 5
+    got = oracle.pack_signs(s, 0)
+    assert got.tolist() == [0x2, 0x0, 0x0, 0x80000000, 0x1, 0x0, 0x20, 0x0]
 
 
 def test_hand_written_words_role_b(oracle):
@@ -45,8 +53,8 @@ def test_hand_written_words_role_b(oracle):
 
 def test_zero_counts_as_plus_one(oracle):
     s = np.array([[0, -1, 5, -128]], dtype=np.int8)
-    assert oracle.pack_signs(s, 0).tolist() == [0b0101]
-    assert oracle.unpack_signs(np.array([0b0101], np.uint32), 1, 4, 0).tolist() == [[1, -1, 1, -1]]
+    assert oracle.pack_signs(s, 0).tolist() == [0b0101, 0]
+    assert oracle.unpack_signs(np.array([0b0101, 0], np.uint32), 1, 4, 0).tolist() == [[1, -1, 1, -1]]
 
 
 @pytest.mark.parametrize("role", [0, 1])
@@ -66,16 +74,18 @@ def test_random_round_trip_popcount_and_size(oracle, rows, cols, role):
     rng = np.random.default_rng(rows * 131 + cols)
     s = rng.integers(0, 2, size=(rows, cols)).astype(np.int8) * 2 - 1
     p = oracle.pack_signs(s, role)
-    n_words = rows * ((cols + 31) // 32) if role == 0 else (rows * cols + 31) // 32
+    n_words = ((cols + 63) // 64) * rows * 2 if role == 0 else (rows * cols + 31) // 32
     assert p.size == n_words == oracle.packed_words(rows, cols, role)
     assert np.array_equal(oracle.unpack_signs(p, rows, cols, role), s)
     pop = int(np.unpackbits(p.view(np.uint8)).sum())
     assert pop == int((s == 1).sum())          # so every pad bit is 0
     # independent statement of the layout with numpy bit ops
     if role == 0:
-        padded = np.zeros((rows, ((cols + 31) // 32) * 32), np.uint8)
+        nb = (cols + 63) // 64
+        padded = np.zeros((rows, nb * 64), np.uint8)
         padded[:, :cols] = (s == 1)
-        want = np.packbits(padded, axis=1, bitorder="little").view(np.uint32).reshape(-1)
+        blocks = padded.reshape(rows, nb, 64).transpose(1, 0, 2)          # block-major, then row
+        want = np.packbits(np.ascontiguousarray(blocks), axis=2, bitorder="little").view(np.uint32).reshape(-1)
     else:
         flat = np.zeros(n_words * 32, np.uint8)
         flat[:rows * cols] = (s == 1).reshape(-1)

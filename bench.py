@@ -186,7 +186,7 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=dev)
     lordba.load()
     if args.variant is not None:
-        lordba.set_variant({"auto": 0, "fma": 1, "tc": 2}[args.variant])
+        lordba.set_variant({"auto": 0, "fma": 1, "tc": 2, "mma": 3}[args.variant])
 
     # inputs: one seeded draw per rank (its own token shard); buffer sets are device-side
     # copies so that consecutive steps never hit L2.
@@ -308,7 +308,7 @@ def run_gpu(args):
         alg_bytes = workloads.algorithmic_bytes(T, D_IN, D_OUT, R, ELEM)
         sec_per_step = ms * 1e-3 / args.steps
         achieved = alg_bytes / sec_per_step / 1e9
-        variant = {0: "auto", 1: "fma", 2: "tc"}[lordba.get_variant()]
+        variant = {0: "auto", 1: "fma", 2: "tc", 3: "mma"}[lordba.get_variant()]
         line = {
             "metric": METRIC, "value": world * T * args.steps / (ms * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -346,7 +346,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=400)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--variant", default=None, choices=["auto", "fma", "tc"],
+    ap.add_argument("--variant", default=None, choices=["auto", "fma", "tc", "mma"],
                     help="pin the kernel family (default: the library's own choice)")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch to report in roofline.traffic")

@@ -69,10 +69,12 @@ typedef enum {
 
 /* Kernel families the forward entry points can be pinned to (default AUTO). */
 typedef enum {
-    LORDBA_VARIANT_AUTO = 0,  /* tensor-core kernel when the shape allows it, else FMA      */
+    LORDBA_VARIANT_AUTO = 0,  /* register-streaming kernel when the shape allows it, else FMA */
     LORDBA_VARIANT_FMA = 1,   /* CUDA-core float32 FMA kernel (always used for LORDBA_F32)  */
-    LORDBA_VARIANT_TC = 2     /* tcgen05/TMA kernel; LORDBA_EUNSUPPORTED if the shape or    */
-                              /* alignment rules it out                                     */
+    LORDBA_VARIANT_TC = 2,    /* tcgen05/TMA cluster kernel; LORDBA_EUNSUPPORTED if the     */
+                              /* shape or alignment rules it out                            */
+    LORDBA_VARIANT_MMA = 3    /* register-streaming mma.sync kernel; LORDBA_EUNSUPPORTED if */
+                              /* the shape or alignment rules it out                        */
 } lordba_variant;
 
 /* One adapted projection for the _ex and _batched entry points.  ldx / ldy are

@@ -68,18 +68,20 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t
 {
     const int variant = g_variant.load(std::memory_order_relaxed);
     if (variant == LORDBA_VARIANT_FMA || dtype == LORDBA_F32) {
-        if (variant == LORDBA_VARIANT_TC) return LORDBA_EUNSUPPORTED;
+        if (variant == LORDBA_VARIANT_TC || variant == LORDBA_VARIANT_MMA) return LORDBA_EUNSUPPORTED;
         return launch_forward_fma(projs, n, T, dtype, stream);
     }
-    // Split the list: what the tensor-core kernel can take, and the rest.
-    std::vector<lordba_proj> tc, fma;
-    for (int i = 0; i < n; ++i) (tc_supported(projs[i], T, dtype) ? tc : fma).push_back(projs[i]);
-    if (variant == LORDBA_VARIANT_TC && !fma.empty()) return LORDBA_EUNSUPPORTED;
-    if (!tc.empty()) {
-        int rc = launch_forward_tc(tc.data(), (int)tc.size(), T, dtype, stream);
-        // the driver refused a tensor map (nothing was launched for this list): CUDA-core kernel
-        if (rc == LORDBA_EUNSUPPORTED && variant == LORDBA_VARIANT_AUTO)
-            rc = launch_forward_fma(tc.data(), (int)tc.size(), T, dtype, stream);
+    // Split the list: what the chosen tensor-core kernel can take, and the rest.
+    const bool use_tc = (variant == LORDBA_VARIANT_TC);
+    std::vector<lordba_proj> fast, fma;
+    for (int i = 0; i < n; ++i) {
+        const bool ok = use_tc ? tc_supported(projs[i], T, dtype) : mma_supported(projs[i], T, dtype);
+        (ok ? fast : fma).push_back(projs[i]);
+    }
+    if (variant != LORDBA_VARIANT_AUTO && !fma.empty()) return LORDBA_EUNSUPPORTED;
+    if (!fast.empty()) {
+        const int rc = use_tc ? launch_forward_tc(fast.data(), (int)fast.size(), T, dtype, stream)
+                              : launch_forward_mma(fast.data(), (int)fast.size(), T, dtype, stream);
         if (rc != LORDBA_OK) return rc;
     }
     if (!fma.empty()) return launch_forward_fma(fma.data(), (int)fma.size(), T, dtype, stream);
@@ -224,7 +226,7 @@ int64_t lordba_adapter_bits(int64_t d_in, int64_t d_out, int r, int ell)
 
 int lordba_set_variant(int variant)
 {
-    if (variant < LORDBA_VARIANT_AUTO || variant > LORDBA_VARIANT_TC) return LORDBA_EUNSUPPORTED;
+    if (variant < LORDBA_VARIANT_AUTO || variant > LORDBA_VARIANT_MMA) return LORDBA_EUNSUPPORTED;
     g_variant.store(variant, std::memory_order_relaxed);
     return LORDBA_OK;
 }

@@ -41,4 +41,10 @@ int launch_forward_fma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
 bool tc_supported(const lordba_proj &p, int64_t T, int dtype);
 int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream);
 
+// --- forward_mma.cu ----------------------------------------------------------
+// True when the register-streaming mma.sync kernel can take this projection
+// (bf16, 16-byte aligned rows, widths and rank multiples of 8).
+bool mma_supported(const lordba_proj &p, int64_t T, int dtype);
+int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream);
+
 }  // namespace lordba

@@ -17,7 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "liblordba.so")
 
 F32, BF16 = 0, 1
-VARIANT_AUTO, VARIANT_FMA, VARIANT_TC = 0, 1, 2
+VARIANT_AUTO, VARIANT_FMA, VARIANT_TC, VARIANT_MMA = 0, 1, 2, 3
 
 _i64 = ctypes.c_int64
 _vp = ctypes.c_void_p

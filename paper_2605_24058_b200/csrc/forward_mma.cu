@@ -11,35 +11,41 @@
 //     the tiles of a call fill the SMs evenly) and needs no other CTA: the
 //     16 x r intermediate lives in registers and shared memory.
 //   * A producer warp streams the CTA's rows of x, then of y, through a ring of
-//     shared-memory slots in chunks of `cw` columns with one bulk copy per row
-//     (cp.async.bulk, completion on an mbarrier).  The chunk's slice of the
-//     scale vector and of the packed carrier travels in the same slot, so there
-//     are no other global loads.  The y chunks are requested while the first
-//     product is still running: the memory system never drains between the two.
-//   * Sixteen consumer warps each take one 64-column group of a chunk.  A lane
+//     shared-memory slots, 1024 columns per item, with ONE tensor copy per item:
+//     the row-major matrix is described to TMA as a 3-D tensor (64 columns,
+//     rows, column groups), so a box of 64 x 16 x 16 lands as sixteen 2 KiB
+//     blocks [16 rows][128 bytes], 128-byte swizzled, one block per consumer
+//     warp.  The item's slice of the scale vector and of the packed carrier
+//     travels in the same slot (two plain bulk copies), so there are no other
+//     global loads.  The y items are requested while the first product is still
+//     running: the memory system never drains between the two products.
+//   * Sixteen consumer warps each take one 64-column group of an item.  A lane
 //     reads 16-byte pieces of two token rows from the slot straight into the
 //     registers that are the A fragments of mma.sync.m16n8k16 (the K order of a
 //     product is free, so the fragment's column pattern is re-labelled to make
-//     every lane's columns contiguous); the D fragments of the second product
-//     are re-labelled the same way, so y is updated and written to global memory
-//     with 16-byte accesses.
-//   * The sign bits are expanded to bf16 operands in registers: a B fragment of
-//     the first product is (s_in as a bf16 hi/lo pair) XOR (sign-flip mask from a
-//     256-entry table), one LOP3 per register; a B fragment of the second
-//     product is +-1.0 looked up from 4 sign bits.  s_in and z = s_r * u are
-//     split into bf16 hi + lo parts, so both products carry ~16 mantissa bits
-//     into the float32 accumulators.
+//     every lane's 16 columns contiguous); the D fragments of the second product
+//     are re-labelled the same way, so a lane updates 32 contiguous bytes of a y
+//     row and writes them to global memory with one 256-bit store.
+//   * The sign bits are expanded to bf16 operands in registers without tables:
+//     a multiply by (2^a + 2^b) moves two sign bits to bits 15 and 31, and one
+//     LOP3 folds them into the operand.  A B fragment of the first product is
+//     s_in (as a bf16 hi/lo pair) with the signs XOR-ed in; a B fragment of the
+//     second product is +-1.0.  s_in and z = s_r * u are split into bf16 hi + lo
+//     parts, so both products carry ~16 mantissa bits into the float32
+//     accumulators.
 //
 // Warps split the d_in axis for the first product (fixed-order reduction
 // through shared memory, hence deterministic) and the d_out axis for the
-// second.  gridDim.z > 1 splits the y chunks over several CTAs that each repeat
+// second.  gridDim.z > 1 splits the y items over several CTAs that each repeat
 // the first product: used when a call has too few tokens to fill the GPU.
 //
 // Every mbarrier wait is bounded: after ~1 s it records a code in the device
 // status word, raises the CTA's abort flag (all later waits return at once) and
 // the kernel runs to its end.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -51,52 +57,74 @@ namespace {
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;      // + the producer warp
-constexpr int kTile = 16;            // token rows of one MMA tile
-constexpr int kGroup = 64;           // columns one warp handles per chunk (128 bytes per row)
-constexpr int kMaxChunk = kGroup * kConsumerWarps;   // 1024 columns
-constexpr int kRowPad = 64;          // bytes: consecutive rows of a slot start 64 bytes apart mod 128
-constexpr int kMaxBatch = 32;        // projections per launch
+constexpr int kTile = 16;            // token rows of one MMA tile = rows of a TMA box
+constexpr int kGroup = 64;           // columns one warp handles per item (128 bytes per row)
+constexpr int kBlockBytes = kTile * kGroup * 2;      // one warp's block of a slot: 2 KiB
+constexpr int kMaxChunk = kGroup * kConsumerWarps;   // 1024 columns per item
+constexpr int kMaxBatch = 24;        // projections per launch (two tensor maps each)
 constexpr int kMaxSlots = 8;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr long long kWaitLimitCycles = 1500000000LL;
 
+struct alignas(64) MmaProj {
+    CUtensorMap x_map;     // (64, T, d_in / 64), box 64 x 16 x 16
+    CUtensorMap y_map;     // (64, T, d_out / 64), box 64 x 16 x (cwy / 64)
+    const uint8_t *packed_A;
+    const uint8_t *packed_B;
+    const float *s_in;
+    const float *s_r;
+    const float *s_out;
+    __nv_bfloat16 *y;
+    int64_t ldy;
+    int d_in, d_out, r;
+    int y_vec32;           // y rows are 32-byte aligned: 256-bit stores
+};
+
 struct MmaBatch {
-    lordba_proj p[kMaxBatch];
+    MmaProj p[kMaxBatch];
 };
 
 struct MmaParams {
     int64_t T;
     int rows;          // token rows per CTA tile (<= 16)
-    int cwy;           // columns per y chunk: a multiple of 64, <= 1024 (x chunks are 1024 wide)
+    int cwy;           // columns per y item: a multiple of 64, <= 1024 (x items are 1024 wide)
     int slots;         // ring depth
     int *status;       // device status word
+    long long *trace;  // development builds only (-DLORDBA_MMA_TRACE): 64 timestamps per CTA
 };
+
+// Optional per-CTA timestamp trace (development builds only).
+#ifdef LORDBA_MMA_TRACE
+__device__ __forceinline__ long long global_ns()
+{
+    long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
+}
+#define MMA_TRACE(idx) do { if (prm.trace && (idx) < 64) \
+    prm.trace[((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 64 + (idx)] = global_ns(); } while (0)
+#else
+#define MMA_TRACE(idx) do { } while (0)
+#endif
 
 // ---- shared-memory plan, same on host and device --------------------------------------------
 struct SmemPlan {
-    int row_stride;    // bytes between token rows of a slot
-    int off_scale;     // slot offset of the chunk's float32 scales
-    int off_bits;      // slot offset of the chunk's sign bytes
-    int slot_bytes;
-    int off_lut1, off_lut2, off_red, off_zh, off_zl, off_bar, total;
+    int off_scale;     // slot offset of the item's float32 scales
+    int off_bits;      // slot offset of the item's sign bytes
+    int slot_bytes;    // multiple of 1024 (swizzle atom)
+    int off_red, off_zh, off_zl, off_bar, total;
 };
 
 __host__ __device__ inline SmemPlan make_plan(int rp, int r, int slots)
 {
-    constexpr int cw = kMaxChunk;
     SmemPlan s;
-    s.row_stride = cw * 2 + kRowPad;
-    s.off_scale = kTile * s.row_stride;
-    s.off_bits = s.off_scale + cw * 4;
-    s.slot_bytes = (s.off_bits + cw * r / 8 + 127) / 128 * 128;
+    s.off_scale = kConsumerWarps * kBlockBytes;
+    s.off_bits = s.off_scale + kMaxChunk * 4;
+    s.slot_bytes = (s.off_bits + kMaxChunk * r / 8 + 1023) / 1024 * 1024;
     const int ks = (rp + 15) / 16;
-    s.off_lut1 = slots * s.slot_bytes;
-    s.off_lut2 = s.off_lut1 + 256 * 16;
-    s.off_red = s.off_lut2 + 16 * 8;
+    s.off_red = slots * s.slot_bytes;
     s.off_zh = s.off_red + kConsumerWarps * kTile * rp * 4;
     s.off_zl = s.off_zh + kTile * ks * 8 * 4;
     s.off_bar = s.off_zl + kTile * ks * 8 * 4;
-    s.total = s.off_bar + (2 * kMaxSlots + 2) * 8;
+    s.total = s.off_bar + (2 * kMaxSlots + 2) * 8 + 1024;    // + slack to align the base to 1 KiB
     return s;
 }
 
@@ -130,6 +158,23 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
+// 3-D tiled tensor copy global -> shared (coordinates innermost first; c0 * 2 bytes % 16 == 0)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
+                 "[%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+__device__ __forceinline__ void st_global_256(void *p, const uint32_t (&a)[4], const uint32_t (&b)[4])
+{
+    asm volatile("st.global.L1::no_allocate.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(p), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]), "r"(b[2]), "r"(b[3])
+                 : "memory");
 }
 
 struct WaitCtx {
@@ -186,7 +231,21 @@ __device__ __forceinline__ void split2(float v0, float v1, uint32_t &hi, uint32_
     lo = pack2(v0 - lo_f(hi), v1 - hi_f(hi));
 }
 
-// The r sign bits of row j_local of a chunk's slice of B_sign (r/8 bytes per row, r % 8 == 0).
+// Sign bits (bit 1 = +1) -> sign-flip masks of bf16 pairs.  b holds sign bits in its low byte
+// (nothing above bit 7); pair p takes bits 2p and 2p+1.  b * (2^(15-2p) + 2^(30-2p)) is two
+// disjoint shifted copies of b that put bit 2p at position 15 and bit 2p+1 at position 31; the
+// caller keeps only those two positions, inverted (a 0 bit flips the sign).
+constexpr uint32_t kSignBits = 0x80008000u;
+__device__ __forceinline__ uint32_t pair_bits(uint32_t b, int p)
+{
+    return b * ((1u << (15 - 2 * p)) + (1u << (30 - 2 * p)));
+}
+__device__ __forceinline__ uint32_t with_signs(uint32_t operand, uint32_t bits)
+{
+    return operand ^ (~bits & kSignBits);
+}
+
+// The r sign bits of row j_local of an item's slice of B_sign (r/8 bytes per row, r % 8 == 0).
 template <int RP>
 __device__ __forceinline__ uint64_t b_row_bits(const uint8_t *bits, int j_local, int r)
 {
@@ -213,20 +272,22 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     constexpr int ZP = KS * 8;                 // bf16 pairs per token row of z
     constexpr bool kSplitAcc = (R8 <= 2);      // separate hi / lo accumulators: shorter MMA chains
 
-    extern __shared__ __align__(128) uint8_t smem[];
-    const lordba_proj &P = batch.p[blockIdx.y];
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzle atoms: 1 KiB
+    const MmaProj &P = batch.p[blockIdx.y];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) MMA_TRACE(0);
     const int rows = prm.rows, cwy = prm.cwy, S = prm.slots;
     constexpr int cwx = kMaxChunk;
     const int64_t t0 = (int64_t)blockIdx.x * rows;
     if (t0 >= prm.T) return;
     const int nt = (int)((prm.T - t0 < rows) ? (prm.T - t0) : rows);
     const int r = P.r;
-    const int d_in = (int)P.d_in, d_out = (int)P.d_out;
+    const int d_in = P.d_in, d_out = P.d_out;
     const SmemPlan plan = make_plan(RP, r, S);
     const uint32_t sm_base = smem_u32(smem);
 
-    // chunk items: all x chunks, then this CTA's share of the y chunks
+    // items: all x chunks, then this CTA's share of the y chunks
     const int n_x = (d_in + cwx - 1) / cwx;
     const int n_yc = (d_out + cwy - 1) / cwy;
     const int yc_begin = (int)((int64_t)blockIdx.z * n_yc / gridDim.z);
@@ -247,30 +308,16 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    uint4 *lut1 = reinterpret_cast<uint4 *>(smem + plan.off_lut1);
-    uint2 *lut2 = reinterpret_cast<uint2 *>(smem + plan.off_lut2);
-    if (tid < 256) {
-        // 8 sign bits (bit 1 = +1) -> XOR masks over four bf16 pairs (bit 0 => flip the sign)
-        uint32_t m[4];
-#pragma unroll
-        for (int p = 0; p < 4; ++p)
-            m[p] = (((tid >> (2 * p)) & 1) ? 0u : 0x8000u) | (((tid >> (2 * p + 1)) & 1) ? 0u : 0x80000000u);
-        lut1[tid] = make_uint4(m[0], m[1], m[2], m[3]);
-    } else if (tid < 256 + 16) {
-        // 4 sign bits -> two registers of +-1.0 bf16 pairs
-        const int t = tid - 256;
-        const uint32_t b0 = 0x3f803f80u ^ ((t & 1) ? 0u : 0x8000u) ^ ((t & 2) ? 0u : 0x80000000u);
-        const uint32_t b1 = 0x3f803f80u ^ ((t & 4) ? 0u : 0x8000u) ^ ((t & 8) ? 0u : 0x80000000u);
-        lut2[t] = make_uint2(b0, b1);
+    if (tid == kConsumerThreads) {
+        prefetch_tensormap(&P.x_map);
+        prefetch_tensormap(&P.y_map);
     }
     __syncthreads();
+    if (tid == 0) MMA_TRACE(1);
 
     if (warp == kConsumerWarps) {
-        // ================= producer warp: lanes 0..15 copy one token row each ===================
-        const __nv_bfloat16 *xrow = static_cast<const __nv_bfloat16 *>(P.x) + (t0 + lane) * P.ldx;
-        const __nv_bfloat16 *yrow = static_cast<const __nv_bfloat16 *>(P.y) + (t0 + lane) * P.ldy;
-        const uint8_t *pa = reinterpret_cast<const uint8_t *>(P.packed_A);
-        const uint8_t *pb = reinterpret_cast<const uint8_t *>(P.packed_B);
+        // ================= producer warp ===========================================================
+        // lane 0: the tensor copy of the item; lane 1: its scales; lane 2: its sign bytes
         for (int it = 0; it < n_items; ++it) {
             const int s = it % S;
             if (it >= S) mbar_wait(wctx, bar_empty(s), ((it / S) - 1) & 1u, kDevTmaWaitTimeout);
@@ -279,28 +326,32 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             const int cw = is_x ? cwx : cwy;
             const int col0 = is_x ? it * cwx : (yc_begin + (it - n_x)) * cwy;
             const int d = is_x ? d_in : d_out;
-            const int cwv = (d - col0 < cw) ? (d - col0) : cw;              // valid columns, % 8 == 0
-            const uint32_t bits_bytes = is_x ? (uint32_t)((cwv + kGroup - 1) / kGroup) * r * 8u
-                                             : (uint32_t)cwv * r / 8u;
+            const int cwv = (d - col0 < cw) ? (d - col0) : cw;              // valid columns, % 64 == 0
+            const uint32_t bits_bytes = (uint32_t)cwv * r / 8u;           // same for A blocks and B rows
+            const uint32_t box_bytes = (uint32_t)(cw / kGroup) * kBlockBytes;   // a box is always whole
             const uint32_t slot = sm_base + s * plan.slot_bytes;
-            if (lane == 0)
-                mbar_arrive_expect_tx(bar_full(s), (uint32_t)nt * cwv * 2u + (uint32_t)cwv * 4u + bits_bytes);
+            if (lane == 0) {
+                MMA_TRACE(2 + it);
+                mbar_arrive_expect_tx(bar_full(s), box_bytes + (uint32_t)cwv * 4u + bits_bytes);
+                tma_load_3d(slot, is_x ? &P.x_map : &P.y_map, 0, (int)t0, col0 / kGroup, bar_full(s));
+            }
             __syncwarp();
-            if (lane < nt) {
-                bulk_load(slot + lane * plan.row_stride, (is_x ? xrow : yrow) + col0, (uint32_t)cwv * 2u, bar_full(s));
-            } else if (lane == 16) {
+            if (lane == 1) {
                 bulk_load(slot + plan.off_scale, (is_x ? P.s_in : P.s_out) + col0, (uint32_t)cwv * 4u, bar_full(s));
-            } else if (lane == 17) {
-                const uint8_t *src = is_x ? pa + (size_t)(col0 / kGroup) * r * 8 : pb + (size_t)col0 * r / 8;
-                bulk_load(slot + plan.off_bits, src, bits_bytes, bar_full(s));
+            } else if (lane == 2) {
+                bulk_load(slot + plan.off_bits, (is_x ? P.packed_A : P.packed_B) + (size_t)col0 * r / 8,
+                          bits_bytes, bar_full(s));
             }
         }
     } else {
         // ================= consumer warps ========================================================
         const int g = lane >> 2, q = lane & 3;
-        const bool v0 = g < nt, v1 = g + 8 < nt;    // this lane's two token rows exist
-        const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
-        const int gcol = warp * kGroup;             // first column of this warp's group within a chunk
+        const bool v0 = g < nt, v1 = g + 8 < nt;    // this lane's two token rows belong to the tile
+        const int gcol = warp * kGroup;             // first column of this warp's group within an item
+        // this lane's pieces of its two rows inside the warp's 2 KiB block (128-byte swizzle:
+        // 16-byte piece c of row i sits at piece c ^ (i & 7))
+        const int off_r0 = warp * kBlockBytes + g * 128, off_r1 = off_r0 + 8 * 128;
+        const int pc0 = ((2 * q) ^ g) * 16, pc1 = ((2 * q + 1) ^ g) * 16;
 
         // ---- first product: u[t,k] = sum_i A_sign[k,i] s_in[i] x[t,i] -----------------------
         float acc[kSplitAcc ? 2 : 1][R8][4];
@@ -316,30 +367,29 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             const int s = it % S;
             const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), (it / S) & 1u, kDevMmaWaitTimeout));
             const int cwv = (d_in - it * cwx < cwx) ? (d_in - it * cwx) : cwx;
+            if (tid == 0) MMA_TRACE(20 + it);
             if (gcol < cwv && ok) {
                 const uint8_t *slot = smem + s * plan.slot_bytes;
-                // this lane's columns: gcol + 8q .. +7 (half A) and gcol + 32 + 8q .. +7 (half B)
-                const int ca = gcol + 8 * q, cb = ca + 32;
-                const uint8_t *r0 = slot + g * plan.row_stride, *r1 = r0 + 8 * plan.row_stride;
-                uint4 v[4];
-                v[0] = (v0 && ca < cwv) ? *reinterpret_cast<const uint4 *>(r0 + 2 * ca) : zero4;
-                v[1] = (v0 && cb < cwv) ? *reinterpret_cast<const uint4 *>(r0 + 2 * cb) : zero4;
-                v[2] = (v1 && ca < cwv) ? *reinterpret_cast<const uint4 *>(r1 + 2 * ca) : zero4;
-                v[3] = (v1 && cb < cwv) ? *reinterpret_cast<const uint4 *>(r1 + 2 * cb) : zero4;
+                // this lane's columns: gcol + 16q .. +7 (piece A) and gcol + 16q + 8 .. +15 (piece B);
+                // rows past the tile are other tokens or zero fill and only reach unused outputs
+                const uint4 xa0 = *reinterpret_cast<const uint4 *>(slot + off_r0 + pc0);
+                const uint4 xb0 = *reinterpret_cast<const uint4 *>(slot + off_r0 + pc1);
+                const uint4 xa1 = *reinterpret_cast<const uint4 *>(slot + off_r1 + pc0);
+                const uint4 xb1 = *reinterpret_cast<const uint4 *>(slot + off_r1 + pc1);
                 // s_in of the group as bf16 pairs (hi, lo): lane l converts columns 2l, 2l+1,
-                // then every lane collects the pairs of its 16 columns
-                uint32_t ph = 0u, pl = 0u;
-                if (gcol + 2 * lane < cwv) {
+                // then every lane collects the 8 pairs of its 16 columns
+                uint32_t ph, pl;
+                {
                     const float2 sc = *reinterpret_cast<const float2 *>(slot + plan.off_scale + 4 * (gcol + 2 * lane));
                     split2(sc.x, sc.y, ph, pl);
                 }
                 uint32_t hA[4], hB[4], lA[4], lB[4];
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
-                    hA[p] = __shfl_sync(0xffffffffu, ph, 4 * q + p);
-                    hB[p] = __shfl_sync(0xffffffffu, ph, 16 + 4 * q + p);
-                    lA[p] = __shfl_sync(0xffffffffu, pl, 4 * q + p);
-                    lB[p] = __shfl_sync(0xffffffffu, pl, 16 + 4 * q + p);
+                    hA[p] = __shfl_sync(0xffffffffu, ph, 8 * q + p);
+                    hB[p] = __shfl_sync(0xffffffffu, ph, 8 * q + 4 + p);
+                    lA[p] = __shfl_sync(0xffffffffu, pl, 8 * q + p);
+                    lB[p] = __shfl_sync(0xffffffffu, pl, 8 * q + 4 + p);
                 }
                 const uint2 *blk = reinterpret_cast<const uint2 *>(slot + plan.off_bits) + warp * r;
 #pragma unroll
@@ -347,22 +397,27 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     int k = 8 * a + g;
                     if (k > r - 1) k = r - 1;                       // padded rank rows: result unused
                     const uint2 sb = blk[k];                         // the row's 64 sign bits of this block
-                    const uint4 mA = lut1[(sb.x >> (8 * q)) & 0xffu];
-                    const uint4 mB = lut1[(sb.y >> (8 * q)) & 0xffu];
+                    const uint32_t w16 = ((q & 2) ? sb.y : sb.x) >> (16 * (q & 1));
+                    const uint32_t bA = w16 & 0xffu, bB = (w16 >> 8) & 0xffu;
                     float(&ch)[4] = acc[0][a];
                     float(&cl)[4] = acc[kSplitAcc ? 1 : 0][a];
-                    mma_bf16(ch, v[0].x, v[2].x, v[0].y, v[2].y, hA[0] ^ mA.x, hA[1] ^ mA.y);
-                    mma_bf16(cl, v[0].x, v[2].x, v[0].y, v[2].y, lA[0] ^ mA.x, lA[1] ^ mA.y);
-                    mma_bf16(ch, v[0].z, v[2].z, v[0].w, v[2].w, hA[2] ^ mA.z, hA[3] ^ mA.w);
-                    mma_bf16(cl, v[0].z, v[2].z, v[0].w, v[2].w, lA[2] ^ mA.z, lA[3] ^ mA.w);
-                    mma_bf16(ch, v[1].x, v[3].x, v[1].y, v[3].y, hB[0] ^ mB.x, hB[1] ^ mB.y);
-                    mma_bf16(cl, v[1].x, v[3].x, v[1].y, v[3].y, lB[0] ^ mB.x, lB[1] ^ mB.y);
-                    mma_bf16(ch, v[1].z, v[3].z, v[1].w, v[3].w, hB[2] ^ mB.z, hB[3] ^ mB.w);
-                    mma_bf16(cl, v[1].z, v[3].z, v[1].w, v[3].w, lB[2] ^ mB.z, lB[3] ^ mB.w);
+                    uint32_t m0 = pair_bits(bA, 0), m1 = pair_bits(bA, 1);
+                    mma_bf16(ch, xa0.x, xa1.x, xa0.y, xa1.y, with_signs(hA[0], m0), with_signs(hA[1], m1));
+                    mma_bf16(cl, xa0.x, xa1.x, xa0.y, xa1.y, with_signs(lA[0], m0), with_signs(lA[1], m1));
+                    m0 = pair_bits(bA, 2); m1 = pair_bits(bA, 3);
+                    mma_bf16(ch, xa0.z, xa1.z, xa0.w, xa1.w, with_signs(hA[2], m0), with_signs(hA[3], m1));
+                    mma_bf16(cl, xa0.z, xa1.z, xa0.w, xa1.w, with_signs(lA[2], m0), with_signs(lA[3], m1));
+                    m0 = pair_bits(bB, 0); m1 = pair_bits(bB, 1);
+                    mma_bf16(ch, xb0.x, xb1.x, xb0.y, xb1.y, with_signs(hB[0], m0), with_signs(hB[1], m1));
+                    mma_bf16(cl, xb0.x, xb1.x, xb0.y, xb1.y, with_signs(lB[0], m0), with_signs(lB[1], m1));
+                    m0 = pair_bits(bB, 2); m1 = pair_bits(bB, 3);
+                    mma_bf16(ch, xb0.z, xb1.z, xb0.w, xb1.w, with_signs(hB[2], m0), with_signs(hB[3], m1));
+                    mma_bf16(cl, xb0.z, xb1.z, xb0.w, xb1.w, with_signs(lB[2], m0), with_signs(lB[3], m1));
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
+            if (tid == 0) MMA_TRACE(40 + it);
         }
 
         // ---- reduce u over the warps in a fixed order, z = s_r * u, split into bf16 hi + lo ---
@@ -399,6 +454,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             zL[idx] = lo;
         }
         consumer_sync();
+        if (tid == 0) MMA_TRACE(60);
 
         // ---- second product: y[t,j] += s_out[j] sum_k B_sign[j,k] z[t,k] ---------------------
         // A fragments: k position (2q, 2q+1, 2q+8, 2q+9) of k-step s <-> ranks 16s + 4q + (0,1,2,3)
@@ -412,73 +468,94 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             zh[s][0] = h0.x; zh[s][1] = h1.x; zh[s][2] = h0.y; zh[s][3] = h1.y;
             zl[s][0] = l0.x; zl[s][1] = l1.x; zl[s][2] = l0.y; zl[s][3] = l1.y;
         }
-        __nv_bfloat16 *yrow0 = static_cast<__nv_bfloat16 *>(P.y) + (t0 + g) * P.ldy;
+        __nv_bfloat16 *yrow0 = P.y + (t0 + g) * P.ldy;
         __nv_bfloat16 *yrow1 = yrow0 + 8 * P.ldy;
+        const bool vec32 = P.y_vec32 != 0;
 
         for (; it < n_items; ++it) {
             const int s = it % S;
             const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), (it / S) & 1u, kDevEpilogueWaitTimeout));
             const int col0 = (yc_begin + (it - n_x)) * cwy;
             const int cwv = (d_out - col0 < cwy) ? (d_out - col0) : cwy;
+            if (tid == 0) MMA_TRACE(20 + it);
             if (gcol < cwv && ok) {
                 const uint8_t *slot = smem + s * plan.slot_bytes;
                 const uint8_t *bits = slot + plan.off_bits;
-                // Output column of n-block (h, nb), accumulator column n = 2q + e:
-                //   gcol + 32h + 8q + 2nb + e, so that a lane owns 8 consecutive columns per half.
-                // As the holder of B-fragment column n = g this lane expands the signs of
-                //   j = gcol + 32h + 8(g>>1) + 2nb + (g&1).
+                // Output column of n-block i, accumulator column n = 2q + e: gcol + 16q + 2i + e, so
+                // that a lane owns 16 consecutive columns.  As the holder of B-fragment column
+                // n = g this lane expands the signs of j = gcol + 16(g>>1) + 2i + (g&1).
                 float c[8][4];
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) c[i][e] = 0.0f;
+                const int jb = gcol + 16 * (g >> 1) + (g & 1);
+                if (RP == 16) {
+                    // rows jb - (g&1) .. + 15 are 16 half-words: word i holds rows 2i (low) and 2i+1
+                    const uint4 w0 = *reinterpret_cast<const uint4 *>(bits + 2 * (jb - (g & 1)));
+                    const uint4 w1 = *reinterpret_cast<const uint4 *>(bits + 2 * (jb - (g & 1)) + 16);
+                    const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+                    const int sh = 16 * (g & 1) + 4 * q;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t nib = (w[i] >> sh) & 0xfu;
+                        const uint32_t b0 = with_signs(0x3f803f80u, nib * 0x40008000u);
+                        const uint32_t b1 = with_signs(0x3f803f80u, nib * 0x10002000u);
+                        mma_bf16(c[i], zh[0][0], zh[0][1], zh[0][2], zh[0][3], b0, b1);
+                        mma_bf16(c[i], zl[0][0], zl[0][1], zl[0][2], zl[0][3], b0, b1);
+                    }
+                } else {
 #pragma unroll
-                    for (int nb = 0; nb < 4; ++nb) {
-                        int j = gcol + 32 * h + 8 * (g >> 1) + 2 * nb + (g & 1);
-                        if (j > cwv - 1) j = cwv - 1;                  // columns past the end: unused
-                        const uint64_t rb = b_row_bits<RP>(bits, j, r);
+                    for (int i = 0; i < 8; ++i) {
+                        const uint64_t rb = b_row_bits<RP>(bits, jb + 2 * i, r);
 #pragma unroll
                         for (int ks = 0; ks < KS; ++ks) {
                             const uint32_t nib = (uint32_t)(rb >> (16 * ks + 4 * q)) & 0xfu;
-                            const uint2 b = lut2[nib];
-                            mma_bf16(c[h * 4 + nb], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b.x, b.y);
-                            mma_bf16(c[h * 4 + nb], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b.x, b.y);
+                            const uint32_t b0 = with_signs(0x3f803f80u, nib * 0x40008000u);
+                            const uint32_t b1 = with_signs(0x3f803f80u, nib * 0x10002000u);
+                            mma_bf16(c[i], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b0, b1);
+                            mma_bf16(c[i], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b0, b1);
                         }
                     }
                 }
-                const uint8_t *r0 = slot + g * plan.row_stride, *r1 = r0 + 8 * plan.row_stride;
+                const float4 *so4 = reinterpret_cast<const float4 *>(slot + plan.off_scale + 4 * (gcol + 16 * q));
+                float so[16];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int col = gcol + 32 * h + 8 * q;
-                    if (col < cwv) {
-                        const float4 s0 = *reinterpret_cast<const float4 *>(slot + plan.off_scale + 4 * col);
-                        const float4 s1 = *reinterpret_cast<const float4 *>(slot + plan.off_scale + 4 * col + 16);
-                        const float so[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                for (int i = 0; i < 4; ++i) {
+                    const float4 t = so4[i];
+                    so[4 * i] = t.x; so[4 * i + 1] = t.y; so[4 * i + 2] = t.z; so[4 * i + 3] = t.w;
+                }
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {          // token rows g and g + 8
-                            if (half == 0 ? v0 : v1) {
-                                const uint4 yv = *reinterpret_cast<const uint4 *>((half == 0 ? r0 : r1) + 2 * col);
-                                const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
-                                uint32_t ow[4];
+                for (int half = 0; half < 2; ++half) {                  // token rows g and g + 8
+                    if (half == 0 ? v0 : v1) {
+                        const int off = half == 0 ? off_r0 : off_r1;
+                        const uint4 ya = *reinterpret_cast<const uint4 *>(slot + off + pc0);
+                        const uint4 yb = *reinterpret_cast<const uint4 *>(slot + off + pc1);
+                        const uint32_t yw[8] = {ya.x, ya.y, ya.z, ya.w, yb.x, yb.y, yb.z, yb.w};
+                        uint32_t oa[4], ob[4];
 #pragma unroll
-                                for (int nb = 0; nb < 4; ++nb) {
-                                    const float o0 = fmaf(so[2 * nb], c[h * 4 + nb][2 * half], lo_f(yw[nb]));
-                                    const float o1 = fmaf(so[2 * nb + 1], c[h * 4 + nb][2 * half + 1], hi_f(yw[nb]));
-                                    ow[nb] = pack2(o0, o1);
-                                }
-                                __stcs(reinterpret_cast<uint4 *>((half == 0 ? yrow0 : yrow1) + col0 + col),
-                                       make_uint4(ow[0], ow[1], ow[2], ow[3]));
-                            }
+                        for (int i = 0; i < 8; ++i) {
+                            const float o0 = fmaf(so[2 * i], c[i][2 * half], lo_f(yw[i]));
+                            const float o1 = fmaf(so[2 * i + 1], c[i][2 * half + 1], hi_f(yw[i]));
+                            if (i < 4) oa[i] = pack2(o0, o1);
+                            else ob[i - 4] = pack2(o0, o1);
+                        }
+                        __nv_bfloat16 *dst = (half == 0 ? yrow0 : yrow1) + col0 + gcol + 16 * q;
+                        if (vec32) {
+                            st_global_256(dst, oa, ob);
+                        } else {
+                            __stcs(reinterpret_cast<uint4 *>(dst), make_uint4(oa[0], oa[1], oa[2], oa[3]));
+                            __stcs(reinterpret_cast<uint4 *>(dst) + 1, make_uint4(ob[0], ob[1], ob[2], ob[3]));
                         }
                     }
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
+            if (tid == 0) MMA_TRACE(40 + it);
         }
     }
+    if (tid == 0) MMA_TRACE(61);
 
     // ---- teardown: after an abort, give copies that may still be in flight time to land ---------
     __syncthreads();
@@ -486,6 +563,41 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         const long long start = clock64();
         while (clock64() - start < 2000000LL) __nanosleep(1000);
     }
+}
+
+// ------------------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Row-major T x d bf16 matrix (row pitch ld elements, d % 64 == 0) seen as the 3-D tensor
+// (column in group: 64, row: T, column group: d / 64); a box is 64 x 16 rows x `groups`.
+bool make_map(CUtensorMap *map, const void *base, int64_t T, int64_t d, int64_t ld, int groups)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)kGroup, (cuuint64_t)T, (cuuint64_t)(d / kGroup)};
+    const cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)kGroup * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)kGroup, (cuuint32_t)kTile, (cuuint32_t)groups};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int padded_rank(int r) { return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64; }
@@ -520,19 +632,17 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
 
 bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
 {
-    if (dtype != LORDBA_BF16 || T < 1) return false;
+    if (dtype != LORDBA_BF16 || T < 1 || T > (1 << 30)) return false;
     if (p.r % 8 != 0 || p.r < 8 || p.r > kMaxRank) return false;
-    if (p.d_in % 8 != 0 || p.d_out % 8 != 0 || p.ldx % 8 != 0 || p.ldy % 8 != 0) return false;
+    // whole 64-column groups (the 3-D tensor view), 16-byte aligned rows
+    if (p.d_in % kGroup != 0 || p.d_out % kGroup != 0 || p.ldx % 8 != 0 || p.ldy % 8 != 0) return false;
     if (p.d_in > (1 << 30) || p.d_out > (1 << 30)) return false;
-    // every bulk copy needs 16-byte aligned addresses and a size that is a multiple of 16:
-    // rows of x / y, chunk slices of the scales, of packed_A (r * 8 bytes per 64 columns) and of
-    // packed_B (r / 8 bytes per column; the last chunk ends at d_out * r / 8 bytes)
     if (reinterpret_cast<uintptr_t>(p.x) % 16 || reinterpret_cast<uintptr_t>(p.y) % 16) return false;
+    // the scale and carrier slices of an item travel as bulk copies: 16-byte aligned sources
     if (reinterpret_cast<uintptr_t>(p.s_in) % 16 || reinterpret_cast<uintptr_t>(p.s_out) % 16 ||
         reinterpret_cast<uintptr_t>(p.packed_A) % 16 || reinterpret_cast<uintptr_t>(p.packed_B) % 16)
         return false;
-    if ((p.d_out * p.r / 8) % 16 != 0) return false;
-    return true;
+    return encode_fn() != nullptr;
 }
 
 int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream)
@@ -543,13 +653,13 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
     if (!status) return LORDBA_ECUDA;
     const int sms = sm_count();
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
-        MmaBatch b;
+        const lordba_proj *sel[kMaxBatch];
         int m = 0, max_r = 0;
         int64_t min_dout = (int64_t)1 << 40;
         for (int i = 0; i <= n; ++i) {
             const bool take = (i < n) && padded_rank(projs[i].r) == rp;
             if (take) {
-                b.p[m++] = projs[i];
+                sel[m++] = &projs[i];
                 if (projs[i].r > max_r) max_r = projs[i].r;
                 if (projs[i].d_out < min_dout) min_dout = projs[i].d_out;
             }
@@ -564,8 +674,8 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                 if (rows > kTile) rows = kTile;
                 if (rows < 1) rows = 1;
                 const int64_t tiles = (T + rows - 1) / rows;
-                // Few tokens: split the y chunks over several CTAs per tile (each repeats the
-                // first product), with narrower chunks so that there is something to split.
+                // Few tokens: split the y items over several CTAs per tile (each repeats the
+                // first product), with narrower items so that there is something to split.
                 int64_t want_splits = sms / (tiles * m);
                 if (want_splits < 1) want_splits = 1;
                 int cw = kMaxChunk;
@@ -574,8 +684,29 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                 if (splits > want_splits) splits = want_splits;
                 if (splits > 64) splits = 64;
 
+                MmaBatch b;
+                std::memset(&b, 0, sizeof(b));
+                for (int k = 0; k < m; ++k) {
+                    const lordba_proj &q = *sel[k];
+                    MmaProj &t = b.p[k];
+                    if (!make_map(&t.x_map, q.x, T, q.d_in, q.ldx, kConsumerWarps) ||
+                        !make_map(&t.y_map, q.y, T, q.d_out, q.ldy, cw / kGroup))
+                        return LORDBA_ECUDA;
+                    t.packed_A = reinterpret_cast<const uint8_t *>(q.packed_A);
+                    t.packed_B = reinterpret_cast<const uint8_t *>(q.packed_B);
+                    t.s_in = q.s_in; t.s_r = q.s_r; t.s_out = q.s_out;
+                    t.y = static_cast<__nv_bfloat16 *>(q.y);
+                    t.ldy = q.ldy;
+                    t.d_in = (int)q.d_in; t.d_out = (int)q.d_out; t.r = q.r;
+                    t.y_vec32 = (reinterpret_cast<uintptr_t>(q.y) % 32 == 0 && q.ldy % 16 == 0) ? 1 : 0;
+                }
                 MmaParams prm;
                 prm.T = T; prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
+                prm.trace = nullptr;
+#ifdef LORDBA_MMA_TRACE
+                if (const char *tp = std::getenv("LORDBA_MMA_TRACE_PTR"))
+                    prm.trace = reinterpret_cast<long long *>(std::strtoull(tp, nullptr, 0));
+#endif
                 int slots = kMaxSlots;
                 while (slots > 2 && make_plan(rp, max_r, slots).total > kSmemBudget) --slots;
                 const SmemPlan plan = make_plan(rp, max_r, slots);

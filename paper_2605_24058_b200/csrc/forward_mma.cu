@@ -61,19 +61,19 @@ constexpr int kTile = 16;            // token rows of one MMA tile = rows of a T
 constexpr int kGroup = 64;           // columns one warp handles per item (128 bytes per row)
 constexpr int kBlockBytes = kTile * kGroup * 2;      // one warp's block of a slot: 2 KiB
 constexpr int kMaxChunk = kGroup * kConsumerWarps;   // 1024 columns per item
-constexpr int kMaxBatch = 24;        // projections per launch (two tensor maps each)
+constexpr int kMaxBatch = 24;        // projections per launch (six tensor maps each)
 constexpr int kMaxSlots = 8;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr long long kWaitLimitCycles = 1500000000LL;
 
 struct alignas(64) MmaProj {
-    CUtensorMap x_map;     // (64, T, d_in / 64), box 64 x 16 x 16
-    CUtensorMap y_map;     // (64, T, d_out / 64), box 64 x 16 x (cwy / 64)
-    const uint8_t *packed_A;
-    const uint8_t *packed_B;
-    const float *s_in;
+    CUtensorMap x_map;     // bf16 (64, T, d_in / 64), box 64 x 16 x 16, 128-byte swizzle
+    CUtensorMap y_map;     // bf16 (64, T, d_out / 64), box 64 x 16 x (cwy / 64), 128-byte swizzle
+    CUtensorMap si_map;    // f32 (64, d_in / 64), box 64 x 16: the scales of an x item
+    CUtensorMap so_map;    // f32 (64, d_out / 64), box 64 x (cwy / 64)
+    CUtensorMap pa_map;    // u32 (16, d_in r / 512), box 16 x 2r: the sign bytes of an x item
+    CUtensorMap pb_map;    // u32 (16, d_out r / 512), box 16 x (cwy r / 512)
     const float *s_r;
-    const float *s_out;
     __nv_bfloat16 *y;
     int64_t ldy;
     int d_in, d_out, r;
@@ -90,17 +90,13 @@ struct MmaParams {
     int cwy;           // columns per y item: a multiple of 64, <= 1024 (x items are 1024 wide)
     int slots;         // ring depth
     int *status;       // device status word
-    long long *trace;  // development builds only (-DLORDBA_MMA_TRACE): 64 timestamps per CTA
+    long long *trace;  // development builds only (-DLORDBA_MMA_TRACE): 64 clock64 stamps per CTA
 };
 
 // Optional per-CTA timestamp trace (development builds only).
 #ifdef LORDBA_MMA_TRACE
-__device__ __forceinline__ long long global_ns()
-{
-    long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
-}
 #define MMA_TRACE(idx) do { if (prm.trace && (idx) < 64) \
-    prm.trace[((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 64 + (idx)] = global_ns(); } while (0)
+    prm.trace[((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 64 + (idx)] = clock64(); } while (0)
 #else
 #define MMA_TRACE(idx) do { } while (0)
 #endif
@@ -153,22 +149,20 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
                  "selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
-// global -> shared bulk copy; both addresses 16-byte aligned, size a multiple of 16
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+// Tiled tensor copies global -> shared (coordinates innermost first; c0 * element size % 16 == 0).
+// Plain (untiled) bulk copies are not used: they were measured at ~8 bytes per cycle here,
+// against more than 100 for a tiled box.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
 {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+                 "[%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
-// 3-D tiled tensor copy global -> shared (coordinates innermost first; c0 * 2 bytes % 16 == 0)
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar)
 {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
                  "[%0], [%1, {%3, %4, %5}], [%2];"
                  ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
-{
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
 __device__ __forceinline__ void st_global_256(void *p, const uint32_t (&a)[4], const uint32_t (&b)[4])
 {
@@ -300,7 +294,9 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + plan.off_bar + 2 * kMaxSlots * 8);
     const WaitCtx wctx{abort_flag, prm.status};
 
-    if (tid == 0) {
+    if (tid == kConsumerThreads) {
+        // the producer's first lane prepares the barriers and requests the first items at once;
+        // everybody else meets it at the barrier below
         for (int s = 0; s < S; ++s) {
             mbar_init(bar_full(s), 1);
             mbar_init(bar_empty(s), kConsumerWarps);
@@ -308,39 +304,33 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (tid == kConsumerThreads) {
-        prefetch_tensormap(&P.x_map);
-        prefetch_tensormap(&P.y_map);
-    }
+    auto issue_item = [&](int it) {       // one thread
+        const int s = it % S;
+        const bool is_x = it < n_x;
+        const int cw = is_x ? cwx : cwy;
+        const int col0 = is_x ? it * cwx : (yc_begin + (it - n_x)) * cwy;
+        // a box is always whole: what lies past the tensor is filled with zeros and counted
+        const uint32_t bytes = (uint32_t)(cw / kGroup) * kBlockBytes + (uint32_t)cw * 4u + (uint32_t)cw * r / 8u;
+        const uint32_t slot = sm_base + s * plan.slot_bytes;
+        MMA_TRACE(2 + it);
+        mbar_arrive_expect_tx(bar_full(s), bytes);
+        tma_load_3d(slot, is_x ? &P.x_map : &P.y_map, 0, (int)t0, col0 / kGroup, bar_full(s));
+        tma_load_2d(slot + plan.off_scale, is_x ? &P.si_map : &P.so_map, 0, col0 / kGroup, bar_full(s));
+        tma_load_2d(slot + plan.off_bits, is_x ? &P.pa_map : &P.pb_map, 0, col0 * r / 512, bar_full(s));
+        MMA_TRACE(10 + it);
+    };
+    const int n_first = n_items < S ? n_items : S;
+    if (tid == kConsumerThreads)
+        for (int it = 0; it < n_first; ++it) issue_item(it);
     __syncthreads();
     if (tid == 0) MMA_TRACE(1);
 
     if (warp == kConsumerWarps) {
-        // ================= producer warp ===========================================================
-        // lane 0: the tensor copy of the item; lane 1: its scales; lane 2: its sign bytes
-        for (int it = 0; it < n_items; ++it) {
-            const int s = it % S;
-            if (it >= S) mbar_wait(wctx, bar_empty(s), ((it / S) - 1) & 1u, kDevTmaWaitTimeout);
-            if (*abort_flag) break;
-            const bool is_x = it < n_x;
-            const int cw = is_x ? cwx : cwy;
-            const int col0 = is_x ? it * cwx : (yc_begin + (it - n_x)) * cwy;
-            const int d = is_x ? d_in : d_out;
-            const int cwv = (d - col0 < cw) ? (d - col0) : cw;              // valid columns, % 64 == 0
-            const uint32_t bits_bytes = (uint32_t)cwv * r / 8u;           // same for A blocks and B rows
-            const uint32_t box_bytes = (uint32_t)(cw / kGroup) * kBlockBytes;   // a box is always whole
-            const uint32_t slot = sm_base + s * plan.slot_bytes;
-            if (lane == 0) {
-                MMA_TRACE(2 + it);
-                mbar_arrive_expect_tx(bar_full(s), box_bytes + (uint32_t)cwv * 4u + bits_bytes);
-                tma_load_3d(slot, is_x ? &P.x_map : &P.y_map, 0, (int)t0, col0 / kGroup, bar_full(s));
-            }
-            __syncwarp();
-            if (lane == 1) {
-                bulk_load(slot + plan.off_scale, (is_x ? P.s_in : P.s_out) + col0, (uint32_t)cwv * 4u, bar_full(s));
-            } else if (lane == 2) {
-                bulk_load(slot + plan.off_bits, (is_x ? P.packed_A : P.packed_B) + (size_t)col0 * r / 8,
-                          bits_bytes, bar_full(s));
+        // ================= producer warp: one lane refills the slots as they are released ========
+        if (lane == 0) {
+            for (int it = n_first; it < n_items; ++it) {
+                if (!mbar_wait(wctx, bar_empty(it % S), ((it / S) - 1) & 1u, kDevTmaWaitTimeout)) break;
+                issue_item(it);
             }
         }
     } else {
@@ -585,19 +575,36 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// Row-major T x d bf16 matrix (row pitch ld elements, d % 64 == 0) seen as the 3-D tensor
-// (column in group: 64, row: T, column group: d / 64); a box is 64 x 16 rows x `groups`.
-bool make_map(CUtensorMap *map, const void *base, int64_t T, int64_t d, int64_t ld, int groups)
+bool encode(CUtensorMap *map, CUtensorMapDataType type, int rank, const void *base, const cuuint64_t *dims,
+            const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swizzle)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, type, (cuuint32_t)rank, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Row-major T x d bf16 matrix (row pitch ld elements, d % 64 == 0) seen as the 3-D tensor
+// (column in group: 64, row: T, column group: d / 64); a box is 64 x 16 rows x `groups`.
+bool make_data_map(CUtensorMap *map, const void *base, int64_t T, int64_t d, int64_t ld, int groups)
+{
     const cuuint64_t dims[3] = {(cuuint64_t)kGroup, (cuuint64_t)T, (cuuint64_t)(d / kGroup)};
     const cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)kGroup * 2};
     const cuuint32_t box[3] = {(cuuint32_t)kGroup, (cuuint32_t)kTile, (cuuint32_t)groups};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+// A dense array seen as n_rows rows of `row_elems` 4-byte elements; a box is `box_rows` whole
+// rows, laid out densely in shared memory.
+bool make_linear_map(CUtensorMap *map, CUtensorMapDataType type, const void *base, int row_elems,
+                     int64_t n_rows, int box_rows)
+{
+    const cuuint64_t dims[2] = {(cuuint64_t)row_elems, (cuuint64_t)n_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_elems * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)row_elems, (cuuint32_t)box_rows};
+    return encode(map, type, 2, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
 int padded_rank(int r) { return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64; }
@@ -689,12 +696,19 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                 for (int k = 0; k < m; ++k) {
                     const lordba_proj &q = *sel[k];
                     MmaProj &t = b.p[k];
-                    if (!make_map(&t.x_map, q.x, T, q.d_in, q.ldx, kConsumerWarps) ||
-                        !make_map(&t.y_map, q.y, T, q.d_out, q.ldy, cw / kGroup))
+                    // sign bytes: d r / 8 per carrier, as rows of 16 words; an item holds cw r / 512 rows
+                    if (!make_data_map(&t.x_map, q.x, T, q.d_in, q.ldx, kConsumerWarps) ||
+                        !make_data_map(&t.y_map, q.y, T, q.d_out, q.ldy, cw / kGroup) ||
+                        !make_linear_map(&t.si_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, q.s_in, kGroup,
+                                         q.d_in / kGroup, kConsumerWarps) ||
+                        !make_linear_map(&t.so_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, q.s_out, kGroup,
+                                         q.d_out / kGroup, cw / kGroup) ||
+                        !make_linear_map(&t.pa_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_A, 16,
+                                         q.d_in * q.r / 512, kMaxChunk * q.r / 512) ||
+                        !make_linear_map(&t.pb_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_B, 16,
+                                         q.d_out * q.r / 512, cw * q.r / 512))
                         return LORDBA_ECUDA;
-                    t.packed_A = reinterpret_cast<const uint8_t *>(q.packed_A);
-                    t.packed_B = reinterpret_cast<const uint8_t *>(q.packed_B);
-                    t.s_in = q.s_in; t.s_r = q.s_r; t.s_out = q.s_out;
+                    t.s_r = q.s_r;
                     t.y = static_cast<__nv_bfloat16 *>(q.y);
                     t.ldy = q.ldy;
                     t.d_in = (int)q.d_in; t.d_out = (int)q.d_out; t.r = q.r;

@@ -16,9 +16,9 @@
 //     rows, column groups), so a box of 64 x 16 x 16 lands as sixteen 2 KiB
 //     blocks [16 rows][128 bytes], 128-byte swizzled, one block per consumer
 //     warp.  The item's slice of the scale vector and of the packed carrier
-//     travels in the same slot (two plain bulk copies), so there are no other
-//     global loads.  The y items are requested while the first product is still
-//     running: the memory system never drains between the two products.
+//     travels in the same slot (two small 2-D tensor copies), so there are no
+//     other global loads.  The y items are requested while the first product is
+//     still running: the memory system never drains between the two products.
 //   * Sixteen consumer warps each take one 64-column group of an item.  A lane
 //     reads 16-byte pieces of two token rows from the slot straight into the
 //     registers that are the A fragments of mma.sync.m16n8k16 (the K order of a
@@ -294,6 +294,9 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + plan.off_bar + 2 * kMaxSlots * 8);
     const WaitCtx wctx{abort_flag, prm.status};
 
+    // Let the next kernel of the stream start its own set-up as soon as SMs free up (it waits
+    // for this grid to complete before it touches global data, as this one does below).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == kConsumerThreads) {
         // the producer's first lane prepares the barriers and requests the first items at once;
         // everybody else meets it at the barrier below
@@ -303,6 +306,8 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // everything before this line overlapped the previous kernel; nothing after it may
+        asm volatile("griddepcontrol.wait;" ::: "memory");
     }
     auto issue_item = [&](int it) {       // one thread
         const int s = it % S;
@@ -631,8 +636,22 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
                                        kSmemBudget);
     });
     if (attr_rc != cudaSuccess) return attr_rc;
-    mma_forward_kernel<RP><<<grid, kThreads, smem, stream>>>(b, prm);
-    return cudaGetLastError();
+    // Programmatic dependent launch: the CTAs of this grid may become resident, fetch their
+    // parameters and set up their barriers while the previous kernel of the stream drains; they
+    // touch no global data before griddepcontrol.wait, which returns once that kernel has
+    // completed and its writes are visible.
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP>, b, prm);
 }
 
 }  // namespace

@@ -64,7 +64,8 @@ typedef enum {
     LORDBA_EUNSUPPORTED = 2,  /* rank outside 1..64, unknown dtype / role / variant         */
     LORDBA_EALIGN = 3,        /* a pointer is not aligned to its element type               */
     LORDBA_ECUDA = 4,         /* a CUDA runtime call or the launch failed                   */
-    LORDBA_ETIMEOUT = 5       /* a bounded device-side wait gave up (see lordba_device_status) */
+    LORDBA_ETIMEOUT = 5,      /* a bounded device-side wait gave up (see lordba_device_status) */
+    LORDBA_ETOOLARGE = 6      /* the call needs more than the library's built-in scratch buffer */
 } lordba_status;
 
 /* Kernel families the forward entry points can be pinned to (default AUTO). */
@@ -151,6 +152,34 @@ int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
                                 const float *s_out, void *y_host, int64_t T, int64_t d_in,
                                 int64_t d_out, int r, int dtype, void *workspace,
                                 size_t workspace_bytes, void *stream);
+
+/*
+ * lordba_adapter_forward_host without a caller-supplied workspace (an addition of this library;
+ * the paper has no counterpart).
+ *
+ * For callers that have host activations but are not in a position to obtain device memory: code
+ * that runs where cudaMalloc is off limits (inside a latency-critical loop, since an allocation
+ * can synchronise the whole device; under a host framework that owns all device memory and hands
+ * none to plug-ins; in a process whose memory budget was fixed at start-up).  The device staging
+ * area for x and y is a buffer of LORDBA_STATIC_SCRATCH_BYTES that is part of the library image:
+ * every GPU on which the library is loaded holds it until the process exits, and this call
+ * allocates nothing and frees nothing.
+ *
+ *   - Same arguments, order of work and result as lordba_adapter_forward_host, minus the
+ *     workspace.  If lordba_host_workspace_bytes(T, d_in, d_out, dtype) exceeds
+ *     LORDBA_STATIC_SCRATCH_BYTES the call returns LORDBA_ETOOLARGE and does nothing.
+ *   - The first call on a device looks up the buffer's device address (with that device current)
+ *     and remembers it; make that first call outside any stream capture.
+ *   - All calls on a device share the one buffer.  It still holds the previous call's x and y;
+ *     nothing in it has to start at zero, because every byte that is read was copied in by the
+ *     same call first.  Two calls whose work overlaps on the GPU (different streams, no
+ *     ordering between them) would overwrite each other's staging data: order them.
+ */
+#define LORDBA_STATIC_SCRATCH_BYTES (8u << 20)
+int lordba_adapter_forward_host_static(const void *x_host, const uint32_t *packed_A,
+                                       const uint32_t *packed_B, const float *s_in, const float *s_r,
+                                       const float *s_out, void *y_host, int64_t T, int64_t d_in,
+                                       int64_t d_out, int r, int dtype, void *stream);
 
 /* Storage of one adapter in bits, Eq. 5: r(d_in+d_out) + 16 ell (d_in+r+d_out). */
 int64_t lordba_adapter_bits(int64_t d_in, int64_t d_out, int r, int ell);

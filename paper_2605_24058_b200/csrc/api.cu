@@ -219,6 +219,60 @@ int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
     return LORDBA_OK;
 }
 
+}  // extern "C"
+
+namespace lordba {
+namespace {
+
+// Staging area of lordba_adapter_forward_host_static.  In host code this name is only a handle
+// for cudaGetSymbolAddress, never a pointer that a kernel or a copy could use.
+static __device__ __align__(256) unsigned char g_static_scratch[LORDBA_STATIC_SCRATCH_BYTES];
+std::mutex g_scratch_mutex;
+void *g_scratch_ptr[64] = {nullptr};
+
+// Device address of the staging area on the current device (looked up once per device).
+void *static_scratch()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        g_scratch_ptr[dev] = p;
+    }
+    return g_scratch_ptr[dev];
+}
+
+}  // namespace
+}  // namespace lordba
+
+extern "C" {
+
+int lordba_adapter_forward_host_static(const void *x_host, const uint32_t *packed_A,
+                                       const uint32_t *packed_B, const float *s_in, const float *s_r,
+                                       const float *s_out, void *y_host, int64_t T, int64_t d_in,
+                                       int64_t d_out, int r, int dtype, void *stream)
+{
+    if (dtype != LORDBA_F32 && dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    if (T < 0 || d_in < 1 || d_out < 1) return LORDBA_EINVAL;
+    const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
+    // sizes that cannot fit are refused before any multiplication can overflow
+    const size_t limit = LORDBA_STATIC_SCRATCH_BYTES;
+    if ((size_t)T > limit || (size_t)d_in > limit || (size_t)d_out > limit ||
+        (size_t)T * (size_t)(d_in + d_out) > limit / e)
+        return LORDBA_ETOOLARGE;
+    const size_t need = lordba_host_workspace_bytes(T, d_in, d_out, dtype);
+    if (need > limit) return LORDBA_ETOOLARGE;
+    void *scratch = static_scratch();
+    if (!scratch) return LORDBA_ECUDA;
+    return lordba_adapter_forward_host(x_host, packed_A, packed_B, s_in, s_r, s_out, y_host, T, d_in,
+                                       d_out, r, dtype, scratch, limit, stream);
+}
+
 int64_t lordba_adapter_bits(int64_t d_in, int64_t d_out, int r, int ell)
 {
     return (int64_t)r * (d_in + d_out) + 16 * (int64_t)ell * (d_in + r + d_out);
@@ -258,6 +312,7 @@ const char *lordba_status_string(int status)
         case LORDBA_EALIGN: return "misaligned pointer";
         case LORDBA_ECUDA: return "CUDA runtime error";
         case LORDBA_ETIMEOUT: return "device-side wait timed out";
+        case LORDBA_ETOOLARGE: return "the call needs more than the built-in scratch buffer";
         default: return "unknown status";
     }
 }

@@ -48,6 +48,8 @@ _SIGNATURES = {
     "lordba_host_workspace_bytes": (ctypes.c_size_t, [_i64, _i64, _i64, ctypes.c_int]),
     "lordba_adapter_forward_host": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int,
                                                                ctypes.c_int, _vp, ctypes.c_size_t, _vp]),
+    "lordba_adapter_forward_host_static": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int,
+                                                                      ctypes.c_int, _vp]),
     "lordba_adapter_bits": (_i64, [_i64, _i64, ctypes.c_int, ctypes.c_int]),
     "lordba_set_variant": (ctypes.c_int, [ctypes.c_int]),
     "lordba_get_variant": (ctypes.c_int, []),
@@ -216,6 +218,28 @@ def adapter_forward_host(x_host, packed_A, packed_B, s_in, s_r, s_out, y_host, r
         _dtype_code(x_host), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
         _stream(stream))
     _check(rc, "lordba_adapter_forward_host")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def adapter_forward_host_static(x_host, packed_A, packed_B, s_in, s_r, s_out, y_host, r: int,
+                                stream=None) -> None:
+    """Host x / y like ``adapter_forward_host``, but the device staging area is the library's own
+    built-in buffer (``STATIC_SCRATCH_BYTES``): for callers that may not allocate device memory.
+    Calls on one device share that buffer and must not overlap on the GPU."""
+    if x_host.is_cuda or y_host.is_cuda:
+        raise ValueError("x_host and y_host must be CPU tensors")
+    if not (x_host.is_contiguous() and y_host.is_contiguous()):
+        raise ValueError("host buffers must be contiguous")
+    _need_cuda(packed_A, packed_B, s_in, s_r, s_out)
+    T, d_in = x_host.shape
+    d_out = y_host.shape[1]
+    rc = load().lordba_adapter_forward_host_static(
+        x_host.data_ptr(), packed_A.data_ptr(), packed_B.data_ptr(), s_in.data_ptr(),
+        s_r.data_ptr(), s_out.data_ptr(), y_host.data_ptr(), T, d_in, d_out, r,
+        _dtype_code(x_host), _stream(stream))
+    _check(rc, "lordba_adapter_forward_host_static")
 
 
 def adapter_bits(d_in: int, d_out: int, r: int, ell: int = 1) -> int:

@@ -204,8 +204,12 @@ def run_gpu(args):
     s_r = torch.from_numpy(p.s_r).to(dev)
     s_out = torch.from_numpy(p.s_out).to(dev)
 
+    # Consecutive steps work on different buffer sets, so every step but the first of a graph is
+    # declared independent of the ones before it (LORDBA_PROJ_OVERLAP): its loads may start while
+    # the previous step's last tiles are still being written.
     def step(i):
-        lordba.adapter_forward(xs[i % n_sets], packed_A, packed_B, s_in, s_r, s_out, ys[i % n_sets], R)
+        lordba.adapter_forward(xs[i % n_sets], packed_A, packed_B, s_in, s_r, s_out, ys[i % n_sets], R,
+                               overlap=(i % n_sets != 0) and not args.no_overlap)
 
     # correctness of the configuration being timed: sampled rows against the oracle (rank 0)
     parity = None
@@ -319,6 +323,9 @@ def run_gpu(args):
                        "l2": "steps rotate through %d device buffer sets (%.0f MB > 4 x L2)"
                              % (n_sets, n_sets * set_bytes / 1e6),
                        "launch": "CUDA graph of %d steps replayed" % n_sets,
+                       "step_dependency": "every step waits for the previous one" if args.no_overlap else
+                                          "steps after the first of a graph are declared independent "
+                                          "(LORDBA_PROJ_OVERLAP): they may overlap the previous step's tail",
                        "kernel_variant": variant, "parallelism": "token shards, no collective",
                        "parity_max_err_over_rms": parity},
             "hbm_gbs": achieved,
@@ -351,6 +358,8 @@ def main():
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch to report in roofline.traffic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="every step waits for the previous one to finish (no LORDBA_PROJ_OVERLAP)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

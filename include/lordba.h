@@ -90,8 +90,22 @@ typedef struct lordba_proj {
     void           *y;          /* [device] T x d_out, pitch ldy, updated in place */
     int64_t d_in, d_out, ldx, ldy;
     int32_t r;
-    int32_t reserved;           /* must be 0 */
+    int32_t flags;              /* 0 or LORDBA_PROJ_OVERLAP; other bits must be 0 */
 } lordba_proj;
+
+/*
+ * lordba_proj.flags: a promise by the caller that lets consecutive calls overlap on the GPU.
+ * A call (all of its projections) made with LORDBA_PROJ_OVERLAP may start while the library
+ * calls before it on the same stream are still running, back to and including the most recent
+ * call made WITHOUT the flag.  The caller guarantees that, within such a run of calls, no call
+ * reads what another one writes (a y buffer) and no call writes what another one reads or
+ * writes, and that nothing else was enqueued on the stream in between.  Example: the q, k and v
+ * adapters of one layer read the same x and update three different y buffers; the first is
+ * called without the flag (it must see the kernel that produced x), the other two with it.
+ * Work enqueued after the run is ordered after all of it, as usual.  Only the streaming bf16
+ * kernel acts on the flag; elsewhere it is accepted and ignored.
+ */
+#define LORDBA_PROJ_OVERLAP 1
 
 /* Number of uint32 words of a packed carrier (layout above); -1 on bad arguments. */
 int64_t lordba_packed_words(int64_t rows, int64_t cols, int role);
@@ -133,7 +147,9 @@ int lordba_adapter_forward_ex(const lordba_proj *p, int64_t T, int dtype, void *
  * instance the seven adapted projections q,k,v,o,gate,up,down of one decoder
  * layer, Section 5 Setup) in as few launches as the kernel-parameter space
  * allows.  projs: [host] array, read before the call returns.  The projections
- * must write disjoint y buffers.
+ * are treated as simultaneous: their y buffers must be pairwise disjoint and no
+ * projection's x may overlap any projection's y (LORDBA_EINVAL otherwise); the
+ * launches of one call may therefore overlap on the GPU.
  */
 int lordba_adapter_forward_batched(const lordba_proj *projs, int n_proj, int64_t T, int dtype,
                                    void *stream);

@@ -47,7 +47,7 @@ int validate_proj(const lordba_proj &p, int64_t T, int dtype)
 {
     if (dtype != LORDBA_F32 && dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
     if (T < 0 || p.d_in < 1 || p.d_out < 1 || p.ldx < p.d_in || p.ldy < p.d_out) return LORDBA_EINVAL;
-    if (p.reserved != 0) return LORDBA_EINVAL;
+    if ((p.flags & ~LORDBA_PROJ_OVERLAP) != 0) return LORDBA_EINVAL;
     if (p.r < 1 || p.r > kMaxRank) return LORDBA_EUNSUPPORTED;
     if (T == 0) return LORDBA_OK;   // nothing is touched: the pointers may be anything
     if (!p.x || !p.packed_A || !p.packed_B || !p.s_in || !p.s_r || !p.s_out || !p.y)
@@ -64,7 +64,9 @@ int validate_proj(const lordba_proj &p, int64_t T, int dtype)
     return LORDBA_OK;
 }
 
-int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream)
+// batch_checked: the caller has verified that the projections of this call are independent of
+// one another (disjoint y buffers, no x inside a y), so its launches may overlap each other.
+int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream, bool batch_checked)
 {
     const int variant = g_variant.load(std::memory_order_relaxed);
     if (variant == LORDBA_VARIANT_FMA || dtype == LORDBA_F32) {
@@ -81,7 +83,8 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t
     if (variant != LORDBA_VARIANT_AUTO && !fma.empty()) return LORDBA_EUNSUPPORTED;
     if (!fast.empty()) {
         const int rc = use_tc ? launch_forward_tc(fast.data(), (int)fast.size(), T, dtype, stream)
-                              : launch_forward_mma(fast.data(), (int)fast.size(), T, dtype, stream);
+                              : launch_forward_mma(fast.data(), (int)fast.size(), T, dtype, stream,
+                                                   batch_checked);
         if (rc != LORDBA_OK) return rc;
     }
     if (!fma.empty()) return launch_forward_fma(fma.data(), (int)fma.size(), T, dtype, stream);
@@ -141,7 +144,7 @@ int lordba_adapter_forward_ex(const lordba_proj *p, int64_t T, int dtype, void *
     const int rc = validate_proj(*p, T, dtype);
     if (rc != LORDBA_OK) return rc;
     if (T == 0) return LORDBA_OK;
-    return dispatch(p, 1, T, dtype, static_cast<cudaStream_t>(stream));
+    return dispatch(p, 1, T, dtype, static_cast<cudaStream_t>(stream), false);
 }
 
 int lordba_adapter_forward(const void *x, const uint32_t *packed_A, const uint32_t *packed_B,
@@ -170,16 +173,20 @@ int lordba_adapter_forward_batched(const lordba_proj *projs, int n_proj, int64_t
         if (rc != LORDBA_OK) return rc;
     }
     if (T > 0) {
-        // outputs must be pairwise disjoint (n_proj is small: 7 per layer, 224 per model)
+        // outputs must be pairwise disjoint and no input may lie in an output (n_proj is small:
+        // 7 per layer, 224 per model)
         for (int i = 0; i < n_proj; ++i)
-            for (int j = i + 1; j < n_proj; ++j) {
+            for (int j = 0; j < n_proj; ++j) {
+                if (i == j) continue;
                 const size_t ni = ((size_t)(T - 1) * projs[i].ldy + projs[i].d_out) * e;
                 const size_t nj = ((size_t)(T - 1) * projs[j].ldy + projs[j].d_out) * e;
-                if (overlaps(projs[i].y, ni, projs[j].y, nj)) return LORDBA_EINVAL;
+                const size_t nx = ((size_t)(T - 1) * projs[i].ldx + projs[i].d_in) * e;
+                if (j > i && overlaps(projs[i].y, ni, projs[j].y, nj)) return LORDBA_EINVAL;
+                if (overlaps(projs[i].x, nx, projs[j].y, nj)) return LORDBA_EINVAL;
             }
     }
     if (T == 0 || n_proj == 0) return LORDBA_OK;
-    return dispatch(projs, n_proj, T, dtype, static_cast<cudaStream_t>(stream));
+    return dispatch(projs, n_proj, T, dtype, static_cast<cudaStream_t>(stream), true);
 }
 
 size_t lordba_host_workspace_bytes(int64_t T, int64_t d_in, int64_t d_out, int dtype)
@@ -213,7 +220,7 @@ int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(xd, x_host, bx, cudaMemcpyHostToDevice, s) != cudaSuccess) return LORDBA_ECUDA;
     if (cudaMemcpyAsync(yd, y_host, by, cudaMemcpyHostToDevice, s) != cudaSuccess) return LORDBA_ECUDA;
-    const int rc2 = dispatch(&p, 1, T, dtype, s);
+    const int rc2 = dispatch(&p, 1, T, dtype, s, false);
     if (rc2 != LORDBA_OK) return rc2;
     if (cudaMemcpyAsync(y_host, yd, by, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LORDBA_ECUDA;
     return LORDBA_OK;

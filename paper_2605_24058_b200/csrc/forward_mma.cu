@@ -89,6 +89,7 @@ struct MmaParams {
     int rows;          // token rows per CTA tile (<= 16)
     int cwy;           // columns per y item: a multiple of 64, <= 1024 (x items are 1024 wide)
     int slots;         // ring depth
+    int wait_prev;     // 1: the previous kernel of the stream must be complete before any global access
     int *status;       // device status word
     long long *trace;  // development builds only (-DLORDBA_MMA_TRACE): 64 clock64 stamps per CTA
 };
@@ -294,9 +295,13 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + plan.off_bar + 2 * kMaxSlots * 8);
     const WaitCtx wctx{abort_flag, prm.status};
 
-    // Let the next kernel of the stream start its own set-up as soon as SMs free up (it waits
-    // for this grid to complete before it touches global data, as this one does below).
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Programmatic dependent launch.  A kernel that must see its predecessor (wait_prev) sets up,
+    // waits for it, and only then lets its own successor in: whatever ran before it is complete
+    // by the time anything after it starts.  A kernel that the caller declared independent of the
+    // calls before it lets its successor in at once, streams without waiting, and waits for its
+    // predecessor just before it exits, so that "this grid is complete" still implies "everything
+    // before it is complete".
+    if (!prm.wait_prev) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == kConsumerThreads) {
         // the producer's first lane prepares the barriers and requests the first items at once;
         // everybody else meets it at the barrier below
@@ -306,8 +311,11 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // everything before this line overlapped the previous kernel; nothing after it may
-        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (prm.wait_prev) {
+            // everything before this line overlapped the previous kernel; nothing after it may
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        }
     }
     auto issue_item = [&](int it) {       // one thread
         const int s = it % S;
@@ -558,6 +566,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         const long long start = clock64();
         while (clock64() - start < 2000000LL) __nanosleep(1000);
     }
+    if (!prm.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ------------------------------------------------------------------------------------- host side
@@ -671,13 +680,17 @@ bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
     return encode_fn() != nullptr;
 }
 
-int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream)
+int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream,
+                       bool batch_checked)
 {
     if (n == 0 || T == 0) return LORDBA_OK;
     if (dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
     int *status = device_status_word();
     if (!status) return LORDBA_ECUDA;
     const int sms = sm_count();
+    bool all_overlap = true;          // the caller's promise covers the call only if every projection carries it
+    for (int i = 0; i < n; ++i) all_overlap = all_overlap && (projs[i].flags & LORDBA_PROJ_OVERLAP);
+    int launches = 0;
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
         const lordba_proj *sel[kMaxBatch];
         int m = 0, max_r = 0;
@@ -735,6 +748,8 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                 }
                 MmaParams prm;
                 prm.T = T; prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
+                prm.wait_prev = (launches == 0) ? !all_overlap : !batch_checked;
+                ++launches;
                 prm.trace = nullptr;
 #ifdef LORDBA_MMA_TRACE
                 if (const char *tp = std::getenv("LORDBA_MMA_TRACE_PTR"))

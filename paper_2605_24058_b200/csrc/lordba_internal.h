@@ -45,6 +45,10 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
 // True when the register-streaming mma.sync kernel can take this projection
 // (bf16, 16-byte aligned rows, widths and rank multiples of 8).
 bool mma_supported(const lordba_proj &p, int64_t T, int dtype);
-int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream);
+// batch_checked: the projections are known to be independent of one another, so the launches of
+// this call may overlap each other; LORDBA_PROJ_OVERLAP on every projection lets the first
+// launch overlap the previous call as well.
+int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream,
+                       bool batch_checked);
 
 }  // namespace lordba

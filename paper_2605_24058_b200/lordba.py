@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_PKG, "liblordba.so")
 
 F32, BF16 = 0, 1
 VARIANT_AUTO, VARIANT_FMA, VARIANT_TC, VARIANT_MMA = 0, 1, 2, 3
+PROJ_OVERLAP = 1
 
 _i64 = ctypes.c_int64
 _vp = ctypes.c_void_p
@@ -33,7 +34,7 @@ class Proj(ctypes.Structure):
     """Mirror of ``lordba_proj``."""
     _fields_ = [("x", _vp), ("packed_A", _vp), ("packed_B", _vp), ("s_in", _vp), ("s_r", _vp),
                 ("s_out", _vp), ("y", _vp), ("d_in", _i64), ("d_out", _i64), ("ldx", _i64),
-                ("ldy", _i64), ("r", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("ldy", _i64), ("r", ctypes.c_int32), ("flags", ctypes.c_int32)]
 
 
 _SIGNATURES = {
@@ -145,7 +146,7 @@ def unpack_signs(packed: torch.Tensor, rows: int, cols: int, role: int, stream=N
     return signs
 
 
-def make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int) -> Proj:
+def make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, flags: int = 0) -> Proj:
     """Fill a ``lordba_proj`` from 2-D (possibly row-strided) x, y and 1-D parameter tensors."""
     _need_cuda(x, packed_A, packed_B, s_in, s_r, s_out, y)
     if x.dim() != 2 or y.dim() != 2 or x.shape[0] != y.shape[0]:
@@ -165,16 +166,18 @@ def make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int) -> Proj:
     ldx = x.stride(0) if x.shape[0] > 1 else max(d_in, x.stride(0))
     ldy = y.stride(0) if y.shape[0] > 1 else max(d_out, y.stride(0))
     return Proj(x.data_ptr(), packed_A.data_ptr(), packed_B.data_ptr(), s_in.data_ptr(),
-                s_r.data_ptr(), s_out.data_ptr(), y.data_ptr(), d_in, d_out, ldx, ldy, r, 0)
+                s_r.data_ptr(), s_out.data_ptr(), y.data_ptr(), d_in, d_out, ldx, ldy, r, flags)
 
 
-def adapter_forward(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, stream=None) -> None:
+def adapter_forward(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, stream=None,
+                    overlap: bool = False) -> None:
     """y += adapter(x) in place, through lordba_adapter_forward{,_f32} (dense rows)
-    or lordba_adapter_forward_ex (row-strided x / y)."""
-    p = make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r)
+    or lordba_adapter_forward_ex (row-strided x / y, or overlap=True: the caller's promise
+    LORDBA_PROJ_OVERLAP that this call is independent of the run of calls before it)."""
+    p = make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r, PROJ_OVERLAP if overlap else 0)
     T = x.shape[0]
     lib = load()
-    dense = x.is_contiguous() and y.is_contiguous()
+    dense = x.is_contiguous() and y.is_contiguous() and not overlap
     if dense and x.dtype == torch.bfloat16:
         rc = lib.lordba_adapter_forward(p.x, p.packed_A, p.packed_B, p.s_in, p.s_r, p.s_out, p.y,
                                         T, p.d_in, p.d_out, r, _stream(stream))

@@ -56,7 +56,7 @@ def test_library_helpers_match_oracle(lib, oracle):
 
 def _proj(lordba, **kw):
     base = dict(x=0x1000, packed_A=0x2000, packed_B=0x3000, s_in=0x4000, s_r=0x5000, s_out=0x6000,
-                y=0x100000, d_in=64, d_out=64, ldx=64, ldy=64, r=8, reserved=0)
+                y=0x100000, d_in=64, d_out=64, ldx=64, ldy=64, r=8, flags=0)
     base.update(kw)
     return lordba.Proj(**base)
 
@@ -75,7 +75,7 @@ def test_bad_arguments_return_codes_without_launching(lib):
     assert call(_proj(lordba, d_in=0)) == EINVAL
     assert call(_proj(lordba, ldx=63)) == EINVAL
     assert call(_proj(lordba, ldy=10)) == EINVAL
-    assert call(_proj(lordba, reserved=7)) == EINVAL
+    assert call(_proj(lordba, flags=6)) == EINVAL
     assert call(_proj(lordba, r=0)) == EUNSUP
     assert call(_proj(lordba, r=65)) == EUNSUP
     assert call(_proj(lordba), dt=9) == EUNSUP
@@ -93,6 +93,9 @@ def test_bad_arguments_return_codes_without_launching(lib):
     two = (lordba.Proj * 2)(_proj(lordba), _proj(lordba, x=0x8000))
     assert lib.lordba_adapter_forward_batched(two, 2, 4, lordba.BF16, None) == EINVAL
     assert lib.lordba_adapter_forward_batched(two, -1, 4, lordba.BF16, None) == EINVAL
+    # batched: one projection's x lies inside another projection's y
+    chained = (lordba.Proj * 2)(_proj(lordba), _proj(lordba, x=0x100000, y=0x200000))
+    assert lib.lordba_adapter_forward_batched(chained, 2, 4, lordba.BF16, None) == EINVAL
     assert lib.lordba_adapter_forward_batched(None, 0, 4, lordba.BF16, None) == 0
     # pack / unpack
     assert lib.lordba_pack_signs(0x1000, 4, 4, 5, 0x2000, None) == EUNSUP

@@ -322,6 +322,30 @@ def test_padded_rank_matches(oracle, vname, variant):
     assert_close(torch_to_f64(b.y), want, "bf16", "r=16 padded " + vname)
 
 
+def test_overlapping_run_of_calls_q_k_v(oracle):
+    """Three adapters on the same x writing three y buffers, the second and third declared
+    independent of the calls before them (LORDBA_PROJ_OVERLAP), then a plain call that reads one
+    of those outputs as its x: every result must still match the oracle."""
+    T = 2048
+    base = workloads.make_projection(4096, 4096, 16, T, "bf16", seed=60)
+    projs = [base] + [workloads.make_projection(4096, 4096, 16, T, "bf16", seed=61 + i) for i in range(2)]
+    for p in projs[1:]:
+        p.x = base.x
+    devs = [DeviceProj(p) for p in projs]
+    for i, d in enumerate(devs):
+        lordba.adapter_forward(devs[0].x, d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, d.y, 16,
+                               overlap=(i > 0))
+    # dependent follow-up: x = the first call's output, no flag
+    nxt = workloads.make_projection(4096, 4096, 16, T, "bf16", seed=70)
+    dn = DeviceProj(nxt)
+    lordba.adapter_forward(devs[0].y, dn.packed_A, dn.packed_B, dn.s_in, dn.s_r, dn.s_out, dn.y, 16)
+    torch.cuda.synchronize()
+    for p, d in zip(projs, devs):
+        assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16", "overlap run " + str(p.meta["seed"]))
+    nxt.x = devs[0].y.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert_close(torch_to_f64(dn.y), oracle_forward(oracle, nxt), "bf16", "call after the run")
+
+
 def test_host_buffer_entry(oracle):
     p = workloads.make_projection(1024, 1536, 16, 300, "bf16", seed=9)
     d = DeviceProj(p)

@@ -54,16 +54,16 @@
 namespace lordba {
 namespace {
 
-constexpr int kConsumerWarps = 16;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;      // + the producer warp
+// Consumer warps per CTA (template parameter NW): 16 with one CTA per SM, or 8 with two CTAs per
+// SM, so that one CTA's start-up and first-load latency hide behind the other's streaming.
 constexpr int kTile = 16;            // token rows of one MMA tile = rows of a TMA box
 constexpr int kGroup = 64;           // columns one warp handles per item (128 bytes per row)
 constexpr int kBlockBytes = kTile * kGroup * 2;      // one warp's block of a slot: 2 KiB
-constexpr int kMaxChunk = kGroup * kConsumerWarps;   // 1024 columns per item
+constexpr int kMaxWarps = 16;
 constexpr int kMaxBatch = 24;        // projections per launch (six tensor maps each)
 constexpr int kMaxSlots = 8;
 constexpr int kSmemBudget = 227 * 1024;
+constexpr int kSmemBudgetHalf = 112 * 1024;      // two CTAs per SM
 constexpr long long kWaitLimitCycles = 1500000000LL;
 
 struct alignas(64) MmaProj {
@@ -110,15 +110,16 @@ struct SmemPlan {
     int off_red, off_zh, off_zl, off_bar, total;
 };
 
-__host__ __device__ inline SmemPlan make_plan(int rp, int r, int slots)
+// nw: consumer warps = 64-column groups per item
+__host__ __device__ inline SmemPlan make_plan(int nw, int rp, int r, int slots)
 {
     SmemPlan s;
-    s.off_scale = kConsumerWarps * kBlockBytes;
-    s.off_bits = s.off_scale + kMaxChunk * 4;
-    s.slot_bytes = (s.off_bits + kMaxChunk * r / 8 + 1023) / 1024 * 1024;
+    s.off_scale = nw * kBlockBytes;
+    s.off_bits = s.off_scale + nw * kGroup * 4;
+    s.slot_bytes = (s.off_bits + nw * kGroup * r / 8 + 1023) / 1024 * 1024;
     const int ks = (rp + 15) / 16;
     s.off_red = slots * s.slot_bytes;
-    s.off_zh = s.off_red + kConsumerWarps * kTile * rp * 4;
+    s.off_zh = s.off_red + nw * kTile * rp * 4;
     s.off_zl = s.off_zh + kTile * ks * 8 * 4;
     s.off_bar = s.off_zl + kTile * ks * 8 * 4;
     s.total = s.off_bar + (2 * kMaxSlots + 2) * 8 + 1024;    // + slack to align the base to 1 KiB
@@ -197,9 +198,10 @@ __device__ __forceinline__ bool mbar_wait(const WaitCtx &w, uint32_t bar, uint32
     }
 }
 
+template <int kThreadsInBarrier>
 __device__ __forceinline__ void consumer_sync()
 {
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreadsInBarrier) : "memory");
 }
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -258,14 +260,15 @@ __device__ __forceinline__ uint64_t b_row_bits(const uint8_t *bits, int j_local,
 }
 
 // RP: rank padded to 8, 16, 32 or 64.
-template <int RP>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int RP, int NW>
+__global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 2)
 mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant__ MmaParams prm)
 {
     constexpr int R8 = RP / 8;                 // 8-row blocks of A_sign = n-blocks of the first product
     constexpr int KS = (RP + 15) / 16;         // k-steps of the second product per z part
     constexpr int ZP = KS * 8;                 // bf16 pairs per token row of z
     constexpr bool kSplitAcc = (R8 <= 2);      // separate hi / lo accumulators: shorter MMA chains
+    constexpr int kConsumerWarps = NW, kConsumerThreads = NW * 32;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzle atoms: 1 KiB
@@ -273,13 +276,13 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) MMA_TRACE(0);
     const int rows = prm.rows, cwy = prm.cwy, S = prm.slots;
-    constexpr int cwx = kMaxChunk;
+    constexpr int cwx = NW * kGroup;
     const int64_t t0 = (int64_t)blockIdx.x * rows;
     if (t0 >= prm.T) return;
     const int nt = (int)((prm.T - t0 < rows) ? (prm.T - t0) : rows);
     const int r = P.r;
     const int d_in = P.d_in, d_out = P.d_out;
-    const SmemPlan plan = make_plan(RP, r, S);
+    const SmemPlan plan = make_plan(NW, RP, r, S);
     const uint32_t sm_base = smem_u32(smem);
 
     // items: all x chunks, then this CTA's share of the y chunks
@@ -436,7 +439,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             *reinterpret_cast<float2 *>(d0) = make_float2(c[0], c[1]);
             *reinterpret_cast<float2 *>(d0 + 8 * RP) = make_float2(c[2], c[3]);
         }
-        consumer_sync();
+        consumer_sync<kConsumerThreads>();
         for (int idx = tid; idx < kTile * ZP; idx += kConsumerThreads) {
             const int tok = idx / ZP, pr = idx - tok * ZP;
             float u0 = 0.0f, u1 = 0.0f;
@@ -456,7 +459,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             zH[idx] = hi;
             zL[idx] = lo;
         }
-        consumer_sync();
+        consumer_sync<kConsumerThreads>();
         if (tid == 0) MMA_TRACE(60);
 
         // ---- second product: y[t,j] += s_out[j] sum_k B_sign[j,k] z[t,k] ---------------------
@@ -635,13 +638,13 @@ int sm_count()
     return n;
 }
 
-template <int RP>
+template <int RP, int NW>
 cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem, cudaStream_t stream)
 {
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, []() {
-        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSmemBudget);
     });
     if (attr_rc != cudaSuccess) return attr_rc;
@@ -652,7 +655,7 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(NW * 32 + 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr;
@@ -660,7 +663,7 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP>, b, prm);
+    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP, NW>, b, prm);
 }
 
 }  // namespace
@@ -717,7 +720,15 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                 // first product), with narrower items so that there is something to split.
                 int64_t want_splits = sms / (tiles * m);
                 if (want_splits < 1) want_splits = 1;
-                int cw = kMaxChunk;
+                // Two small CTAs per SM when there is a second CTA to pair with: more than one
+                // wave of tiles, or a call that may overlap its neighbours.  One's start-up and
+                // first-load latency then hide behind the other's streaming.  A lone single-wave
+                // call keeps one CTA with 16 consumer warps per SM.
+                const bool overlaps_neighbours = (launches == 0) ? all_overlap : batch_checked;
+                const int nw = (tiles * m > sms || overlaps_neighbours) ? 8 : kMaxWarps;
+                const int max_chunk = nw * kGroup;
+                const int smem_budget = (nw == kMaxWarps) ? kSmemBudget : kSmemBudgetHalf;
+                int cw = max_chunk;
                 while (cw > 128 && (min_dout + cw - 1) / cw < want_splits) cw /= 2;
                 int64_t splits = (min_dout + cw - 1) / cw;
                 if (splits > want_splits) splits = want_splits;
@@ -729,14 +740,14 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                     const lordba_proj &q = *sel[k];
                     MmaProj &t = b.p[k];
                     // sign bytes: d r / 8 per carrier, as rows of 16 words; an item holds cw r / 512 rows
-                    if (!make_data_map(&t.x_map, q.x, T, q.d_in, q.ldx, kConsumerWarps) ||
+                    if (!make_data_map(&t.x_map, q.x, T, q.d_in, q.ldx, nw) ||
                         !make_data_map(&t.y_map, q.y, T, q.d_out, q.ldy, cw / kGroup) ||
                         !make_linear_map(&t.si_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, q.s_in, kGroup,
-                                         q.d_in / kGroup, kConsumerWarps) ||
+                                         q.d_in / kGroup, nw) ||
                         !make_linear_map(&t.so_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, q.s_out, kGroup,
                                          q.d_out / kGroup, cw / kGroup) ||
                         !make_linear_map(&t.pa_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_A, 16,
-                                         q.d_in * q.r / 512, kMaxChunk * q.r / 512) ||
+                                         q.d_in * q.r / 512, max_chunk * q.r / 512) ||
                         !make_linear_map(&t.pb_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_B, 16,
                                          q.d_out * q.r / 512, cw * q.r / 512))
                         return LORDBA_ECUDA;
@@ -748,7 +759,7 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                 }
                 MmaParams prm;
                 prm.T = T; prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
-                prm.wait_prev = (launches == 0) ? !all_overlap : !batch_checked;
+                prm.wait_prev = !overlaps_neighbours;
                 ++launches;
                 prm.trace = nullptr;
 #ifdef LORDBA_MMA_TRACE
@@ -756,17 +767,26 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                     prm.trace = reinterpret_cast<long long *>(std::strtoull(tp, nullptr, 0));
 #endif
                 int slots = kMaxSlots;
-                while (slots > 2 && make_plan(rp, max_r, slots).total > kSmemBudget) --slots;
-                const SmemPlan plan = make_plan(rp, max_r, slots);
+                while (slots > 2 && make_plan(nw, rp, max_r, slots).total > smem_budget) --slots;
+                const SmemPlan plan = make_plan(nw, rp, max_r, slots);
                 if (plan.total > kSmemBudget) return LORDBA_ECUDA;
                 prm.slots = slots;
                 const dim3 grid((unsigned)tiles, (unsigned)m, (unsigned)splits);
                 cudaError_t e;
-                switch (rp) {
-                    case 8:  e = launch_one<8>(b, prm, grid, plan.total, stream); break;
-                    case 16: e = launch_one<16>(b, prm, grid, plan.total, stream); break;
-                    case 32: e = launch_one<32>(b, prm, grid, plan.total, stream); break;
-                    default: e = launch_one<64>(b, prm, grid, plan.total, stream); break;
+                if (nw == kMaxWarps) {
+                    switch (rp) {
+                        case 8:  e = launch_one<8, 16>(b, prm, grid, plan.total, stream); break;
+                        case 16: e = launch_one<16, 16>(b, prm, grid, plan.total, stream); break;
+                        case 32: e = launch_one<32, 16>(b, prm, grid, plan.total, stream); break;
+                        default: e = launch_one<64, 16>(b, prm, grid, plan.total, stream); break;
+                    }
+                } else {
+                    switch (rp) {
+                        case 8:  e = launch_one<8, 8>(b, prm, grid, plan.total, stream); break;
+                        case 16: e = launch_one<16, 8>(b, prm, grid, plan.total, stream); break;
+                        case 32: e = launch_one<32, 8>(b, prm, grid, plan.total, stream); break;
+                        default: e = launch_one<64, 8>(b, prm, grid, plan.total, stream); break;
+                    }
                 }
                 if (e != cudaSuccess) return LORDBA_ECUDA;
                 count_launch();

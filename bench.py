@@ -195,7 +195,7 @@ def run_gpu(args):
     x_host = to_bf16(p.x).pin_memory()
     y_host = to_bf16(p.y).pin_memory()
     set_bytes = (T * D_IN + T * D_OUT) * ELEM
-    n_sets = int(np.ceil(4 * L2_BYTES / set_bytes))
+    n_sets = int(np.ceil(8 * L2_BYTES / set_bytes))
     xs = [x_host.to(dev) for _ in range(n_sets)]
     ys = [y_host.to(dev) for _ in range(n_sets)]
     packed_A = lordba.pack_signs(torch.from_numpy(p.A_sign).to(dev), 0)
@@ -320,7 +320,7 @@ def run_gpu(args):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "config1: LLaMA-2-7B attention projection adapter, d_in=d_out=4096, "
                                    "r=16, T=2048 tokens per GPU per step, bf16 x/y, fp32 scales",
-                       "l2": "steps rotate through %d device buffer sets (%.0f MB > 4 x L2)"
+                       "l2": "steps rotate through %d device buffer sets (%.0f MB > 8 x L2)"
                              % (n_sets, n_sets * set_bytes / 1e6),
                        "launch": "CUDA graph of %d steps replayed" % n_sets,
                        "step_dependency": "every step waits for the previous one" if args.no_overlap else
@@ -347,6 +347,111 @@ def run_gpu(args):
     return 0
 
 
+# ----------------------------------------------------------------------------- other workloads
+
+def run_workload(args):
+    """The other configurations (single GPU, device-generated inputs, no oracle leg): one step =
+    ONE library call, single or batched.  Prints the same kind of JSON line; parity of these shapes
+    is covered by the GPU tests, not here."""
+    import torch
+    from paper_2605_24058_b200 import lordba
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    lordba.load()
+    r, Tn = args.rank, args.tokens
+    H, F = workloads.HIDDEN, workloads.FFN
+    layer = [(di, do) for _, di, do in workloads.LAYER_PROJECTIONS]
+    shapes = {"gate": [(H, F)], "down": [(F, H)], "layer": layer, "decode": layer,
+              "full": layer * workloads.N_LAYERS}[args.workload]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234)
+
+    def rand_signs(rows, cols):
+        return (torch.randint(0, 2, (rows, cols), device=dev, generator=gen, dtype=torch.int8) * 2 - 1)
+
+    adapters = []
+    for di, do in shapes:
+        adapters.append(dict(
+            pa=lordba.pack_signs(rand_signs(r, di), 0), pb=lordba.pack_signs(rand_signs(do, r), 1),
+            s_in=torch.exp(0.5 * torch.randn(di, device=dev, generator=gen)),
+            s_r=64.0 * (0.02 * torch.randn(r, device=dev, generator=gen)).abs(),
+            s_out=torch.exp(0.5 * torch.randn(do, device=dev, generator=gen))))
+    set_bytes = sum(Tn * (di + do) * ELEM for di, do in shapes)
+    alg_bytes = sum(workloads.algorithmic_bytes(Tn, di, do, r, ELEM) for di, do in shapes)
+    n_sets = int(max(1, min(np.ceil(8 * L2_BYTES / set_bytes), 40e9 // set_bytes)))
+    if set_bytes > 2 * L2_BYTES:
+        n_sets = 1                       # one set already exceeds the L2: every step re-reads it from DRAM
+    sets = []
+    for _ in range(n_sets):
+        sets.append([(torch.randn(Tn, di, device=dev, generator=gen, dtype=torch.float32).to(torch.bfloat16),
+                      torch.randn(Tn, do, device=dev, generator=gen, dtype=torch.float32).to(torch.bfloat16))
+                     for di, do in shapes])
+    overlap_ok = n_sets > 1 and not args.no_overlap
+
+    def step(i):
+        flags = lordba.PROJ_OVERLAP if (overlap_ok and i % n_sets != 0) else 0
+        bufs = sets[i % n_sets]
+        projs = [lordba.make_proj(x, a["pa"], a["pb"], a["s_in"], a["s_r"], a["s_out"], y, r, flags)
+                 for (x, y), a in zip(bufs, adapters)]
+        if len(projs) == 1:
+            lordba.adapter_forward_ex(projs[0], Tn, lordba.BF16)
+        else:
+            lordba.adapter_forward_batched(projs, Tn, lordba.BF16)
+
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        n_graph = max(n_sets, 4)
+        for i in range(n_graph):
+            step(i)
+        stream.synchronize()
+        n0 = lordba.launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(n_graph):
+                step(i)
+        launches_per_step = (lordba.launch_count() - n0) / n_graph
+        reps_w, reps = max(1, args.warmup // n_graph), max(1, args.steps // n_graph)
+        sampler = ClockSampler(0)
+        sampler.start()
+        for _ in range(reps_w):
+            graph.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.recording = True
+        e0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+        sampler.recording = False
+        sampler.stop()
+    steps = reps * n_graph
+    ms = e0.elapsed_time(e1)
+    if lordba.device_status() != 0:
+        raise RuntimeError("device status word set")
+    peak, peak_kind = measured_peak()
+    achieved = alg_bytes / (ms * 1e-3 / steps) / 1e9
+    line = {
+        "metric": "adapter-branch tokens/s, workload %s (r=%d, T=%d, %d projection(s) per call)"
+                  % (args.workload, r, Tn, len(shapes)),
+        "value": Tn * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
+        "warmup": reps_w * n_graph, "ms_per_step": ms / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "projections": len(shapes), "rank": r, "tokens": Tn,
+                   "l2": "%d buffer set(s) of %.0f MB" % (n_sets, set_bytes / 1e6),
+                   "launch": "CUDA graph of %d steps replayed" % n_graph,
+                   "step_dependency": "declared independent" if overlap_ok else "each step waits for the previous one"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_kind": "of " + peak_kind,
+                     "algorithmic_bytes_per_launch": alg_bytes},
+        "e2e": None, "gpu_launches": int(round(launches_per_step * steps)), "clocks": sampler.summary(),
+    }
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -358,12 +463,20 @@ def main():
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch to report in roofline.traffic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full"],
+                    help="attn = the headline configuration (default); the others are supplementary: one "
+                         "MLP projection, a layer's seven projections in one batched call (prefill, or "
+                         "decode with --tokens 1..64), or all 224 projections in one call")
+    ap.add_argument("--rank", type=int, default=R)
+    ap.add_argument("--tokens", type=int, default=T)
     ap.add_argument("--no-overlap", action="store_true",
                     help="every step waits for the previous one to finish (no LORDBA_PROJ_OVERLAP)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload != "attn":
+        return run_workload(args)
     return run_gpu(args)
 
 

@@ -215,24 +215,29 @@ def run_gpu(args):
     parity = None
     if rank == 0:
         import oracle
+        # both launch shapes that the timed region uses: step 0 (waits for its predecessor) and
+        # step 1 (declared independent: the two-CTA-per-SM kernel)
         step(0)
+        step(1)
         torch.cuda.synchronize()
-        rows = np.array([0, 1, 127, 128, 1000, 2047])
-        got = ys[0][torch.from_numpy(rows).to(dev)].to(torch.float64).cpu().numpy()
+        rows = np.array([0, 1, 13, 14, 127, 128, 1000, 2047])
         f8 = np.float64
         want = oracle.adapter_forward(p.x_f64()[rows], p.A_sign, p.B_sign, p.s_in.astype(f8),
                                       p.s_r.astype(f8), p.s_out.astype(f8), p.y_f64()[rows])
         rms = float(np.sqrt(np.mean(want * want)))
-        err = np.abs(got - want)
-        # 2e-2 rms(y') as stated where the bf16 output rounding (<= 2^-8 |y'|) fits inside it,
-        # and rounding + 2^-12 rms(y') everywhere
-        region = np.abs(want) <= 5.0 * rms
-        parity = float(err[region].max() / rms)
-        tight_ok = bool((err <= 2.0 ** -8 * np.abs(want) + 2.0 ** -12 * rms).all())
-        if not (parity <= 2e-2 and tight_ok):
-            raise RuntimeError("bench configuration fails parity: max err / rms = %g, rounding "
-                               "bound held: %s" % (parity, tight_ok))
-        ys[0].copy_(y_host)
+        parity = 0.0
+        for k in (0, 1):
+            got = ys[k][torch.from_numpy(rows).to(dev)].to(torch.float64).cpu().numpy()
+            err = np.abs(got - want)
+            # 2e-2 rms(y') as stated where the bf16 output rounding (<= 2^-8 |y'|) fits inside it,
+            # and rounding + 2^-12 rms(y') everywhere
+            region = np.abs(want) <= 5.0 * rms
+            parity = max(parity, float(err[region].max() / rms))
+            tight_ok = bool((err <= 2.0 ** -8 * np.abs(want) + 2.0 ** -12 * rms).all())
+            if not (parity <= 2e-2 and tight_ok):
+                raise RuntimeError("bench configuration fails parity (step %d): max err / rms = %g, "
+                                   "rounding bound held: %s" % (k, parity, tight_ok))
+            ys[k].copy_(y_host)
 
     # one CUDA graph holds n_sets consecutive steps (one per buffer set): launches are then
     # issued faster than the ~10 us kernels retire.

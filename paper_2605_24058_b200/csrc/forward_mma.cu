@@ -207,7 +207,7 @@ __device__ __forceinline__ void consumer_sync()
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
                  "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
@@ -398,27 +398,31 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     lB[p] = __shfl_sync(0xffffffffu, pl, 8 * q + 4 + p);
                 }
                 const uint2 *blk = reinterpret_cast<const uint2 *>(slot + plan.off_bits) + warp * r;
+                uint32_t bytes[R8];                                  // sign bytes of this lane's 16 columns
 #pragma unroll
                 for (int a = 0; a < R8; ++a) {
                     int k = 8 * a + g;
                     if (k > r - 1) k = r - 1;                       // padded rank rows: result unused
                     const uint2 sb = blk[k];                         // the row's 64 sign bits of this block
-                    const uint32_t w16 = ((q & 2) ? sb.y : sb.x) >> (16 * (q & 1));
-                    const uint32_t bA = w16 & 0xffu, bB = (w16 >> 8) & 0xffu;
-                    float(&ch)[4] = acc[0][a];
-                    float(&cl)[4] = acc[kSplitAcc ? 1 : 0][a];
-                    uint32_t m0 = pair_bits(bA, 0), m1 = pair_bits(bA, 1);
-                    mma_bf16(ch, xa0.x, xa1.x, xa0.y, xa1.y, with_signs(hA[0], m0), with_signs(hA[1], m1));
-                    mma_bf16(cl, xa0.x, xa1.x, xa0.y, xa1.y, with_signs(lA[0], m0), with_signs(lA[1], m1));
-                    m0 = pair_bits(bA, 2); m1 = pair_bits(bA, 3);
-                    mma_bf16(ch, xa0.z, xa1.z, xa0.w, xa1.w, with_signs(hA[2], m0), with_signs(hA[3], m1));
-                    mma_bf16(cl, xa0.z, xa1.z, xa0.w, xa1.w, with_signs(lA[2], m0), with_signs(lA[3], m1));
-                    m0 = pair_bits(bB, 0); m1 = pair_bits(bB, 1);
-                    mma_bf16(ch, xb0.x, xb1.x, xb0.y, xb1.y, with_signs(hB[0], m0), with_signs(hB[1], m1));
-                    mma_bf16(cl, xb0.x, xb1.x, xb0.y, xb1.y, with_signs(lB[0], m0), with_signs(lB[1], m1));
-                    m0 = pair_bits(bB, 2); m1 = pair_bits(bB, 3);
-                    mma_bf16(ch, xb0.z, xb1.z, xb0.w, xb1.w, with_signs(hB[2], m0), with_signs(hB[3], m1));
-                    mma_bf16(cl, xb0.z, xb1.z, xb0.w, xb1.w, with_signs(lB[2], m0), with_signs(lB[3], m1));
+                    bytes[a] = (((q & 2) ? sb.y : sb.x) >> (16 * (q & 1))) & 0xffffu;
+                }
+                // k-step outermost, rank blocks innermost: consecutive MMAs go to different
+                // accumulators, so none waits for the one before it
+                const uint32_t xk[4][4] = {{xa0.x, xa1.x, xa0.y, xa1.y}, {xa0.z, xa1.z, xa0.w, xa1.w},
+                                           {xb0.x, xb1.x, xb0.y, xb1.y}, {xb0.z, xb1.z, xb0.w, xb1.w}};
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint32_t h0 = (ks < 2) ? hA[2 * ks] : hB[2 * ks - 4], h1 = (ks < 2) ? hA[2 * ks + 1] : hB[2 * ks - 3];
+                    const uint32_t l0 = (ks < 2) ? lA[2 * ks] : lB[2 * ks - 4], l1 = (ks < 2) ? lA[2 * ks + 1] : lB[2 * ks - 3];
+#pragma unroll
+                    for (int a = 0; a < R8; ++a) {
+                        const uint32_t b = (ks < 2) ? (bytes[a] & 0xffu) : (bytes[a] >> 8);
+                        const uint32_t m0 = pair_bits(b, 2 * (ks & 1)), m1 = pair_bits(b, 2 * (ks & 1) + 1);
+                        mma_bf16(acc[0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                 with_signs(h0, m0), with_signs(h1, m1));
+                        mma_bf16(acc[kSplitAcc ? 1 : 0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                 with_signs(l0, m0), with_signs(l1, m1));
+                    }
                 }
             }
             __syncwarp();
@@ -496,6 +500,9 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
 #pragma unroll
                     for (int e = 0; e < 4; ++e) c[i][e] = 0.0f;
                 const int jb = gcol + 16 * (g >> 1) + (g & 1);
+                // the r sign bits of this lane's 8 B_sign rows, shifted so that k-step ks reads its
+                // 4 bits at bit 16 ks
+                uint64_t rb[8];
                 if (RP == 16) {
                     // rows jb - (g&1) .. + 15 are 16 half-words: word i holds rows 2i (low) and 2i+1
                     const uint4 w0 = *reinterpret_cast<const uint4 *>(bits + 2 * (jb - (g & 1)));
@@ -503,26 +510,27 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
                     const int sh = 16 * (g & 1) + 4 * q;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const uint32_t nib = (w[i] >> sh) & 0xfu;
-                        const uint32_t b0 = with_signs(0x3f803f80u, nib * 0x40008000u);
-                        const uint32_t b1 = with_signs(0x3f803f80u, nib * 0x10002000u);
-                        mma_bf16(c[i], zh[0][0], zh[0][1], zh[0][2], zh[0][3], b0, b1);
-                        mma_bf16(c[i], zl[0][0], zl[0][1], zl[0][2], zl[0][3], b0, b1);
-                    }
+                    for (int i = 0; i < 8; ++i) rb[i] = w[i] >> sh;
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const uint64_t rb = b_row_bits<RP>(bits, jb + 2 * i, r);
+                    for (int i = 0; i < 8; ++i) rb[i] = b_row_bits<RP>(bits, jb + 2 * i, r) >> (4 * q);
+                }
+                // k-step outermost, n-blocks innermost: consecutive MMAs go to different accumulators
 #pragma unroll
-                        for (int ks = 0; ks < KS; ++ks) {
-                            const uint32_t nib = (uint32_t)(rb >> (16 * ks + 4 * q)) & 0xfu;
-                            const uint32_t b0 = with_signs(0x3f803f80u, nib * 0x40008000u);
-                            const uint32_t b1 = with_signs(0x3f803f80u, nib * 0x10002000u);
-                            mma_bf16(c[i], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b0, b1);
-                            mma_bf16(c[i], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b0, b1);
-                        }
+                for (int ks = 0; ks < KS; ++ks) {
+                    uint32_t b0[8], b1[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t nib = (uint32_t)(rb[i] >> (16 * ks)) & 0xfu;
+                        b0[i] = with_signs(0x3f803f80u, nib * 0x40008000u);
+                        b1[i] = with_signs(0x3f803f80u, nib * 0x10002000u);
                     }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        mma_bf16(c[i], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b0[i], b1[i]);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        mma_bf16(c[i], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b0[i], b1[i]);
                 }
                 const float4 *so4 = reinterpret_cast<const float4 *>(slot + plan.off_scale + 4 * (gcol + 16 * q));
                 float so[16];

@@ -364,6 +364,8 @@ def run_workload(args):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
     lordba.load()
+    if args.variant is not None:
+        lordba.set_variant({"auto": 0, "fma": 1, "tc": 2, "mma": 3}[args.variant])
     r, Tn = args.rank, args.tokens
     H, F = workloads.HIDDEN, workloads.FFN
     layer = [(di, do) for _, di, do in workloads.LAYER_PROJECTIONS]

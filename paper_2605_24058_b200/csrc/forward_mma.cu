@@ -11,15 +11,18 @@
 //     the tiles of a call fill the SMs evenly) and needs no other CTA: the
 //     16 x r intermediate lives in registers and shared memory.
 //   * A producer warp streams the CTA's rows of x, then of y, through a ring of
-//     shared-memory slots, 1024 columns per item, with ONE tensor copy per item:
-//     the row-major matrix is described to TMA as a 3-D tensor (64 columns,
-//     rows, column groups), so a box of 64 x 16 x 16 lands as sixteen 2 KiB
-//     blocks [16 rows][128 bytes], 128-byte swizzled, one block per consumer
-//     warp.  The item's slice of the scale vector and of the packed carrier
+//     shared-memory slots, NW x 64 columns per item (NW = consumer warps), with
+//     ONE tensor copy per item: the row-major matrix is described to TMA as a
+//     3-D tensor (64 columns, rows, column groups), so a box of 64 x 16 x NW
+//     lands as NW blocks of 2 KiB, [16 rows][128 bytes], 128-byte swizzled, one
+//     block per consumer warp.  The item's slice of the scale vector and of the packed carrier
 //     travels in the same slot (two small 2-D tensor copies), so there are no
 //     other global loads.  The y items are requested while the first product is
 //     still running: the memory system never drains between the two products.
-//   * Sixteen consumer warps each take one 64-column group of an item.  A lane
+//   * The NW consumer warps each take one 64-column group of an item.  NW = 16
+//     with one CTA per SM for a lone call of a single wave of tiles; NW = 8 with
+//     two CTAs per SM otherwise, so that one CTA's start-up and first-load
+//     latency hide behind the other's streaming.  A lane
 //     reads 16-byte pieces of two token rows from the slot straight into the
 //     registers that are the A fragments of mma.sync.m16n8k16 (the K order of a
 //     product is free, so the fragment's column pattern is re-labelled to make

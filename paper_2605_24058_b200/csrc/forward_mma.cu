@@ -35,7 +35,8 @@
 //     s_in (as a bf16 hi/lo pair) with the signs XOR-ed in; a B fragment of the
 //     second product is +-1.0.  s_in and z = s_r * u are split into bf16 hi + lo
 //     parts, so both products carry ~16 mantissa bits into the float32
-//     accumulators.
+//     accumulators.  MMAs are issued k-step outermost, so that consecutive
+//     ones go to different accumulators.
 //
 // Warps split the d_in axis for the first product (fixed-order reduction
 // through shared memory, hence deterministic) and the d_out axis for the

@@ -44,6 +44,10 @@ T = 2048
 ELEM = 2
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel on this workload
+# (ncu capture summarised under profiles/; reads only, the write-back L2 defers the y writes past
+# the end of the kernel).  Set to None whenever the kernel changes after the capture.
+NCU_DRAM_BYTES_PER_LAUNCH = 33634304
 
 
 def measured_peak():
@@ -467,7 +471,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default=None, choices=["auto", "fma", "tc", "mma"],
                     help="pin the kernel family (default: the library's own choice)")
-    ap.add_argument("--traffic", type=float, default=None,
+    ap.add_argument("--traffic", type=float, default=NCU_DRAM_BYTES_PER_LAUNCH,
                     help="ncu DRAM bytes per launch to report in roofline.traffic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full"],

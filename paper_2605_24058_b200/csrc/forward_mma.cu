@@ -52,6 +52,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include "lordba_internal.h"
 
@@ -60,6 +61,7 @@ namespace {
 
 // Consumer warps per CTA (template parameter NW): 16 with one CTA per SM, or 8 with two CTAs per
 // SM, so that one CTA's start-up and first-load latency hide behind the other's streaming.
+// (Three CTAs per SM at 72 registers were measured slower: fewer slots per ring.)
 constexpr int kTile = 16;            // token rows of one MMA tile = rows of a TMA box
 constexpr int kGroup = 64;           // columns one warp handles per item (128 bytes per row)
 constexpr int kBlockBytes = kTile * kGroup * 2;      // one warp's block of a slot: 2 KiB
@@ -498,15 +500,11 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 // Output column of n-block i, accumulator column n = 2q + e: gcol + 16q + 2i + e, so
                 // that a lane owns 16 consecutive columns.  As the holder of B-fragment column
                 // n = g this lane expands the signs of j = gcol + 16(g>>1) + 2i + (g&1).
-                float c[8][4];
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) c[i][e] = 0.0f;
                 const int jb = gcol + 16 * (g >> 1) + (g & 1);
                 // the r sign bits of this lane's 8 B_sign rows, shifted so that k-step ks reads its
                 // 4 bits at bit 16 ks
-                uint64_t rb[8];
+                typedef typename std::conditional<(RP > 32), uint64_t, uint32_t>::type bits_t;
+                bits_t rb[8];
                 if (RP == 16) {
                     // rows jb - (g&1) .. + 15 are 16 half-words: word i holds rows 2i (low) and 2i+1
                     const uint4 w0 = *reinterpret_cast<const uint4 *>(bits + 2 * (jb - (g & 1)));
@@ -514,51 +512,60 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
                     const int sh = 16 * (g & 1) + 4 * q;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) rb[i] = w[i] >> sh;
+                    for (int i = 0; i < 8; ++i) rb[i] = (bits_t)(w[i] >> sh);
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) rb[i] = b_row_bits<RP>(bits, jb + 2 * i, r) >> (4 * q);
+                    for (int i = 0; i < 8; ++i) rb[i] = (bits_t)(b_row_bits<RP>(bits, jb + 2 * i, r) >> (4 * q));
                 }
-                // k-step outermost, n-blocks innermost: consecutive MMAs go to different accumulators
+                // The lane's 16 columns are done as two halves of 8 (n-blocks 4cc .. 4cc+3) to keep
+                // the live registers low; the results of both halves leave in one 256-bit store.
+                uint32_t out[2][8];
 #pragma unroll
-                for (int ks = 0; ks < KS; ++ks) {
-                    uint32_t b0[8], b1[8];
+                for (int cc = 0; cc < 2; ++cc) {
+                    float c[4][4];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const uint32_t nib = (uint32_t)(rb[i] >> (16 * ks)) & 0xfu;
-                        b0[i] = with_signs(0x3f803f80u, nib * 0x40008000u);
-                        b1[i] = with_signs(0x3f803f80u, nib * 0x10002000u);
+                    for (int i = 0; i < 4; ++i)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) c[i][e] = 0.0f;
+                    // k-step outermost, n-blocks innermost: consecutive MMAs go to different accumulators
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        uint32_t b0[4], b1[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t nib = (uint32_t)(rb[4 * cc + i] >> (16 * ks)) & 0xfu;
+                            b0[i] = with_signs(0x3f803f80u, nib * 0x40008000u);
+                            b1[i] = with_signs(0x3f803f80u, nib * 0x10002000u);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            mma_bf16(c[i], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b0[i], b1[i]);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            mma_bf16(c[i], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b0[i], b1[i]);
                     }
+                    const float4 *so4 = reinterpret_cast<const float4 *>(slot + plan.off_scale + 4 * (gcol + 16 * q + 8 * cc));
+                    const float4 s0 = so4[0], s1 = so4[1];
+                    const float so[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        mma_bf16(c[i], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b0[i], b1[i]);
+                    for (int half = 0; half < 2; ++half) {              // token rows g and g + 8
+                        const uint4 yv = *reinterpret_cast<const uint4 *>(slot + (half == 0 ? off_r0 : off_r1) +
+                                                                           (cc == 0 ? pc0 : pc1));
+                        const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        mma_bf16(c[i], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b0[i], b1[i]);
-                }
-                const float4 *so4 = reinterpret_cast<const float4 *>(slot + plan.off_scale + 4 * (gcol + 16 * q));
-                float so[16];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float4 t = so4[i];
-                    so[4 * i] = t.x; so[4 * i + 1] = t.y; so[4 * i + 2] = t.z; so[4 * i + 3] = t.w;
-                }
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {                  // token rows g and g + 8
-                    if (half == 0 ? v0 : v1) {
-                        const int off = half == 0 ? off_r0 : off_r1;
-                        const uint4 ya = *reinterpret_cast<const uint4 *>(slot + off + pc0);
-                        const uint4 yb = *reinterpret_cast<const uint4 *>(slot + off + pc1);
-                        const uint32_t yw[8] = {ya.x, ya.y, ya.z, ya.w, yb.x, yb.y, yb.z, yb.w};
-                        uint32_t oa[4], ob[4];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
+                        for (int i = 0; i < 4; ++i) {
                             const float o0 = fmaf(so[2 * i], c[i][2 * half], lo_f(yw[i]));
                             const float o1 = fmaf(so[2 * i + 1], c[i][2 * half + 1], hi_f(yw[i]));
-                            if (i < 4) oa[i] = pack2(o0, o1);
-                            else ob[i - 4] = pack2(o0, o1);
+                            out[half][4 * cc + i] = pack2(o0, o1);
                         }
+                    }
+                }
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    if (half == 0 ? v0 : v1) {
                         __nv_bfloat16 *dst = (half == 0 ? yrow0 : yrow1) + col0 + gcol + 16 * q;
+                        const uint32_t oa[4] = {out[half][0], out[half][1], out[half][2], out[half][3]};
+                        const uint32_t ob[4] = {out[half][4], out[half][5], out[half][6], out[half][7]};
                         if (vec32) {
                             st_global_256(dst, oa, ob);
                         } else {

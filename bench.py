@@ -174,6 +174,23 @@ def run_reference(args):
 
 # ----------------------------------------------------------------------------- GPU arm
 
+def max_over_ranks(values, device=None):
+    """The slowest rank's timings: element-wise MAX over the ranks of the default process group
+    (values unchanged when no group is initialised).  Every rank gets the same list back."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def aggregate_tokens_per_s(world, tokens_per_rank_step, steps, ms):
+    """Whole-job throughput: what all ranks processed divided by the slowest rank's time."""
+    return world * tokens_per_rank_step * steps / (ms * 1e-3)
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -311,10 +328,7 @@ def run_gpu(args):
     if status != 0:
         raise RuntimeError("device status word is %d after the timed region" % status)
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], dev if world > 1 else None)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -323,7 +337,7 @@ def run_gpu(args):
         achieved = alg_bytes / sec_per_step / 1e9
         variant = {0: "auto", 1: "fma", 2: "tc", 3: "mma"}[lordba.get_variant()]
         line = {
-            "metric": METRIC, "value": world * T * args.steps / (ms * 1e-3), "unit": UNIT,
+            "metric": METRIC, "value": aggregate_tokens_per_s(world, T, args.steps, ms), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",

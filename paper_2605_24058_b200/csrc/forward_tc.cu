@@ -43,7 +43,7 @@ namespace {
 
 constexpr int kTileM = 128;             // MMA M = TMEM lanes; a tile holds tile_rows <= 128 tokens
 constexpr int kChunk = 64;              // columns per TMA box (128 bytes of bf16)
-constexpr int kGenThreads = 128;          // warps 2-5
+constexpr int kGenThreads = 256;          // warps 2-9
 constexpr int kEpiThreads = 256;          // warps 6-13
 constexpr int kThreads = 64 + kGenThreads + kEpiThreads;
 constexpr int kMaxTcBatch = 24;
@@ -220,7 +220,7 @@ __device__ __forceinline__ bool mbar_wait(const WaitCtx &w, uint32_t bar, uint32
 
 __device__ __forceinline__ void fence_proxy_async()
 {
-    asm volatile("fence.proxy.async;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }

@@ -73,8 +73,19 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t
         if (variant == LORDBA_VARIANT_TC || variant == LORDBA_VARIANT_MMA) return LORDBA_EUNSUPPORTED;
         return launch_forward_fma(projs, n, T, dtype, stream);
     }
-    // Split the list: what the chosen tensor-core kernel can take, and the rest.
-    const bool use_tc = (variant == LORDBA_VARIANT_TC);
+    // Split the list: what the chosen tensor-core kernel can take, and the rest.  Left to itself
+    // the library takes the tcgen05 kernel where it was measured ahead of the streaming one: ranks
+    // above 32 with at least two waves of full 128-token tiles.
+    bool use_tc = (variant == LORDBA_VARIANT_TC);
+    if (variant == LORDBA_VARIANT_AUTO) {
+        int64_t big_rank_tiles = 0;
+        bool all_big = n > 0;
+        for (int i = 0; i < n; ++i) {
+            all_big = all_big && projs[i].r > 32 && tc_supported(projs[i], T, dtype);
+            big_rank_tiles += T / 128;
+        }
+        use_tc = all_big && big_rank_tiles >= 2 * 148;
+    }
     std::vector<lordba_proj> fast, fma;
     for (int i = 0; i < n; ++i) {
         const bool ok = use_tc ? tc_supported(projs[i], T, dtype) : mma_supported(projs[i], T, dtype);

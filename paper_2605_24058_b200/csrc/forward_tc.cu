@@ -845,6 +845,15 @@ bool choose_shape(int r, int kp, int n_proj, int64_t T, int min_chunks, LaunchSh
     const int forced_rows = env_int("LORDBA_TC_ROWS", 0);
     double best_cost = 1e300;
     bool found = false;
+    // Plenty of full-height tiles (two waves or more): no cluster, nothing to exchange.
+    if (forced_c == 0 && forced_rows == 0) {
+        LaunchShape solo;
+        const int64_t full_tiles = (int64_t)n_proj * ((T + kTileM - 1) / kTileM);
+        if (plan_launch(r, kp, 1, kTileM, &solo) && full_tiles >= 2 * (int64_t)solo.max_clusters) {
+            *best = solo;
+            return true;
+        }
+    }
     for (int c = 8; c >= 1; c /= 2) {
         if (c > min_chunks) continue;
         if (forced_c >= 1 && forced_c <= 8 && c != forced_c && c * 2 <= min_chunks) continue;

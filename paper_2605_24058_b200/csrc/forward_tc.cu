@@ -43,7 +43,9 @@ namespace {
 
 constexpr int kTileM = 128;             // MMA M = TMEM lanes; a tile holds tile_rows <= 128 tokens
 constexpr int kChunk = 64;              // columns per TMA box (128 bytes of bf16)
-constexpr int kGenThreads = 256;          // warps 2-9
+constexpr int kGenGroupThreads = 128;      // one generator group: four warps
+constexpr int kGenGroups = 2;             // the groups take alternate chunks, so two operands are in the making
+constexpr int kGenThreads = kGenGroups * kGenGroupThreads;   // warps 2-9
 constexpr int kEpiThreads = 256;          // warps 6-13
 constexpr int kThreads = 64 + kGenThreads + kEpiThreads;
 constexpr int kMaxTcBatch = 24;
@@ -81,9 +83,12 @@ struct TcBatch {
 };
 
 // ---- shared-memory plan (offsets from a 1024-byte aligned base), same on host and device ----
+constexpr int kOps = 3;    // operand buffers (generated W1 / W2 tiles), a ring of their own
+
 struct SmemPlan {
     int slot_data;          // bytes reserved for the x / y box of a slot (multiple of 1024)
-    int slot_stride, aux_op_bytes;
+    int slot_stride;        // + the slot's raw scale values and sign bytes
+    int op_bytes, off_ops;  // one generated operand tile; start of the operand ring
     int off_zhi, off_zlo, z_bytes;
     int off_rx, off_lut, off_bar, off_misc, total;
 };
@@ -100,20 +105,24 @@ __host__ __device__ inline int aux_operand_bytes(int r, int kp)
 __host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile_rows)
 {
     SmemPlan s;
-    s.aux_op_bytes = aux_operand_bytes(r, kp);
     // The MMA reads 128 rows (16 KiB) from the start of a slot whatever tile_rows is; what lies
-    // beyond the box (this slot's operand area, the next slot) only reaches accumulator rows that
+    // beyond the box (this slot's raw area, the next slot) only reaches accumulator rows that
     // nobody reads.  `total` is padded so that this read stays inside the allocation.
     s.slot_data = round_up(tile_rows * kChunk * 2, 1024);
-    // behind the operand: 256 B of raw scale values and up to 512 B of raw sign bytes
-    s.slot_stride = s.slot_data + round_up(s.aux_op_bytes + 256 + 8 * kMaxRank, 1024);
+    // behind the box: 256 B of raw scale values and up to 512 B of raw sign bytes
+    s.slot_stride = s.slot_data + round_up(256 + 8 * kMaxRank, 1024);
+    // The generated operands live in a short ring of their own (the MMA is done with one within
+    // a microsecond), so that the data ring can be deep enough to cover the load latency at
+    // any rank.
+    s.op_bytes = round_up(aux_operand_bytes(r, kp), 1024);
+    s.off_ops = slots * s.slot_stride;
     s.z_bytes = (kTileM / 8) * (kp / 8) * 128;
-    s.off_zhi = slots * s.slot_stride;
+    s.off_zhi = s.off_ops + kOps * s.op_bytes;
     s.off_zlo = s.off_zhi + s.z_bytes;
     s.off_rx = s.off_zlo + s.z_bytes;
     s.off_lut = s.off_rx + kTileM * r * 4;
     s.off_bar = s.off_lut + 4096;
-    s.off_misc = s.off_bar + (3 * slots + 8) * 8;
+    s.off_misc = s.off_bar + (3 * slots + 2 * kOps + 8) * 8;
     s.total = s.off_misc + 16;
     const int last_read_end = (slots - 1) * s.slot_stride + kTileM * kChunk * 2;
     if (s.total < last_read_end) s.total = last_read_end;
@@ -344,6 +353,8 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     const uint32_t bar_rx_full = bar0 + 8u * (3 * S + 2);
     auto bar_v_full = [&](int b) { return bar0 + 8u * (3 * S + 3 + b); };
     auto bar_v_empty = [&](int b) { return bar0 + 8u * (3 * S + 5 + b); };
+    auto bar_op_full = [&](int o) { return bar0 + 8u * (3 * S + 8 + o); };           // operand tile generated
+    auto bar_op_empty = [&](int o) { return bar0 + 8u * (3 * S + 8 + kOps + o); };   // MMAs that read it are done
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + plan.off_misc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + plan.off_misc + 4);
     const WaitCtx wctx{abort_flag, B.status};
@@ -355,9 +366,13 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     // ---- one-time setup ---------------------------------------------------------------------
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(bar_full(s), 1 + kGenThreads);   // producer's expect_tx arrive + generator threads
+            mbar_init(bar_full(s), 1);                 // the producer's expect_tx arrive
             mbar_init(bar_empty(s), 1);
             mbar_init(bar_raw(s), 1);
+        }
+        for (int o = 0; o < kOps; ++o) {
+            mbar_init(bar_op_full(o), kGenGroupThreads);
+            mbar_init(bar_op_empty(o), 1);
         }
         mbar_init(bar_u_full, 1);
         mbar_init(bar_z_full, (uint32_t)(tile_rows * r8));   // one arrive per (row, 8-wide piece), all owners
@@ -422,7 +437,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     mbar_wait<false>(wctx, bar_empty(s), ph ^ 1u, kDevTmaWaitTimeout);
                     TC_TRACE(0, it, 0);
                     const uint32_t slot = sm_base + s * plan.slot_stride;
-                    const uint32_t rawdst = slot + plan.slot_data + plan.aux_op_bytes;
+                    const uint32_t rawdst = slot + plan.slot_data;
                     if ((c + 1) * kChunk <= P.d_in) {
                         mbar_arrive_expect_tx(bar_raw(s), 256u + sign_bytes);
                         bulk_load(rawdst, P.s_in + (size_t)c * kChunk, 256u, bar_raw(s));
@@ -439,7 +454,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     mbar_wait<false>(wctx, bar_empty(s), ph ^ 1u, kDevTmaWaitTimeout);
                     TC_TRACE(0, it, 0);
                     const uint32_t slot = sm_base + s * plan.slot_stride;
-                    const uint32_t rawdst = slot + plan.slot_data + plan.aux_op_bytes;
+                    const uint32_t rawdst = slot + plan.slot_data;
                     if ((c + 1) * kChunk <= P.d_out) {
                         mbar_arrive_expect_tx(bar_raw(s), 256u + sign_bytes);
                         bulk_load(rawdst, P.s_out + (size_t)c * kChunk, 256u, bar_raw(s));
@@ -459,11 +474,13 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 const uint32_t idesc2 = instr_desc(kTileM, kChunk);
                 for (int c = kb; c < ke; ++c, ++it) {
                     const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                    const int o = it % kOps; const uint32_t oph = (it / kOps) & 1u;
                     mbar_wait<false>(wctx, bar_full(s), ph, kDevMmaWaitTimeout);
+                    mbar_wait<false>(wctx, bar_op_full(o), oph, kDevMmaWaitTimeout);
                     TC_TRACE(1, it, 0);
                     tc_fence_after();
                     const uint32_t a0 = sm_base + s * plan.slot_stride;       // x tile, 128B swizzle
-                    const uint32_t b0 = a0 + plan.slot_data;                  // W1, no swizzle
+                    const uint32_t b0 = sm_base + plan.off_ops + o * plan.op_bytes;   // W1, no swizzle
 #pragma unroll
                     for (int ks = 0; ks < kChunk / 16; ++ks) {
                         const uint64_t ad = smem_desc(a0 + ks * 32, 16, 1024, 2);
@@ -471,6 +488,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                         mma_bf16(tmem_base + kTmemU, ad, bd, idesc1, (c > kb || ks > 0) ? 1u : 0u);
                     }
                     mma_commit(bar_empty(s));
+                    mma_commit(bar_op_empty(o));
                 }
                 mma_commit(bar_u_full);
                 mbar_wait<true>(wctx, bar_z_full, tphase, kDevMmaWaitTimeout);
@@ -480,14 +498,14 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 const uint32_t zhi = sm_base + plan.off_zhi, zlo = sm_base + plan.off_zlo;
                 const uint32_t z_sbo = kt8 * 128;
                 for (int c = nb; c < ne; ++c, ++it, ++vit) {
-                    const int s = it % S; const uint32_t ph = (it / S) & 1u;
                     const int vb = vit & 1u; const uint32_t vph = (vit >> 1) & 1u;
-                    mbar_wait<false>(wctx, bar_full(s), ph, kDevMmaWaitTimeout);
+                    const int o = it % kOps; const uint32_t oph = (it / kOps) & 1u;
+                    mbar_wait<false>(wctx, bar_op_full(o), oph, kDevMmaWaitTimeout);   // the y box is not needed here
                     TC_TRACE(1, it, 0);
                     mbar_wait<false>(wctx, bar_v_empty(vb), vph ^ 1u, kDevMmaWaitTimeout);
                     TC_TRACE(1, it, 1);
                     tc_fence_after();
-                    const uint32_t b0 = sm_base + s * plan.slot_stride + plan.slot_data;   // W2, no swizzle
+                    const uint32_t b0 = sm_base + plan.off_ops + o * plan.op_bytes;   // W2, no swizzle
                     const uint32_t d = tmem_base + kTmemV + vb * kChunk;
                     uint32_t acc = 0;
                     for (int half = 0; half < 2; ++half) {
@@ -500,27 +518,32 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                         }
                     }
                     mma_commit(bar_v_full(vb));
+                    mma_commit(bar_op_empty(o));
                 }
             }
         } else if (warp < 2 + kGenThreads / 32) {
             // ================= operand generators =================
-            const int g = tid - 64;                // 0..kGenThreads-1
+            const int group = (tid - 64) / kGenGroupThreads;    // this thread's generator group
+            const int g = (tid - 64) % kGenGroupThreads;        // 0..kGenGroupThreads-1 within the group
             const int rsub = g & 7;                // row within an 8-row core matrix
             const int cc = (g >> 3) & 7;           // 16-byte chunk (8 columns) within the 64-column box
             const int kg0 = g >> 6;                // first 8-row group handled by this thread (stage 1)
             for (int c = kb; c < ke; ++c, ++it) {
+                if ((int)(it % kGenGroups) != group) continue;
                 const int s = it % S; const uint32_t ph = (it / S) & 1u;
                 mbar_wait<false>(wctx, bar_raw(s), ph, kDevTmaWaitTimeout);
                 if (g == 0) TC_TRACE(2, it, 0);
-                uint8_t *aux = sm + s * plan.slot_stride + plan.slot_data;
-                float *raw_scale = reinterpret_cast<float *>(aux + plan.aux_op_bytes);
-                uint8_t *raw_sign = aux + plan.aux_op_bytes + 256;
+                const int o = it % kOps;
+                mbar_wait<false>(wctx, bar_op_empty(o), ((it / kOps) & 1u) ^ 1u, kDevMmaWaitTimeout);
+                uint8_t *aux = sm + plan.off_ops + o * plan.op_bytes;
+                float *raw_scale = reinterpret_cast<float *>(sm + s * plan.slot_stride + plan.slot_data);
+                uint8_t *raw_sign = reinterpret_cast<uint8_t *>(raw_scale) + 256;
                 if ((c + 1) * kChunk > P.d_in) {
                     // ragged last chunk: guarded loads (the sign block itself is always complete)
                     if (g < kChunk) raw_scale[g] = (c * kChunk + g < P.d_in) ? __ldg(P.s_in + c * kChunk + g) : 0.0f;
-                    for (int w = g; w < 2 * r; w += kGenThreads)
+                    for (int w = g; w < 2 * r; w += kGenGroupThreads)
                         reinterpret_cast<uint32_t *>(raw_sign)[w] = __ldg(P.packed_A + (size_t)c * 2 * r + w);
-                    asm volatile("bar.sync 2, %0;" ::"n"(kGenThreads) : "memory");
+                    asm volatile("bar.sync %0, %1;" ::"r"(2 + group), "n"(kGenGroupThreads) : "memory");
                 }
                 // s_in of this thread's 8 columns, split into bf16 hi + bf16 lo
                 const float4 sa = *reinterpret_cast<const float4 *>(raw_scale + cc * 8);
@@ -534,7 +557,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     lo[p] = pack2_bf16(sv[2 * p] - ah, sv[2 * p + 1] - bh);
                 }
                 uint8_t *w1 = aux;
-                for (int k = kg0 * 8 + rsub; k < r; k += kGenThreads / 8) {
+                for (int k = kg0 * 8 + rsub; k < r; k += kGenGroupThreads / 8) {
                     const uint4 m = lut[raw_sign[k * 8 + cc]];
                     const int row_hi = k, row_lo = r + k;
                     *reinterpret_cast<uint4 *>(w1 + (row_hi >> 3) * 1024 + cc * 128 + (row_hi & 7) * 16) =
@@ -543,28 +566,31 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                         make_uint4(lo[0] ^ m.x, lo[1] ^ m.y, lo[2] ^ m.z, lo[3] ^ m.w);
                 }
                 fence_proxy_async();
-                mbar_arrive(bar_full(s));
+                mbar_arrive(bar_op_full(o));
                 if (g == 0) TC_TRACE(2, it, 1);
             }
             for (int c = nb; c < ne; ++c, ++it) {
+                if ((int)(it % kGenGroups) != group) continue;
                 const int s = it % S; const uint32_t ph = (it / S) & 1u;
                 mbar_wait<false>(wctx, bar_raw(s), ph, kDevTmaWaitTimeout);
                 if (g == 0) TC_TRACE(2, it, 0);
-                uint8_t *aux = sm + s * plan.slot_stride + plan.slot_data;
-                float *raw_scale = reinterpret_cast<float *>(aux + plan.aux_op_bytes);
-                uint8_t *raw_sign = aux + plan.aux_op_bytes + 256;
+                const int o = it % kOps;
+                mbar_wait<false>(wctx, bar_op_empty(o), ((it / kOps) & 1u) ^ 1u, kDevMmaWaitTimeout);
+                uint8_t *aux = sm + plan.off_ops + o * plan.op_bytes;
+                float *raw_scale = reinterpret_cast<float *>(sm + s * plan.slot_stride + plan.slot_data);
+                uint8_t *raw_sign = reinterpret_cast<uint8_t *>(raw_scale) + 256;
                 if ((c + 1) * kChunk > P.d_out) {
                     const int64_t n_words = ((int64_t)P.d_out * r + 31) / 32;
                     if (g < kChunk) raw_scale[g] = (c * kChunk + g < P.d_out) ? __ldg(P.s_out + c * kChunk + g) : 0.0f;
-                    for (int w = g; w < 2 * r; w += kGenThreads) {
+                    for (int w = g; w < 2 * r; w += kGenGroupThreads) {
                         const int64_t gw = (int64_t)c * 2 * r + w;
                         reinterpret_cast<uint32_t *>(raw_sign)[w] = (gw < n_words) ? __ldg(P.packed_B + gw) : 0u;
                     }
-                    asm volatile("bar.sync 2, %0;" ::"n"(kGenThreads) : "memory");
+                    asm volatile("bar.sync %0, %1;" ::"r"(2 + group), "n"(kGenGroupThreads) : "memory");
                 }
                 uint8_t *w2 = aux;
                 // 64 rows x kt8 chunks; task = (row group, chunk, row in group)
-                for (int task = g; task < kChunk * kt8; task += kGenThreads) {
+                for (int task = g; task < kChunk * kt8; task += kGenGroupThreads) {
                     const int rs = task & 7;
                     const int ch = (task >> 3) % kt8;
                     const int row = ((task >> 3) / kt8) * 8 + rs;
@@ -576,7 +602,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     *reinterpret_cast<uint4 *>(w2 + (row >> 3) * (kt8 * 128) + ch * 128 + rs * 16) = v;
                 }
                 fence_proxy_async();
-                mbar_arrive(bar_full(s));
+                mbar_arrive(bar_op_full(o));
                 if (g == 0) TC_TRACE(2, it, 1);
             }
         } else {
@@ -662,7 +688,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 __syncwarp();
                 tc_fence_after();
                 uint8_t *ytile = sm + s * plan.slot_stride;
-                const float *so = reinterpret_cast<const float *>(ytile + plan.slot_data + plan.aux_op_bytes);
+                const float *so = reinterpret_cast<const float *>(ytile + plan.slot_data);
                 if (warp_has_rows) {
                     uint32_t v[32];
                     tmem_ld32(tlane + kTmemV + vb * kChunk + chalf * 32, v);   // warp-collective

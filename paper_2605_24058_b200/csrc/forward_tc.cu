@@ -90,7 +90,7 @@ struct SmemPlan {
     int slot_stride;        // + the slot's raw scale values and sign bytes
     int op_bytes, off_ops;  // one generated operand tile; start of the operand ring
     int off_zhi, off_zlo, z_bytes;
-    int off_rx, off_lut, off_bar, off_misc, total;
+    int off_rx, off_bar, off_misc, total;
 };
 
 __host__ __device__ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
@@ -120,8 +120,7 @@ __host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile
     s.off_zhi = s.off_ops + kOps * s.op_bytes;
     s.off_zlo = s.off_zhi + s.z_bytes;
     s.off_rx = s.off_zlo + s.z_bytes;
-    s.off_lut = s.off_rx + kTileM * r * 4;
-    s.off_bar = s.off_lut + 4096;
+    s.off_bar = s.off_rx + kTileM * r * 4;
     s.off_misc = s.off_bar + (3 * slots + 2 * kOps + 8) * 8;
     s.total = s.off_misc + 16;
     const int last_read_end = (slots - 1) * s.slot_stride + kTileM * kChunk * 2;
@@ -316,6 +315,20 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi)
 }
 __device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
+// 8 sign bits (bit 1 = +1) -> XOR masks over four bf16 pairs (a 0 bit flips the sign).  b times
+// (2^(15-2p) + 2^(30-2p)) is two disjoint shifted copies of the byte that put bit 2p at position
+// 15 and bit 2p+1 at position 31; only those two positions are kept, inverted.  No table: the
+// shared-memory pipe is the busiest unit of this kernel.
+__device__ __forceinline__ uint4 sign_masks(uint32_t b)
+{
+    uint4 m;
+    m.x = ~(b * ((1u << 15) + (1u << 30))) & 0x80008000u;
+    m.y = ~(b * ((1u << 13) + (1u << 28))) & 0x80008000u;
+    m.z = ~(b * ((1u << 11) + (1u << 26))) & 0x80008000u;
+    m.w = ~(b * ((1u << 9) + (1u << 24))) & 0x80008000u;
+    return m;
+}
+
 // balanced contiguous split of n chunks over `parts` CTAs
 __device__ __forceinline__ void split_range(int n, int parts, int idx, int &begin, int &end)
 {
@@ -389,14 +402,6 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                      ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // sign-flip table: byte of 8 sign bits -> four 32-bit XOR masks over bf16 pairs (bit 0 => flip)
-    if (tid < 256) {
-        uint32_t m[4];
-#pragma unroll
-        for (int p = 0; p < 4; ++p)
-            m[p] = (((tid >> (2 * p)) & 1) ? 0u : 0x8000u) | (((tid >> (2 * p + 1)) & 1) ? 0u : 0x80000000u);
-        reinterpret_cast<uint4 *>(sm + plan.off_lut)[tid] = make_uint4(m[0], m[1], m[2], m[3]);
-    }
     // stage-2 A operands start as zeros (K padding beyond r and rows beyond tile_rows stay zero)
     for (int i = tid; i < 2 * plan.z_bytes / 16; i += kThreads)
         reinterpret_cast<uint4 *>(sm + plan.off_zhi)[i] = make_uint4(0, 0, 0, 0);
@@ -408,7 +413,6 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     const uint32_t tmem_base = *tmem_slot;
     if (tid == 0) TC_TRACE(4, 0, 1);
 
-    const uint4 *lut = reinterpret_cast<const uint4 *>(sm + plan.off_lut);
     const int rows_per = tile_rows / C;      // token rows of a tile owned by each CTA of the cluster
 
     // Every role walks the same sequence of (tile, chunk) and derives slot and phase from `it`.
@@ -558,7 +562,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 }
                 uint8_t *w1 = aux;
                 for (int k = kg0 * 8 + rsub; k < r; k += kGenGroupThreads / 8) {
-                    const uint4 m = lut[raw_sign[k * 8 + cc]];
+                    const uint4 m = sign_masks(raw_sign[k * 8 + cc]);
                     const int row_hi = k, row_lo = r + k;
                     *reinterpret_cast<uint4 *>(w1 + (row_hi >> 3) * 1024 + cc * 128 + (row_hi & 7) * 16) =
                         make_uint4(hi[0] ^ m.x, hi[1] ^ m.y, hi[2] ^ m.z, hi[3] ^ m.w);
@@ -596,7 +600,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     const int row = ((task >> 3) / kt8) * 8 + rs;
                     uint4 v = make_uint4(0, 0, 0, 0);
                     if (c * kChunk + row < P.d_out && ch < r8) {
-                        const uint4 m = lut[raw_sign[row * r8 + ch]];
+                        const uint4 m = sign_masks(raw_sign[row * r8 + ch]);
                         v = make_uint4(0x3f803f80u ^ m.x, 0x3f803f80u ^ m.y, 0x3f803f80u ^ m.z, 0x3f803f80u ^ m.w);
                     }
                     *reinterpret_cast<uint4 *>(w2 + (row >> 3) * (kt8 * 128) + ch * 128 + rs * 16) = v;

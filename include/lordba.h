@@ -90,8 +90,19 @@ typedef struct lordba_proj {
     void           *y;          /* [device] T x d_out, pitch ldy, updated in place */
     int64_t d_in, d_out, ldx, ldy;
     int32_t r;
-    int32_t flags;              /* 0 or LORDBA_PROJ_OVERLAP; other bits must be 0 */
+    int32_t flags;              /* LORDBA_PROJ_OVERLAP and / or LORDBA_PROJ_ELL(ell); other bits 0 */
 } lordba_proj;
+
+/*
+ * Multi-envelope adapters (Def. 1 / Eq. 4 with ell > 1): Delta-W is the sum of ell terms that
+ * share the two sign carriers and differ in their scale triples.  A projection made with
+ * LORDBA_PROJ_ELL(ell) in its flags, 1 <= ell <= LORDBA_MAX_ELL, takes s_in as ell x d_in,
+ * s_r as ell x r and s_out as ell x d_out (row-major, envelope e in row e), and the call adds
+ *     sum_e  s_out[e] * ( B_sign ( s_r[e] * ( A_sign ( s_in[e] * x[t,:] ) ) ) )
+ * to y[t,:] with one rounding.  Flags without this field mean ell = 1.
+ */
+#define LORDBA_MAX_ELL 8
+#define LORDBA_PROJ_ELL(ell) ((((ell) - 1) & 0xf) << 8)
 
 /*
  * lordba_proj.flags: a promise by the caller that lets consecutive calls overlap on the GPU.
@@ -138,6 +149,15 @@ int lordba_adapter_forward(const void *x, const uint32_t *packed_A, const uint32
 int lordba_adapter_forward_f32(const float *x, const uint32_t *packed_A, const uint32_t *packed_B,
                                const float *s_in, const float *s_r, const float *s_out, float *y,
                                int64_t T, int64_t d_in, int64_t d_out, int r, void *stream);
+
+/*
+ * Multi-envelope form of the two calls above (Eq. 4, ell >= 1), dense rows: s_in is ell x d_in,
+ * s_r ell x r, s_out ell x d_out.  dtype: LORDBA_BF16 or LORDBA_F32.
+ */
+int lordba_adapter_forward_ell(const void *x, const uint32_t *packed_A, const uint32_t *packed_B,
+                               const float *s_in, const float *s_r, const float *s_out, void *y,
+                               int64_t T, int64_t d_in, int64_t d_out, int r, int ell, int dtype,
+                               void *stream);
 
 /* Same operation with explicit row pitches and dtype.  p: [host]. */
 int lordba_adapter_forward_ex(const lordba_proj *p, int64_t T, int dtype, void *stream);

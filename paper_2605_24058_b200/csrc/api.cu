@@ -47,7 +47,8 @@ int validate_proj(const lordba_proj &p, int64_t T, int dtype)
 {
     if (dtype != LORDBA_F32 && dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
     if (T < 0 || p.d_in < 1 || p.d_out < 1 || p.ldx < p.d_in || p.ldy < p.d_out) return LORDBA_EINVAL;
-    if ((p.flags & ~LORDBA_PROJ_OVERLAP) != 0) return LORDBA_EINVAL;
+    if ((p.flags & ~(LORDBA_PROJ_OVERLAP | 0xf00)) != 0) return LORDBA_EINVAL;
+    if (((p.flags >> 8) & 0xf) + 1 > LORDBA_MAX_ELL) return LORDBA_EUNSUPPORTED;
     if (p.r < 1 || p.r > kMaxRank) return LORDBA_EUNSUPPORTED;
     if (T == 0) return LORDBA_OK;   // nothing is touched: the pointers may be anything
     if (!p.x || !p.packed_A || !p.packed_B || !p.s_in || !p.s_r || !p.s_out || !p.y)
@@ -164,6 +165,17 @@ int lordba_adapter_forward(const void *x, const uint32_t *packed_A, const uint32
 {
     const lordba_proj p = dense_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, d_in, d_out, r);
     return lordba_adapter_forward_ex(&p, T, LORDBA_BF16, stream);
+}
+
+int lordba_adapter_forward_ell(const void *x, const uint32_t *packed_A, const uint32_t *packed_B,
+                               const float *s_in, const float *s_r, const float *s_out, void *y,
+                               int64_t T, int64_t d_in, int64_t d_out, int r, int ell, int dtype,
+                               void *stream)
+{
+    if (ell < 1 || ell > LORDBA_MAX_ELL) return LORDBA_EUNSUPPORTED;
+    lordba_proj p = dense_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, d_in, d_out, r);
+    p.flags = LORDBA_PROJ_ELL(ell);
+    return lordba_adapter_forward_ex(&p, T, dtype, stream);
 }
 
 int lordba_adapter_forward_f32(const float *x, const uint32_t *packed_A, const uint32_t *packed_B,

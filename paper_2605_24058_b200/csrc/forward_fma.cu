@@ -22,6 +22,7 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxBatch = 32;      // projections per launch (kernel-parameter space)
 constexpr int kAccPerThread = 64;  // TT * RP
+constexpr int kMaxEll = 8;         // envelopes per adapter
 
 struct FmaBatch {
     lordba_proj p[kMaxBatch];
@@ -127,9 +128,12 @@ fma_forward_kernel(const __grid_constant__ FmaBatch batch, int64_t T_tokens)
     const bool x_vec = (reinterpret_cast<uintptr_t>(x) % 16 == 0) && (P.ldx % kVecElems == 0);
     const bool y_vec = (reinterpret_cast<uintptr_t>(y) % 16 == 0) && (P.ldy % kVecElems == 0);
 
+    // envelopes (Eq. 4): ell scale triples sharing the two carriers; ell = 1 is the canonical adapter
+    const int ell = ((P.flags >> 8) & 0xf) + 1;
+
     __shared__ float4 lut[512];                     // byte -> 8 x (+-1.0f)
     __shared__ float red[kWarps][kAccPerThread];
-    __shared__ __align__(16) float zs[kAccPerThread];
+    __shared__ __align__(16) float zs[kMaxEll][kAccPerThread];
 
     {
         float s[8];
@@ -140,141 +144,139 @@ fma_forward_kernel(const __grid_constant__ FmaBatch batch, int64_t T_tokens)
     }
     __syncthreads();
 
-    // ---- stage 1: u[t,k] = sum_i A_sign[k,i] * (s_in[i] * x[t,i]) -------------------------
-    float acc[kAccPerThread];
-#pragma unroll
-    for (int i = 0; i < kAccPerThread; ++i) acc[i] = 0.0f;
-
     const uint8_t *__restrict__ pa = reinterpret_cast<const uint8_t *>(P.packed_A);
     // block-major layout: 64-column block b, row k -> 8 bytes at (b * r + k) * 8
-    const bool s_vec = (reinterpret_cast<uintptr_t>(P.s_in) % 16 == 0);
 
-    for (int64_t c0 = (int64_t)tid * 8; c0 < d_in; c0 += (int64_t)kThreads * 8) {
-        float si[8];
-        if (s_vec && c0 + 8 <= d_in) {
-            const float4 a = __ldg(reinterpret_cast<const float4 *>(P.s_in + c0));
-            const float4 b = __ldg(reinterpret_cast<const float4 *>(P.s_in + c0 + 4));
-            si[0] = a.x; si[1] = a.y; si[2] = a.z; si[3] = a.w;
-            si[4] = b.x; si[5] = b.y; si[6] = b.z; si[7] = b.w;
-        } else {
+    // ---- stage 1, per envelope: u[t,k] = sum_i A_sign[k,i] * (s_in[i] * x[t,i]), z = s_r * u ----
+    for (int env = 0; env < ell; ++env) {
+        const float *__restrict__ s_in = P.s_in + (int64_t)env * d_in;
+        const bool s_vec = (reinterpret_cast<uintptr_t>(s_in) % 16 == 0);
+        float acc[kAccPerThread];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) si[e] = (c0 + e < d_in) ? __ldg(P.s_in + c0 + e) : 0.0f;
-        }
-        float xs[TT][8];
-#pragma unroll
-        for (int t = 0; t < TT; ++t) {
-            if (t < nt) {
-                load8(x + (t0 + t) * P.ldx, c0, d_in, x_vec, xs[t]);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) xs[t][e] *= si[e];
+        for (int i = 0; i < kAccPerThread; ++i) acc[i] = 0.0f;
+
+        for (int64_t c0 = (int64_t)tid * 8; c0 < d_in; c0 += (int64_t)kThreads * 8) {
+            float si[8];
+            if (s_vec && c0 + 8 <= d_in) {
+                const float4 a = __ldg(reinterpret_cast<const float4 *>(s_in + c0));
+                const float4 b = __ldg(reinterpret_cast<const float4 *>(s_in + c0 + 4));
+                si[0] = a.x; si[1] = a.y; si[2] = a.z; si[3] = a.w;
+                si[4] = b.x; si[5] = b.y; si[6] = b.z; si[7] = b.w;
             } else {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) xs[t][e] = 0.0f;
+                for (int e = 0; e < 8; ++e) si[e] = (c0 + e < d_in) ? __ldg(s_in + c0 + e) : 0.0f;
             }
-        }
+            float xs[TT][8];
 #pragma unroll
-        for (int k = 0; k < RP; ++k) {
-            if (k < r) {
-                const uint32_t b = __ldg(pa + ((c0 >> 6) * r + k) * 8 + ((c0 & 63) >> 3));
-                const float4 lo = lut[2 * b], hi = lut[2 * b + 1];
+            for (int t = 0; t < TT; ++t) {
+                if (t < nt) {
+                    load8(x + (t0 + t) * P.ldx, c0, d_in, x_vec, xs[t]);
 #pragma unroll
-                for (int t = 0; t < TT; ++t) {
-                    float a = acc[t * RP + k];
-                    a = fmaf(xs[t][0], lo.x, a); a = fmaf(xs[t][1], lo.y, a);
-                    a = fmaf(xs[t][2], lo.z, a); a = fmaf(xs[t][3], lo.w, a);
-                    a = fmaf(xs[t][4], hi.x, a); a = fmaf(xs[t][5], hi.y, a);
-                    a = fmaf(xs[t][6], hi.z, a); a = fmaf(xs[t][7], hi.w, a);
-                    acc[t * RP + k] = a;
+                    for (int e = 0; e < 8; ++e) xs[t][e] *= si[e];
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) xs[t][e] = 0.0f;
                 }
             }
-        }
-    }
-
-    // ---- reduce across the 32 lanes: transposing butterfly, 64 -> 2 values per lane ----------
 #pragma unroll
-    for (int step = 16, n = kAccPerThread; step >= 1; step >>= 1, n >>= 1) {
-        const bool upper = (lane & step) != 0;
-        const int half = n >> 1;
-#pragma unroll
-        for (int i = 0; i < half; ++i) {
-            const float send = upper ? acc[i] : acc[i + half];
-            const float keep = upper ? acc[i + half] : acc[i];
-            acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
-        }
-    }
-    // lane now holds elements 2*lane and 2*lane+1 of the (t,k) grid
-    red[warp][2 * lane] = acc[0];
-    red[warp][2 * lane + 1] = acc[1];
-    __syncthreads();
-    if (tid < kAccPerThread) {
-        float u = 0.0f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) u += red[w][tid];     // fixed order: deterministic
-        const int k = tid % RP;
-        zs[tid] = (k < r) ? u * __ldg(P.s_r + k) : 0.0f;       // z = s_r * u
-    }
-    __syncthreads();
-
-    // ---- stage 2: y[t,j] += s_out[j] * sum_k B_sign[j,k] * z[t,k] ---------------------------
-    float z[kAccPerThread];
-#pragma unroll
-    for (int i = 0; i < kAccPerThread; i += 4) {
-        const float4 q = *reinterpret_cast<const float4 *>(&zs[i]);
-        z[i] = q.x; z[i + 1] = q.y; z[i + 2] = q.z; z[i + 3] = q.w;
-    }
-    const uint32_t *__restrict__ pb = P.packed_B;
-    const int64_t b_words = (d_out * r + 31) / 32;
-    const bool so_vec = (reinterpret_cast<uintptr_t>(P.s_out) % 16 == 0);
-
-    for (int64_t j0 = (int64_t)tid * 8; j0 < d_out; j0 += (int64_t)kThreads * 8) {
-        float v[TT][8];
-#pragma unroll
-        for (int t = 0; t < TT; ++t)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) v[t][e] = 0.0f;
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj) {
-            const int64_t j = j0 + jj;
-            if (j < d_out) {
-                const uint64_t bits = b_row_bits(pb, b_words, j, r);
-#pragma unroll
-                for (int kc = 0; kc < RP / 8; ++kc) {
-                    const uint32_t b = (uint32_t)(bits >> (8 * kc)) & 0xffu;
+            for (int k = 0; k < RP; ++k) {
+                if (k < r) {
+                    const uint32_t b = __ldg(pa + ((c0 >> 6) * r + k) * 8 + ((c0 & 63) >> 3));
                     const float4 lo = lut[2 * b], hi = lut[2 * b + 1];
 #pragma unroll
                     for (int t = 0; t < TT; ++t) {
-                        const float *zt = &z[t * RP + kc * 8];
-                        float a = v[t][jj];
-                        a = fmaf(zt[0], lo.x, a); a = fmaf(zt[1], lo.y, a);
-                        a = fmaf(zt[2], lo.z, a); a = fmaf(zt[3], lo.w, a);
-                        a = fmaf(zt[4], hi.x, a); a = fmaf(zt[5], hi.y, a);
-                        a = fmaf(zt[6], hi.z, a); a = fmaf(zt[7], hi.w, a);
-                        v[t][jj] = a;
+                        float a = acc[t * RP + k];
+                        a = fmaf(xs[t][0], lo.x, a); a = fmaf(xs[t][1], lo.y, a);
+                        a = fmaf(xs[t][2], lo.z, a); a = fmaf(xs[t][3], lo.w, a);
+                        a = fmaf(xs[t][4], hi.x, a); a = fmaf(xs[t][5], hi.y, a);
+                        a = fmaf(xs[t][6], hi.z, a); a = fmaf(xs[t][7], hi.w, a);
+                        acc[t * RP + k] = a;
                     }
                 }
             }
         }
-        float so[8];
-        if (so_vec && j0 + 8 <= d_out) {
-            const float4 a = __ldg(reinterpret_cast<const float4 *>(P.s_out + j0));
-            const float4 b = __ldg(reinterpret_cast<const float4 *>(P.s_out + j0 + 4));
-            so[0] = a.x; so[1] = a.y; so[2] = a.z; so[3] = a.w;
-            so[4] = b.x; so[5] = b.y; so[6] = b.z; so[7] = b.w;
-        } else {
+
+        // reduce across the 32 lanes: transposing butterfly, 64 -> 2 values per lane
 #pragma unroll
-            for (int e = 0; e < 8; ++e) so[e] = (j0 + e < d_out) ? __ldg(P.s_out + j0 + e) : 0.0f;
+        for (int step = 16, n = kAccPerThread; step >= 1; step >>= 1, n >>= 1) {
+            const bool upper = (lane & step) != 0;
+            const int half = n >> 1;
+#pragma unroll
+            for (int i = 0; i < half; ++i) {
+                const float send = upper ? acc[i] : acc[i + half];
+                const float keep = upper ? acc[i + half] : acc[i];
+                acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
+            }
         }
+        // lane now holds elements 2*lane and 2*lane+1 of the (t,k) grid
+        red[warp][2 * lane] = acc[0];
+        red[warp][2 * lane + 1] = acc[1];
+        __syncthreads();
+        if (tid < kAccPerThread) {
+            float u = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) u += red[w][tid];     // fixed order: deterministic
+            const int k = tid % RP;
+            zs[env][tid] = (k < r) ? u * __ldg(P.s_r + env * r + k) : 0.0f;       // z = s_r * u
+        }
+        __syncthreads();
+    }
+
+    // ---- stage 2: y[t,j] += sum_env s_out[env,j] * sum_k B_sign[j,k] * z[env,t,k] --------------
+    const uint32_t *__restrict__ pb = P.packed_B;
+    const int64_t b_words = (d_out * r + 31) / 32;
+
+    for (int64_t j0 = (int64_t)tid * 8; j0 < d_out; j0 += (int64_t)kThreads * 8) {
+        float yo[TT][8];
 #pragma unroll
         for (int t = 0; t < TT; ++t) {
             if (t < nt) {
-                T *yrow = y + (t0 + t) * P.ldy;
-                float yo[8];
-                load8(yrow, j0, d_out, y_vec, yo);
+                load8(y + (t0 + t) * P.ldy, j0, d_out, y_vec, yo[t]);
+            } else {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) yo[e] = fmaf(so[e], v[t][e], yo[e]);
-                store8(yrow, j0, d_out, y_vec, yo);
+                for (int e = 0; e < 8; ++e) yo[t][e] = 0.0f;
             }
         }
+        for (int env = 0; env < ell; ++env) {
+            float z[kAccPerThread];
+#pragma unroll
+            for (int i = 0; i < kAccPerThread; i += 4) {
+                const float4 q = *reinterpret_cast<const float4 *>(&zs[env][i]);
+                z[i] = q.x; z[i + 1] = q.y; z[i + 2] = q.z; z[i + 3] = q.w;
+            }
+            const float *__restrict__ s_out = P.s_out + (int64_t)env * d_out;
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+                const int64_t j = j0 + jj;
+                if (j < d_out) {
+                    float v[TT];
+#pragma unroll
+                    for (int t = 0; t < TT; ++t) v[t] = 0.0f;
+                    const uint64_t bits = b_row_bits(pb, b_words, j, r);
+#pragma unroll
+                    for (int kc = 0; kc < RP / 8; ++kc) {
+                        const uint32_t b = (uint32_t)(bits >> (8 * kc)) & 0xffu;
+                        const float4 lo = lut[2 * b], hi = lut[2 * b + 1];
+#pragma unroll
+                        for (int t = 0; t < TT; ++t) {
+                            const float *zt = &z[t * RP + kc * 8];
+                            float a = v[t];
+                            a = fmaf(zt[0], lo.x, a); a = fmaf(zt[1], lo.y, a);
+                            a = fmaf(zt[2], lo.z, a); a = fmaf(zt[3], lo.w, a);
+                            a = fmaf(zt[4], hi.x, a); a = fmaf(zt[5], hi.y, a);
+                            a = fmaf(zt[6], hi.z, a); a = fmaf(zt[7], hi.w, a);
+                            v[t] = a;
+                        }
+                    }
+                    const float so = __ldg(s_out + j);
+#pragma unroll
+                    for (int t = 0; t < TT; ++t) yo[t][jj] = fmaf(so, v[t], yo[t][jj]);
+                }
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t)
+            if (t < nt) store8(y + (t0 + t) * P.ldy, j0, d_out, y_vec, yo[t]);
     }
 }
 

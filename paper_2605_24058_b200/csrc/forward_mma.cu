@@ -690,6 +690,7 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
 bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
 {
     if (dtype != LORDBA_BF16 || T < 1 || T > (1 << 30)) return false;
+    if (((p.flags >> 8) & 0xf) != 0) return false;          // multi-envelope adapters: FMA kernel
     if (p.r % 8 != 0 || p.r < 8 || p.r > kMaxRank) return false;
     // whole 64-column groups (the 3-D tensor view), 16-byte aligned rows
     if (p.d_in % kGroup != 0 || p.d_out % kGroup != 0 || p.ldx % 8 != 0 || p.ldy % 8 != 0) return false;

@@ -916,6 +916,7 @@ bool choose_shape(int r, int kp, int n_proj, int64_t T, int min_chunks, LaunchSh
 bool tc_supported(const lordba_proj &p, int64_t T, int dtype)
 {
     if (dtype != LORDBA_BF16 || T < 1) return false;
+    if (((p.flags >> 8) & 0xf) != 0) return false;          // multi-envelope adapters: other kernels
     if (p.r % 8 != 0 || p.r < 8 || p.r > kMaxRank) return false;
     if (p.d_in < kChunk || p.d_out < kChunk) return false;
     if (p.d_in > (1 << 30) || p.d_out > (1 << 30) || T > (1 << 30)) return false;

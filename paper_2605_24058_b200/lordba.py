@@ -19,6 +19,12 @@ LIB_PATH = os.path.join(_PKG, "liblordba.so")
 F32, BF16 = 0, 1
 VARIANT_AUTO, VARIANT_FMA, VARIANT_TC, VARIANT_MMA = 0, 1, 2, 3
 PROJ_OVERLAP = 1
+MAX_ELL = 8
+
+
+def proj_ell(ell: int) -> int:
+    """Flag field for an adapter with ``ell`` envelopes (mirror of LORDBA_PROJ_ELL)."""
+    return ((ell - 1) & 0xF) << 8
 
 _i64 = ctypes.c_int64
 _vp = ctypes.c_void_p
@@ -43,6 +49,8 @@ _SIGNATURES = {
     "lordba_unpack_signs": (ctypes.c_int, [_vp, _i64, _i64, ctypes.c_int, _vp, _vp]),
     "lordba_adapter_forward": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int, _vp]),
     "lordba_adapter_forward_f32": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int, _vp]),
+    "lordba_adapter_forward_ell": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int, ctypes.c_int,
+                                                  ctypes.c_int, _vp]),
     "lordba_adapter_forward_ex": (ctypes.c_int, [ctypes.POINTER(Proj), _i64, ctypes.c_int, _vp]),
     "lordba_adapter_forward_batched": (ctypes.c_int, [ctypes.POINTER(Proj), ctypes.c_int, _i64,
                                                        ctypes.c_int, _vp]),
@@ -188,6 +196,28 @@ def adapter_forward(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, stream=N
         _check(rc, "lordba_adapter_forward_f32")
     else:
         adapter_forward_ex(p, T, _dtype_code(x), stream)
+
+
+def adapter_forward_ell(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, stream=None) -> None:
+    """Multi-envelope adapter (Eq. 4): s_in (ell, d_in), s_r (ell, r), s_out (ell, d_out); dense x, y."""
+    _need_cuda(x, packed_A, packed_B, s_in, s_r, s_out, y)
+    if s_in.dim() != 2 or s_r.dim() != 2 or s_out.dim() != 2 or not (s_in.shape[0] == s_r.shape[0] == s_out.shape[0]):
+        raise ValueError("scales must be (ell, d_in), (ell, r), (ell, d_out)")
+    for s in (s_in, s_r, s_out):
+        if s.dtype != torch.float32 or not s.is_contiguous():
+            raise TypeError("scales must be contiguous float32")
+    if not (x.is_contiguous() and y.is_contiguous()) or x.dtype != y.dtype:
+        raise ValueError("x and y must be dense and of one dtype")
+    ell = s_in.shape[0]
+    T, d_in = x.shape
+    d_out = y.shape[1]
+    if s_in.shape[1] != d_in or s_out.shape[1] != d_out or s_r.shape[1] != r:
+        raise ValueError("scale shapes do not match (d_in, r, d_out)")
+    rc = load().lordba_adapter_forward_ell(x.data_ptr(), packed_A.data_ptr(), packed_B.data_ptr(),
+                                           s_in.data_ptr(), s_r.data_ptr(), s_out.data_ptr(),
+                                           y.data_ptr(), T, d_in, d_out, r, ell, _dtype_code(x),
+                                           _stream(stream))
+    _check(rc, "lordba_adapter_forward_ell")
 
 
 def adapter_forward_ex(p: Proj, T: int, dtype: int, stream=None) -> None:

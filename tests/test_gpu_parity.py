@@ -363,3 +363,40 @@ def test_carriers_packed_by_oracle_and_by_library_agree(oracle):
     a = DeviceProj(p, pack_on_gpu=True)
     b = DeviceProj(p, pack_on_gpu=False, oracle=oracle)
     assert torch.equal(a.packed_A, b.packed_A) and torch.equal(a.packed_B, b.packed_B)
+
+
+# ---------------------------------------------------------------- multi-envelope adapters (Eq. 4, ell > 1)
+
+def _ell_inputs(d_in, d_out, r, T, dtype, ell, seed):
+    base = workloads.make_projection(d_in, d_out, r, T, dtype, seed=seed)
+    rng = np.random.default_rng(seed + 77)
+    s_in = np.exp(rng.normal(0.0, 0.5, size=(ell, d_in))).astype(np.float32)
+    s_r = (64.0 * np.abs(rng.normal(0.0, 0.02, size=(ell, r)))).astype(np.float32)
+    s_out = np.exp(rng.normal(0.0, 0.5, size=(ell, d_out))).astype(np.float32)
+    return base, s_in, s_r, s_out
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("T,d_in,d_out,r,ell", [(70, 256, 192, 8, 2), (300, 1024, 768, 16, 2), (33, 200, 136, 24, 3),
+                                                (150, 4096, 1024, 16, 4), (2048, 4096, 4096, 16, 2)])
+def test_multi_envelope_forward(oracle, dtype, T, d_in, d_out, r, ell):
+    if dtype == "f32" and T > 1000:
+        pytest.skip("full-size case is checked in bf16 only")
+    base, s_in, s_r, s_out = _ell_inputs(d_in, d_out, r, T, dtype, ell, seed=90 + ell + r)
+    d = DeviceProj(base)
+    dev = d.x.device
+    lordba.adapter_forward_ell(d.x, d.packed_A, d.packed_B, torch.from_numpy(s_in).to(dev),
+                               torch.from_numpy(s_r).to(dev), torch.from_numpy(s_out).to(dev), d.y, r)
+    want = oracle.adapter_forward_ell(base.x_f64(), base.A_sign, base.B_sign, s_in.astype(np.float64),
+                                      s_r.astype(np.float64), s_out.astype(np.float64), base.y_f64())
+    assert_close(torch_to_f64(d.y), want, dtype, "ell=%d %s" % (ell, dtype))
+
+
+def test_multi_envelope_with_one_envelope_equals_plain_call(oracle):
+    base, s_in, s_r, s_out = _ell_inputs(1024, 1024, 16, 200, "bf16", 1, seed=95)
+    a, b = DeviceProj(base), DeviceProj(base)
+    dev = a.x.device
+    t = lambda v: torch.from_numpy(v).to(dev)
+    lordba.adapter_forward_ell(a.x, a.packed_A, a.packed_B, t(s_in), t(s_r), t(s_out), a.y, 16)
+    lordba.adapter_forward(b.x, b.packed_A, b.packed_B, t(s_in[0]), t(s_r[0]), t(s_out[0]), b.y, 16)
+    assert torch.equal(a.y, b.y)

@@ -47,7 +47,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel on this workload
 # (ncu capture summarised under profiles/; reads only, the write-back L2 defers the y writes past
 # the end of the kernel).  Set to None whenever the kernel changes after the capture.
-NCU_DRAM_BYTES_PER_LAUNCH = 33634304
+NCU_DRAM_BYTES_PER_LAUNCH = None
 
 
 def measured_peak():
@@ -387,7 +387,7 @@ def run_workload(args):
     r, Tn = args.rank, args.tokens
     H, F = workloads.HIDDEN, workloads.FFN
     layer = [(di, do) for _, di, do in workloads.LAYER_PROJECTIONS]
-    shapes = {"gate": [(H, F)], "down": [(F, H)], "layer": layer, "decode": layer,
+    shapes = {"attn": [(H, H)], "gate": [(H, F)], "down": [(F, H)], "layer": layer, "decode": layer,
               "full": layer * workloads.N_LAYERS}[args.workload]
     gen = torch.Generator(device=dev)
     gen.manual_seed(1234)
@@ -395,15 +395,17 @@ def run_workload(args):
     def rand_signs(rows, cols):
         return (torch.randint(0, 2, (rows, cols), device=dev, generator=gen, dtype=torch.int8) * 2 - 1)
 
+    esh = (args.ell,) if args.ell > 1 else ()      # (ell, d) scales: a multi-envelope adapter (Eq. 4)
     adapters = []
     for di, do in shapes:
         adapters.append(dict(
             pa=lordba.pack_signs(rand_signs(r, di), 0), pb=lordba.pack_signs(rand_signs(do, r), 1),
-            s_in=torch.exp(0.5 * torch.randn(di, device=dev, generator=gen)),
-            s_r=64.0 * (0.02 * torch.randn(r, device=dev, generator=gen)).abs(),
-            s_out=torch.exp(0.5 * torch.randn(do, device=dev, generator=gen))))
+            s_in=torch.exp(0.5 * torch.randn(*esh, di, device=dev, generator=gen)),
+            s_r=64.0 * (0.02 * torch.randn(*esh, r, device=dev, generator=gen)).abs(),
+            s_out=torch.exp(0.5 * torch.randn(*esh, do, device=dev, generator=gen))))
     set_bytes = sum(Tn * (di + do) * ELEM for di, do in shapes)
-    alg_bytes = sum(workloads.algorithmic_bytes(Tn, di, do, r, ELEM) for di, do in shapes)
+    alg_bytes = sum(workloads.algorithmic_bytes(Tn, di, do, r, ELEM) + 4 * (args.ell - 1) * (di + r + do)
+                    for di, do in shapes)
     n_sets = int(max(1, min(np.ceil(8 * L2_BYTES / set_bytes), 40e9 // set_bytes)))
     if set_bytes > 2 * L2_BYTES:
         n_sets = 1                       # one set already exceeds the L2: every step re-reads it from DRAM
@@ -459,8 +461,8 @@ def run_workload(args):
     peak, peak_kind = measured_peak()
     achieved = alg_bytes / (ms * 1e-3 / steps) / 1e9
     line = {
-        "metric": "adapter-branch tokens/s, workload %s (r=%d, T=%d, %d projection(s) per call)"
-                  % (args.workload, r, Tn, len(shapes)),
+        "metric": "adapter-branch tokens/s, workload %s (r=%d, ell=%d, T=%d, %d projection(s) per call)"
+                  % (args.workload, r, args.ell, Tn, len(shapes)),
         "value": Tn * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
         "warmup": reps_w * n_graph, "ms_per_step": ms / steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -493,6 +495,7 @@ def main():
                          "MLP projection, a layer's seven projections in one batched call (prefill, or "
                          "decode with --tokens 1..64), or all 224 projections in one call")
     ap.add_argument("--rank", type=int, default=R)
+    ap.add_argument("--ell", type=int, default=1, help="envelopes per adapter (supplementary workloads only)")
     ap.add_argument("--tokens", type=int, default=T)
     ap.add_argument("--no-overlap", action="store_true",
                     help="every step waits for the previous one to finish (no LORDBA_PROJ_OVERLAP)")
@@ -500,7 +503,7 @@ def main():
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         return run_reference(args)
-    if args.workload != "attn":
+    if args.workload != "attn" or args.ell != 1 or args.rank != R or args.tokens != T:
         return run_workload(args)
     return run_gpu(args)
 

@@ -75,8 +75,8 @@ constexpr long long kWaitLimitCycles = 1500000000LL;
 struct alignas(64) MmaProj {
     CUtensorMap x_map;     // bf16 (64, T, d_in / 64), box 64 x 16 x 16, 128-byte swizzle
     CUtensorMap y_map;     // bf16 (64, T, d_out / 64), box 64 x 16 x (cwy / 64), 128-byte swizzle
-    CUtensorMap si_map;    // f32 (64, d_in / 64), box 64 x 16: the scales of an x item
-    CUtensorMap so_map;    // f32 (64, d_out / 64), box 64 x (cwy / 64)
+    CUtensorMap si_map;    // f32 (64, d_in / 64, ell), box 64 x NW x ell: the scales of an x item
+    CUtensorMap so_map;    // f32 (64, d_out / 64, ell), box 64 x (cwy / 64) x ell
     CUtensorMap pa_map;    // u32 (16, d_in r / 512), box 16 x 2r: the sign bytes of an x item
     CUtensorMap pb_map;    // u32 (16, d_out r / 512), box 16 x (cwy r / 512)
     const float *s_r;
@@ -117,17 +117,18 @@ struct SmemPlan {
 };
 
 // nw: consumer warps = 64-column groups per item
-__host__ __device__ inline SmemPlan make_plan(int nw, int rp, int r, int slots)
+// ell: envelopes (scale triples) of the adapter: ell rows of scales per item, ell partial sums
+__host__ __device__ inline SmemPlan make_plan(int nw, int rp, int r, int slots, int ell)
 {
     SmemPlan s;
     s.off_scale = nw * kBlockBytes;
-    s.off_bits = s.off_scale + nw * kGroup * 4;
+    s.off_bits = s.off_scale + ell * nw * kGroup * 4;
     s.slot_bytes = (s.off_bits + nw * kGroup * r / 8 + 1023) / 1024 * 1024;
     const int ks = (rp + 15) / 16;
     s.off_red = slots * s.slot_bytes;
-    s.off_zh = s.off_red + nw * kTile * rp * 4;
-    s.off_zl = s.off_zh + kTile * ks * 8 * 4;
-    s.off_bar = s.off_zl + kTile * ks * 8 * 4;
+    s.off_zh = s.off_red + ell * nw * kTile * rp * 4;
+    s.off_zl = s.off_zh + ell * kTile * ks * 8 * 4;
+    s.off_bar = s.off_zl + ell * kTile * ks * 8 * 4;
     s.total = s.off_bar + (2 * kMaxSlots + 2) * 8 + 1024;    // + slack to align the base to 1 KiB
     return s;
 }
@@ -266,7 +267,7 @@ __device__ __forceinline__ uint64_t b_row_bits(const uint8_t *bits, int j_local,
 }
 
 // RP: rank padded to 8, 16, 32 or 64.
-template <int RP, int NW>
+template <int RP, int NW, int ELL>
 __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 2)
 mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant__ MmaParams prm)
 {
@@ -288,7 +289,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     const int nt = (int)((prm.T - t0 < rows) ? (prm.T - t0) : rows);
     const int r = P.r;
     const int d_in = P.d_in, d_out = P.d_out;
-    const SmemPlan plan = make_plan(NW, RP, r, S);
+    const SmemPlan plan = make_plan(NW, RP, r, S, ELL);
     const uint32_t sm_base = smem_u32(smem);
 
     // items: all x chunks, then this CTA's share of the y chunks
@@ -332,12 +333,12 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         const int cw = is_x ? cwx : cwy;
         const int col0 = is_x ? it * cwx : (yc_begin + (it - n_x)) * cwy;
         // a box is always whole: what lies past the tensor is filled with zeros and counted
-        const uint32_t bytes = (uint32_t)(cw / kGroup) * kBlockBytes + (uint32_t)cw * 4u + (uint32_t)cw * r / 8u;
+        const uint32_t bytes = (uint32_t)(cw / kGroup) * kBlockBytes + (uint32_t)ELL * cw * 4u + (uint32_t)cw * r / 8u;
         const uint32_t slot = sm_base + s * plan.slot_bytes;
         MMA_TRACE(2 + it);
         mbar_arrive_expect_tx(bar_full(s), bytes);
         tma_load_3d(slot, is_x ? &P.x_map : &P.y_map, 0, (int)t0, col0 / kGroup, bar_full(s));
-        tma_load_2d(slot + plan.off_scale, is_x ? &P.si_map : &P.so_map, 0, col0 / kGroup, bar_full(s));
+        tma_load_3d(slot + plan.off_scale, is_x ? &P.si_map : &P.so_map, 0, col0 / kGroup, 0, bar_full(s));
         tma_load_2d(slot + plan.off_bits, is_x ? &P.pa_map : &P.pb_map, 0, col0 * r / 512, bar_full(s));
         MMA_TRACE(10 + it);
     };
@@ -366,13 +367,15 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         const int pc0 = ((2 * q) ^ g) * 16, pc1 = ((2 * q + 1) ^ g) * 16;
 
         // ---- first product: u[t,k] = sum_i A_sign[k,i] s_in[i] x[t,i] -----------------------
-        float acc[kSplitAcc ? 2 : 1][R8][4];
+        float acc[ELL][kSplitAcc ? 2 : 1][R8][4];
 #pragma unroll
-        for (int h = 0; h < (kSplitAcc ? 2 : 1); ++h)
+        for (int env = 0; env < ELL; ++env)
 #pragma unroll
-            for (int a = 0; a < R8; ++a)
+            for (int h = 0; h < (kSplitAcc ? 2 : 1); ++h)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) acc[h][a][e] = 0.0f;
+                for (int a = 0; a < R8; ++a)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[env][h][a][e] = 0.0f;
 
         int it = 0;
         for (; it < n_x; ++it) {
@@ -388,21 +391,6 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 const uint4 xb0 = *reinterpret_cast<const uint4 *>(slot + off_r0 + pc1);
                 const uint4 xa1 = *reinterpret_cast<const uint4 *>(slot + off_r1 + pc0);
                 const uint4 xb1 = *reinterpret_cast<const uint4 *>(slot + off_r1 + pc1);
-                // s_in of the group as bf16 pairs (hi, lo): lane l converts columns 2l, 2l+1,
-                // then every lane collects the 8 pairs of its 16 columns
-                uint32_t ph, pl;
-                {
-                    const float2 sc = *reinterpret_cast<const float2 *>(slot + plan.off_scale + 4 * (gcol + 2 * lane));
-                    split2(sc.x, sc.y, ph, pl);
-                }
-                uint32_t hA[4], hB[4], lA[4], lB[4];
-#pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    hA[p] = __shfl_sync(0xffffffffu, ph, 8 * q + p);
-                    hB[p] = __shfl_sync(0xffffffffu, ph, 8 * q + 4 + p);
-                    lA[p] = __shfl_sync(0xffffffffu, pl, 8 * q + p);
-                    lB[p] = __shfl_sync(0xffffffffu, pl, 8 * q + 4 + p);
-                }
                 const uint2 *blk = reinterpret_cast<const uint2 *>(slot + plan.off_bits) + warp * r;
                 uint32_t bytes[R8];                                  // sign bytes of this lane's 16 columns
 #pragma unroll
@@ -412,22 +400,41 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     const uint2 sb = blk[k];                         // the row's 64 sign bits of this block
                     bytes[a] = (((q & 2) ? sb.y : sb.x) >> (16 * (q & 1))) & 0xffffu;
                 }
-                // k-step outermost, rank blocks innermost: consecutive MMAs go to different
-                // accumulators, so none waits for the one before it
                 const uint32_t xk[4][4] = {{xa0.x, xa1.x, xa0.y, xa1.y}, {xa0.z, xa1.z, xa0.w, xa1.w},
                                            {xb0.x, xb1.x, xb0.y, xb1.y}, {xb0.z, xb1.z, xb0.w, xb1.w}};
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint32_t h0 = (ks < 2) ? hA[2 * ks] : hB[2 * ks - 4], h1 = (ks < 2) ? hA[2 * ks + 1] : hB[2 * ks - 3];
-                    const uint32_t l0 = (ks < 2) ? lA[2 * ks] : lB[2 * ks - 4], l1 = (ks < 2) ? lA[2 * ks + 1] : lB[2 * ks - 3];
+                for (int env = 0; env < ELL; ++env) {
+                    // s_in[env] of the group as bf16 pairs (hi, lo): lane l converts columns 2l, 2l+1,
+                    // then every lane collects the 8 pairs of its 16 columns
+                    uint32_t ph, pl;
+                    {
+                        const float2 sc = *reinterpret_cast<const float2 *>(slot + plan.off_scale +
+                                                                            4 * (env * cwx + gcol + 2 * lane));
+                        split2(sc.x, sc.y, ph, pl);
+                    }
+                    uint32_t hA[4], hB[4], lA[4], lB[4];
 #pragma unroll
-                    for (int a = 0; a < R8; ++a) {
-                        const uint32_t b = (ks < 2) ? (bytes[a] & 0xffu) : (bytes[a] >> 8);
-                        const uint32_t m0 = pair_bits(b, 2 * (ks & 1)), m1 = pair_bits(b, 2 * (ks & 1) + 1);
-                        mma_bf16(acc[0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
-                                 with_signs(h0, m0), with_signs(h1, m1));
-                        mma_bf16(acc[kSplitAcc ? 1 : 0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
-                                 with_signs(l0, m0), with_signs(l1, m1));
+                    for (int p = 0; p < 4; ++p) {
+                        hA[p] = __shfl_sync(0xffffffffu, ph, 8 * q + p);
+                        hB[p] = __shfl_sync(0xffffffffu, ph, 8 * q + 4 + p);
+                        lA[p] = __shfl_sync(0xffffffffu, pl, 8 * q + p);
+                        lB[p] = __shfl_sync(0xffffffffu, pl, 8 * q + 4 + p);
+                    }
+                    // k-step outermost, rank blocks innermost: consecutive MMAs go to different
+                    // accumulators, so none waits for the one before it
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint32_t h0 = (ks < 2) ? hA[2 * ks] : hB[2 * ks - 4], h1 = (ks < 2) ? hA[2 * ks + 1] : hB[2 * ks - 3];
+                        const uint32_t l0 = (ks < 2) ? lA[2 * ks] : lB[2 * ks - 4], l1 = (ks < 2) ? lA[2 * ks + 1] : lB[2 * ks - 3];
+#pragma unroll
+                        for (int a = 0; a < R8; ++a) {
+                            const uint32_t b = (ks < 2) ? (bytes[a] & 0xffu) : (bytes[a] >> 8);
+                            const uint32_t m0 = pair_bits(b, 2 * (ks & 1)), m1 = pair_bits(b, 2 * (ks & 1) + 1);
+                            mma_bf16(acc[env][0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                     with_signs(h0, m0), with_signs(h1, m1));
+                            mma_bf16(acc[env][kSplitAcc ? 1 : 0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                     with_signs(l0, m0), with_signs(l1, m1));
+                        }
                     }
                 }
             }
@@ -441,29 +448,35 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         uint32_t *zH = reinterpret_cast<uint32_t *>(smem + plan.off_zh);
         uint32_t *zL = reinterpret_cast<uint32_t *>(smem + plan.off_zl);
 #pragma unroll
-        for (int a = 0; a < R8; ++a) {
-            float c[4];
+        for (int env = 0; env < ELL; ++env) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) c[e] = kSplitAcc ? acc[0][a][e] + acc[kSplitAcc ? 1 : 0][a][e] : acc[0][a][e];
-            float *d0 = red + ((warp * kTile + g) * RP + 8 * a + 2 * q);
-            *reinterpret_cast<float2 *>(d0) = make_float2(c[0], c[1]);
-            *reinterpret_cast<float2 *>(d0 + 8 * RP) = make_float2(c[2], c[3]);
+            for (int a = 0; a < R8; ++a) {
+                float c[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    c[e] = kSplitAcc ? acc[env][0][a][e] + acc[env][kSplitAcc ? 1 : 0][a][e] : acc[env][0][a][e];
+                float *d0 = red + (((env * kConsumerWarps + warp) * kTile + g) * RP + 8 * a + 2 * q);
+                *reinterpret_cast<float2 *>(d0) = make_float2(c[0], c[1]);
+                *reinterpret_cast<float2 *>(d0 + 8 * RP) = make_float2(c[2], c[3]);
+            }
         }
         consumer_sync<kConsumerThreads>();
-        for (int idx = tid; idx < kTile * ZP; idx += kConsumerThreads) {
-            const int tok = idx / ZP, pr = idx - tok * ZP;
+        for (int idx = tid; idx < ELL * kTile * ZP; idx += kConsumerThreads) {
+            const int env = idx / (kTile * ZP), rem = idx - env * (kTile * ZP);
+            const int tok = rem / ZP, pr = rem - tok * ZP;
             float u0 = 0.0f, u1 = 0.0f;
             if (2 * pr < RP) {
 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float2 v = *reinterpret_cast<const float2 *>(red + ((w * kTile + tok) * RP + 2 * pr));
+                    const float2 v = *reinterpret_cast<const float2 *>(
+                        red + (((env * kConsumerWarps + w) * kTile + tok) * RP + 2 * pr));
                     u0 += v.x;
                     u1 += v.y;
                 }
             }
             const int k = 2 * pr;
-            const float z0 = (k < r) ? u0 * __ldg(P.s_r + k) : 0.0f;
-            const float z1 = (k + 1 < r) ? u1 * __ldg(P.s_r + k + 1) : 0.0f;
+            const float z0 = (k < r) ? u0 * __ldg(P.s_r + env * r + k) : 0.0f;
+            const float z1 = (k + 1 < r) ? u1 * __ldg(P.s_r + env * r + k + 1) : 0.0f;
             uint32_t hi, lo;
             split2(z0, z1, hi, lo);
             zH[idx] = hi;
@@ -474,16 +487,21 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
 
         // ---- second product: y[t,j] += s_out[j] sum_k B_sign[j,k] z[t,k] ---------------------
         // A fragments: k position (2q, 2q+1, 2q+8, 2q+9) of k-step s <-> ranks 16s + 4q + (0,1,2,3)
-        uint32_t zh[KS][4], zl[KS][4];
+        // (with one envelope they are loaded once here, with several inside the item loop)
+        auto load_z = [&](int env, uint32_t (&zh)[KS][4], uint32_t (&zl)[KS][4]) {
+            const uint32_t *eh = zH + env * (kTile * ZP), *el = zL + env * (kTile * ZP);
 #pragma unroll
-        for (int s = 0; s < KS; ++s) {
-            const uint2 h0 = *reinterpret_cast<const uint2 *>(zH + g * ZP + 8 * s + 2 * q);
-            const uint2 h1 = *reinterpret_cast<const uint2 *>(zH + (g + 8) * ZP + 8 * s + 2 * q);
-            const uint2 l0 = *reinterpret_cast<const uint2 *>(zL + g * ZP + 8 * s + 2 * q);
-            const uint2 l1 = *reinterpret_cast<const uint2 *>(zL + (g + 8) * ZP + 8 * s + 2 * q);
-            zh[s][0] = h0.x; zh[s][1] = h1.x; zh[s][2] = h0.y; zh[s][3] = h1.y;
-            zl[s][0] = l0.x; zl[s][1] = l1.x; zl[s][2] = l0.y; zl[s][3] = l1.y;
-        }
+            for (int s = 0; s < KS; ++s) {
+                const uint2 h0 = *reinterpret_cast<const uint2 *>(eh + g * ZP + 8 * s + 2 * q);
+                const uint2 h1 = *reinterpret_cast<const uint2 *>(eh + (g + 8) * ZP + 8 * s + 2 * q);
+                const uint2 l0 = *reinterpret_cast<const uint2 *>(el + g * ZP + 8 * s + 2 * q);
+                const uint2 l1 = *reinterpret_cast<const uint2 *>(el + (g + 8) * ZP + 8 * s + 2 * q);
+                zh[s][0] = h0.x; zh[s][1] = h1.x; zh[s][2] = h0.y; zh[s][3] = h1.y;
+                zl[s][0] = l0.x; zl[s][1] = l1.x; zl[s][2] = l0.y; zl[s][3] = l1.y;
+            }
+        };
+        uint32_t zh[KS][4], zl[KS][4];
+        if (ELL == 1) load_z(0, zh, zl);
         __nv_bfloat16 *yrow0 = P.y + (t0 + g) * P.ldy;
         __nv_bfloat16 *yrow1 = yrow0 + 8 * P.ldy;
         const bool vec32 = P.y_vec32 != 0;
@@ -522,31 +540,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 uint32_t out[2][8];
 #pragma unroll
                 for (int cc = 0; cc < 2; ++cc) {
-                    float c[4][4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) c[i][e] = 0.0f;
-                    // k-step outermost, n-blocks innermost: consecutive MMAs go to different accumulators
-#pragma unroll
-                    for (int ks = 0; ks < KS; ++ks) {
-                        uint32_t b0[4], b1[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint32_t nib = (uint32_t)(rb[4 * cc + i] >> (16 * ks)) & 0xfu;
-                            b0[i] = with_signs(0x3f803f80u, nib * 0x40008000u);
-                            b1[i] = with_signs(0x3f803f80u, nib * 0x10002000u);
-                        }
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            mma_bf16(c[i], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b0[i], b1[i]);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            mma_bf16(c[i], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b0[i], b1[i]);
-                    }
-                    const float4 *so4 = reinterpret_cast<const float4 *>(slot + plan.off_scale + 4 * (gcol + 16 * q + 8 * cc));
-                    const float4 s0 = so4[0], s1 = so4[1];
-                    const float so[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                    float vs[2][8];                                  // y + sum over the envelopes of s_out * v
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {              // token rows g and g + 8
                         const uint4 yv = *reinterpret_cast<const uint4 *>(slot + (half == 0 ? off_r0 : off_r1) +
@@ -554,11 +548,52 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                         const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            const float o0 = fmaf(so[2 * i], c[i][2 * half], lo_f(yw[i]));
-                            const float o1 = fmaf(so[2 * i + 1], c[i][2 * half + 1], hi_f(yw[i]));
-                            out[half][4 * cc + i] = pack2(o0, o1);
+                            vs[half][2 * i] = lo_f(yw[i]);
+                            vs[half][2 * i + 1] = hi_f(yw[i]);
                         }
                     }
+#pragma unroll
+                    for (int env = 0; env < ELL; ++env) {
+                        if (ELL > 1) load_z(env, zh, zl);
+                        float c[4][4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) c[i][e] = 0.0f;
+                        // k-step outermost, n-blocks innermost: consecutive MMAs go to different accumulators
+#pragma unroll
+                        for (int ks = 0; ks < KS; ++ks) {
+                            uint32_t b0[4], b1[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const uint32_t nib = (uint32_t)(rb[4 * cc + i] >> (16 * ks)) & 0xfu;
+                                b0[i] = with_signs(0x3f803f80u, nib * 0x40008000u);
+                                b1[i] = with_signs(0x3f803f80u, nib * 0x10002000u);
+                            }
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                mma_bf16(c[i], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b0[i], b1[i]);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                mma_bf16(c[i], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b0[i], b1[i]);
+                        }
+                        const float4 *so4 = reinterpret_cast<const float4 *>(
+                            slot + plan.off_scale + 4 * (env * cwy + gcol + 16 * q + 8 * cc));
+                        const float4 s0 = so4[0], s1 = so4[1];
+                        const float so[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+                        for (int half = 0; half < 2; ++half)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                vs[half][2 * i] = fmaf(so[2 * i], c[i][2 * half], vs[half][2 * i]);
+                                vs[half][2 * i + 1] = fmaf(so[2 * i + 1], c[i][2 * half + 1], vs[half][2 * i + 1]);
+                            }
+                    }
+#pragma unroll
+                    for (int half = 0; half < 2; ++half)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            out[half][4 * cc + i] = pack2(vs[half][2 * i], vs[half][2 * i + 1]);
                 }
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
@@ -643,6 +678,16 @@ bool make_linear_map(CUtensorMap *map, CUtensorMapDataType type, const void *bas
     return encode(map, type, 2, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
+// ell x d float32 scales (envelope e in row e, d % 64 == 0) seen as (64, d / 64, ell); a box is
+// `groups` groups of all envelopes: it lands as [envelope][group][64 floats].
+bool make_scale_map(CUtensorMap *map, const float *base, int64_t d, int ell, int groups)
+{
+    const cuuint64_t dims[3] = {(cuuint64_t)kGroup, (cuuint64_t)(d / kGroup), (cuuint64_t)ell};
+    const cuuint64_t strides[2] = {(cuuint64_t)kGroup * 4, (cuuint64_t)d * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)kGroup, (cuuint32_t)groups, (cuuint32_t)ell};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+
 int padded_rank(int r) { return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64; }
 
 int sm_count()
@@ -657,13 +702,13 @@ int sm_count()
     return n;
 }
 
-template <int RP, int NW>
+template <int RP, int NW, int ELL>
 cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem, cudaStream_t stream)
 {
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, []() {
-        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW, ELL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSmemBudget);
     });
     if (attr_rc != cudaSuccess) return attr_rc;
@@ -682,7 +727,7 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP, NW>, b, prm);
+    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP, NW, ELL>, b, prm);
 }
 
 }  // namespace
@@ -690,7 +735,8 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
 bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
 {
     if (dtype != LORDBA_BF16 || T < 1 || T > (1 << 30)) return false;
-    if (((p.flags >> 8) & 0xf) != 0) return false;          // multi-envelope adapters: FMA kernel
+    const int ell = ((p.flags >> 8) & 0xf) + 1;
+    if (ell > 2 || (ell == 2 && p.r > 32)) return false;    // more envelopes, or two at high rank: FMA kernel
     if (p.r % 8 != 0 || p.r < 8 || p.r > kMaxRank) return false;
     // whole 64-column groups (the 3-D tensor view), 16-byte aligned rows
     if (p.d_in % kGroup != 0 || p.d_out % kGroup != 0 || p.ldx % 8 != 0 || p.ldy % 8 != 0) return false;
@@ -714,12 +760,13 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
     bool all_overlap = true;          // the caller's promise covers the call only if every projection carries it
     for (int i = 0; i < n; ++i) all_overlap = all_overlap && (projs[i].flags & LORDBA_PROJ_OVERLAP);
     int launches = 0;
+    for (int ell = 1; ell <= 2; ++ell)
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
         const lordba_proj *sel[kMaxBatch];
         int m = 0, max_r = 0;
         int64_t min_dout = (int64_t)1 << 40;
         for (int i = 0; i <= n; ++i) {
-            const bool take = (i < n) && padded_rank(projs[i].r) == rp;
+            const bool take = (i < n) && padded_rank(projs[i].r) == rp && ((projs[i].flags >> 8) & 0xf) + 1 == ell;
             if (take) {
                 sel[m++] = &projs[i];
                 if (projs[i].r > max_r) max_r = projs[i].r;
@@ -762,10 +809,8 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                     // sign bytes: d r / 8 per carrier, as rows of 16 words; an item holds cw r / 512 rows
                     if (!make_data_map(&t.x_map, q.x, T, q.d_in, q.ldx, nw) ||
                         !make_data_map(&t.y_map, q.y, T, q.d_out, q.ldy, cw / kGroup) ||
-                        !make_linear_map(&t.si_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, q.s_in, kGroup,
-                                         q.d_in / kGroup, nw) ||
-                        !make_linear_map(&t.so_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, q.s_out, kGroup,
-                                         q.d_out / kGroup, cw / kGroup) ||
+                        !make_scale_map(&t.si_map, q.s_in, q.d_in, ell, nw) ||
+                        !make_scale_map(&t.so_map, q.s_out, q.d_out, ell, cw / kGroup) ||
                         !make_linear_map(&t.pa_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_A, 16,
                                          q.d_in * q.r / 512, max_chunk * q.r / 512) ||
                         !make_linear_map(&t.pb_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_B, 16,
@@ -787,25 +832,37 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                     prm.trace = reinterpret_cast<long long *>(std::strtoull(tp, nullptr, 0));
 #endif
                 int slots = kMaxSlots;
-                while (slots > 2 && make_plan(nw, rp, max_r, slots).total > smem_budget) --slots;
-                const SmemPlan plan = make_plan(nw, rp, max_r, slots);
+                while (slots > 2 && make_plan(nw, rp, max_r, slots, ell).total > smem_budget) --slots;
+                const SmemPlan plan = make_plan(nw, rp, max_r, slots, ell);
                 if (plan.total > kSmemBudget) return LORDBA_ECUDA;
                 prm.slots = slots;
                 const dim3 grid((unsigned)tiles, (unsigned)m, (unsigned)splits);
                 cudaError_t e;
-                if (nw == kMaxWarps) {
+                if (ell == 1 && nw == kMaxWarps) {
                     switch (rp) {
-                        case 8:  e = launch_one<8, 16>(b, prm, grid, plan.total, stream); break;
-                        case 16: e = launch_one<16, 16>(b, prm, grid, plan.total, stream); break;
-                        case 32: e = launch_one<32, 16>(b, prm, grid, plan.total, stream); break;
-                        default: e = launch_one<64, 16>(b, prm, grid, plan.total, stream); break;
+                        case 8:  e = launch_one<8, 16, 1>(b, prm, grid, plan.total, stream); break;
+                        case 16: e = launch_one<16, 16, 1>(b, prm, grid, plan.total, stream); break;
+                        case 32: e = launch_one<32, 16, 1>(b, prm, grid, plan.total, stream); break;
+                        default: e = launch_one<64, 16, 1>(b, prm, grid, plan.total, stream); break;
+                    }
+                } else if (ell == 1) {
+                    switch (rp) {
+                        case 8:  e = launch_one<8, 8, 1>(b, prm, grid, plan.total, stream); break;
+                        case 16: e = launch_one<16, 8, 1>(b, prm, grid, plan.total, stream); break;
+                        case 32: e = launch_one<32, 8, 1>(b, prm, grid, plan.total, stream); break;
+                        default: e = launch_one<64, 8, 1>(b, prm, grid, plan.total, stream); break;
+                    }
+                } else if (nw == kMaxWarps) {
+                    switch (rp) {
+                        case 8:  e = launch_one<8, 16, 2>(b, prm, grid, plan.total, stream); break;
+                        case 16: e = launch_one<16, 16, 2>(b, prm, grid, plan.total, stream); break;
+                        default: e = launch_one<32, 16, 2>(b, prm, grid, plan.total, stream); break;
                     }
                 } else {
                     switch (rp) {
-                        case 8:  e = launch_one<8, 8>(b, prm, grid, plan.total, stream); break;
-                        case 16: e = launch_one<16, 8>(b, prm, grid, plan.total, stream); break;
-                        case 32: e = launch_one<32, 8>(b, prm, grid, plan.total, stream); break;
-                        default: e = launch_one<64, 8>(b, prm, grid, plan.total, stream); break;
+                        case 8:  e = launch_one<8, 8, 2>(b, prm, grid, plan.total, stream); break;
+                        case 16: e = launch_one<16, 8, 2>(b, prm, grid, plan.total, stream); break;
+                        default: e = launch_one<32, 8, 2>(b, prm, grid, plan.total, stream); break;
                     }
                 }
                 if (e != cudaSuccess) return LORDBA_ECUDA;

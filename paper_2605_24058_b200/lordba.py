@@ -167,7 +167,11 @@ def make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, flags: int = 0
         if s.dtype != torch.float32 or not s.is_contiguous():
             raise TypeError("scales must be contiguous float32")
     d_in, d_out = x.shape[1], y.shape[1]
-    if s_in.numel() != d_in or s_out.numel() != d_out or s_r.numel() != r:
+    # 2-D scales (ell, d) make a multi-envelope adapter: the envelope count goes into the flags
+    ell = s_in.shape[0] if s_in.dim() == 2 else 1
+    if ell > 1:
+        flags |= proj_ell(ell)
+    if s_in.numel() != ell * d_in or s_out.numel() != ell * d_out or s_r.numel() != ell * r:
         raise ValueError("scale vector sizes do not match d_in / r / d_out")
     if packed_A.numel() != packed_words(r, d_in, 0) or packed_B.numel() != packed_words(d_out, r, 1):
         raise ValueError("packed carrier sizes do not match (r, d_in, d_out)")

@@ -47,7 +47,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel on this workload
 # (ncu capture summarised under profiles/; reads only, the write-back L2 defers the y writes past
 # the end of the kernel).  Set to None whenever the kernel changes after the capture.
-NCU_DRAM_BYTES_PER_LAUNCH = None
+NCU_DRAM_BYTES_PER_LAUNCH = 33633792
 
 
 def measured_peak():

@@ -70,11 +70,12 @@ typedef enum {
 
 /* Kernel families the forward entry points can be pinned to (default AUTO). */
 typedef enum {
-    LORDBA_VARIANT_AUTO = 0,  /* register-streaming kernel when the shape allows it, else FMA */
+    LORDBA_VARIANT_AUTO = 0,  /* the library's choice: streaming kernel where the shape allows  */
+                              /* it (tcgen05 kernel for rank > 32 with many tiles), else FMA   */
     LORDBA_VARIANT_FMA = 1,   /* CUDA-core float32 FMA kernel (always used for LORDBA_F32)  */
     LORDBA_VARIANT_TC = 2,    /* tcgen05/TMA cluster kernel; LORDBA_EUNSUPPORTED if the     */
                               /* shape or alignment rules it out                            */
-    LORDBA_VARIANT_MMA = 3    /* register-streaming mma.sync kernel; LORDBA_EUNSUPPORTED if */
+    LORDBA_VARIANT_MMA = 3    /* TMA-fed streaming mma.sync kernel; LORDBA_EUNSUPPORTED if   */
                               /* the shape or alignment rules it out                        */
 } lordba_variant;
 

@@ -387,7 +387,8 @@ def run_workload(args):
     r, Tn = args.rank, args.tokens
     H, F = workloads.HIDDEN, workloads.FFN
     layer = [(di, do) for _, di, do in workloads.LAYER_PROJECTIONS]
-    shapes = {"attn": [(H, H)], "gate": [(H, F)], "down": [(F, H)], "layer": layer, "decode": layer,
+    n_seg = args.segments if args.workload == "multi" else 0
+    shapes = {"attn": [(H, H)], "multi": [(H, H)] * max(n_seg, 1), "gate": [(H, F)], "down": [(F, H)], "layer": layer, "decode": layer,
               "full": layer * workloads.N_LAYERS}[args.workload]
     gen = torch.Generator(device=dev)
     gen.manual_seed(1234)
@@ -421,7 +422,10 @@ def run_workload(args):
         bufs = sets[i % n_sets]
         projs = [lordba.make_proj(x, a["pa"], a["pb"], a["s_in"], a["s_r"], a["s_out"], y, r, flags)
                  for (x, y), a in zip(bufs, adapters)]
-        if len(projs) == 1:
+        if n_seg:
+            # multi-adapter batch: n_seg segments of Tn tokens, one adapter each, one call
+            lordba.adapter_forward_segments(projs, [Tn] * n_seg, lordba.BF16)
+        elif len(projs) == 1:
             lordba.adapter_forward_ex(projs[0], Tn, lordba.BF16)
         else:
             lordba.adapter_forward_batched(projs, Tn, lordba.BF16)
@@ -490,10 +494,12 @@ def main():
     ap.add_argument("--traffic", type=float, default=NCU_DRAM_BYTES_PER_LAUNCH,
                     help="ncu DRAM bytes per launch to report in roofline.traffic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full"],
+    ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full", "multi"],
                     help="attn = the headline configuration (default); the others are supplementary: one "
                          "MLP projection, a layer's seven projections in one batched call (prefill, or "
                          "decode with --tokens 1..64), or all 224 projections in one call")
+    ap.add_argument("--segments", type=int, default=8,
+                    help="workload multi: segments (adapters) per call, --tokens rows each, attention shape")
     ap.add_argument("--rank", type=int, default=R)
     ap.add_argument("--ell", type=int, default=1, help="envelopes per adapter (supplementary workloads only)")
     ap.add_argument("--tokens", type=int, default=T)

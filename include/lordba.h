@@ -176,6 +176,18 @@ int lordba_adapter_forward_batched(const lordba_proj *projs, int n_proj, int64_t
                                    void *stream);
 
 /*
+ * Multi-adapter batch (Section 3.1, condition A4: many task adapters served over one frozen
+ * base): segment i is tokens[i] consecutive token rows that go through their own adapter.
+ * segs[i].x / .y point at the segment's first row (usually into one shared x / y matrix),
+ * the other fields name the segment's adapter; several segments may share an adapter.
+ * segs, tokens: [host] arrays of n_seg entries, read before the call returns.  Segments are
+ * treated as simultaneous (same disjointness rules as the batched call); empty segments are
+ * skipped.  One launch per 24 segments of equal padded rank.
+ */
+int lordba_adapter_forward_segments(const lordba_proj *segs, const int64_t *tokens, int n_seg, int dtype,
+                                    void *stream);
+
+/*
  * Host-buffer form of lordba_adapter_forward{,_f32}: x_host and y_host are
  * [host] (pinned memory makes the copies asynchronous), dense rows; the carriers
  * and scales stay [device] because they are loaded once per adapter.

@@ -67,18 +67,24 @@ int validate_proj(const lordba_proj &p, int64_t T, int dtype)
 
 // batch_checked: the caller has verified that the projections of this call are independent of
 // one another (disjoint y buffers, no x inside a y), so its launches may overlap each other.
-int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream, bool batch_checked)
+// tokens: per-projection token rows, or nullptr when every projection has T rows.
+int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, int dtype, cudaStream_t stream,
+             bool batch_checked)
 {
     const int variant = g_variant.load(std::memory_order_relaxed);
+    std::vector<int64_t> rows(n, T);
+    if (tokens) rows.assign(tokens, tokens + n);
     if (variant == LORDBA_VARIANT_FMA || dtype == LORDBA_F32) {
         if (variant == LORDBA_VARIANT_TC || variant == LORDBA_VARIANT_MMA) return LORDBA_EUNSUPPORTED;
-        return launch_forward_fma(projs, n, T, dtype, stream);
+        return launch_forward_fma(projs, rows.data(), n, dtype, stream);
     }
     // Split the list: what the chosen tensor-core kernel can take, and the rest.  Left to itself
     // the library takes the tcgen05 kernel where it was measured ahead of the streaming one: ranks
-    // above 32 with at least two waves of full 128-token tiles.
+    // above 32 with at least two waves of full 128-token tiles.  (That kernel wants one token
+    // count for all projections.)
     bool use_tc = (variant == LORDBA_VARIANT_TC);
-    if (variant == LORDBA_VARIANT_AUTO) {
+    if (use_tc && tokens) return LORDBA_EUNSUPPORTED;
+    if (variant == LORDBA_VARIANT_AUTO && !tokens) {
         int64_t big_rank_tiles = 0;
         bool all_big = n > 0;
         for (int i = 0; i < n; ++i) {
@@ -88,18 +94,21 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t
         use_tc = all_big && big_rank_tiles >= 2 * 148;
     }
     std::vector<lordba_proj> fast, fma;
+    std::vector<int64_t> fast_rows, fma_rows;
     for (int i = 0; i < n; ++i) {
-        const bool ok = use_tc ? tc_supported(projs[i], T, dtype) : mma_supported(projs[i], T, dtype);
+        if (rows[i] == 0) continue;
+        const bool ok = use_tc ? tc_supported(projs[i], rows[i], dtype) : mma_supported(projs[i], rows[i], dtype);
         (ok ? fast : fma).push_back(projs[i]);
+        (ok ? fast_rows : fma_rows).push_back(rows[i]);
     }
     if (variant != LORDBA_VARIANT_AUTO && !fma.empty()) return LORDBA_EUNSUPPORTED;
     if (!fast.empty()) {
         const int rc = use_tc ? launch_forward_tc(fast.data(), (int)fast.size(), T, dtype, stream)
-                              : launch_forward_mma(fast.data(), (int)fast.size(), T, dtype, stream,
+                              : launch_forward_mma(fast.data(), fast_rows.data(), (int)fast.size(), dtype, stream,
                                                    batch_checked);
         if (rc != LORDBA_OK) return rc;
     }
-    if (!fma.empty()) return launch_forward_fma(fma.data(), (int)fma.size(), T, dtype, stream);
+    if (!fma.empty()) return launch_forward_fma(fma.data(), fma_rows.data(), (int)fma.size(), dtype, stream);
     return LORDBA_OK;
 }
 
@@ -156,7 +165,7 @@ int lordba_adapter_forward_ex(const lordba_proj *p, int64_t T, int dtype, void *
     const int rc = validate_proj(*p, T, dtype);
     if (rc != LORDBA_OK) return rc;
     if (T == 0) return LORDBA_OK;
-    return dispatch(p, 1, T, dtype, static_cast<cudaStream_t>(stream), false);
+    return dispatch(p, 1, T, nullptr, dtype, static_cast<cudaStream_t>(stream), false);
 }
 
 int lordba_adapter_forward(const void *x, const uint32_t *packed_A, const uint32_t *packed_B,
@@ -209,7 +218,30 @@ int lordba_adapter_forward_batched(const lordba_proj *projs, int n_proj, int64_t
             }
     }
     if (T == 0 || n_proj == 0) return LORDBA_OK;
-    return dispatch(projs, n_proj, T, dtype, static_cast<cudaStream_t>(stream), true);
+    return dispatch(projs, n_proj, T, nullptr, dtype, static_cast<cudaStream_t>(stream), true);
+}
+
+int lordba_adapter_forward_segments(const lordba_proj *segs, const int64_t *tokens, int n_seg, int dtype,
+                                    void *stream)
+{
+    if (n_seg < 0 || (n_seg > 0 && (!segs || !tokens))) return LORDBA_EINVAL;
+    const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
+    for (int i = 0; i < n_seg; ++i) {
+        const int rc = validate_proj(segs[i], tokens[i], dtype);
+        if (rc != LORDBA_OK) return rc;
+    }
+    // segments are simultaneous: outputs pairwise disjoint, no input inside an output
+    for (int i = 0; i < n_seg; ++i)
+        for (int j = 0; j < n_seg; ++j) {
+            if (i == j || tokens[i] == 0 || tokens[j] == 0) continue;
+            const size_t ni = ((size_t)(tokens[i] - 1) * segs[i].ldy + segs[i].d_out) * e;
+            const size_t nj = ((size_t)(tokens[j] - 1) * segs[j].ldy + segs[j].d_out) * e;
+            const size_t nx = ((size_t)(tokens[i] - 1) * segs[i].ldx + segs[i].d_in) * e;
+            if (j > i && overlaps(segs[i].y, ni, segs[j].y, nj)) return LORDBA_EINVAL;
+            if (overlaps(segs[i].x, nx, segs[j].y, nj)) return LORDBA_EINVAL;
+        }
+    if (n_seg == 0) return LORDBA_OK;
+    return dispatch(segs, n_seg, 0, tokens, dtype, static_cast<cudaStream_t>(stream), true);
 }
 
 size_t lordba_host_workspace_bytes(int64_t T, int64_t d_in, int64_t d_out, int dtype)
@@ -243,7 +275,7 @@ int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(xd, x_host, bx, cudaMemcpyHostToDevice, s) != cudaSuccess) return LORDBA_ECUDA;
     if (cudaMemcpyAsync(yd, y_host, by, cudaMemcpyHostToDevice, s) != cudaSuccess) return LORDBA_ECUDA;
-    const int rc2 = dispatch(&p, 1, T, dtype, s, false);
+    const int rc2 = dispatch(&p, 1, T, nullptr, dtype, s, false);
     if (rc2 != LORDBA_OK) return rc2;
     if (cudaMemcpyAsync(y_host, yd, by, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LORDBA_ECUDA;
     return LORDBA_OK;

@@ -26,6 +26,7 @@ constexpr int kMaxEll = 8;         // envelopes per adapter
 
 struct FmaBatch {
     lordba_proj p[kMaxBatch];
+    int64_t tokens[kMaxBatch];    // token rows of each projection
 };
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -109,8 +110,9 @@ __device__ __forceinline__ uint64_t b_row_bits(const uint32_t *__restrict__ pb, 
 
 template <typename T, int RP>
 __global__ void __launch_bounds__(kThreads)
-fma_forward_kernel(const __grid_constant__ FmaBatch batch, int64_t T_tokens)
+fma_forward_kernel(const __grid_constant__ FmaBatch batch)
 {
+    const int64_t T_tokens = batch.tokens[blockIdx.y];
     constexpr int TT = kAccPerThread / RP;          // tokens per CTA
     const lordba_proj &P = batch.p[blockIdx.y];
     const int tid = threadIdx.x;
@@ -281,16 +283,18 @@ fma_forward_kernel(const __grid_constant__ FmaBatch batch, int64_t T_tokens)
 }
 
 template <typename T>
-cudaError_t launch_rank(const FmaBatch &b, int n, int64_t T_tokens, int rp, cudaStream_t stream)
+cudaError_t launch_rank(const FmaBatch &b, int n, int rp, cudaStream_t stream)
 {
     const int tt = kAccPerThread / rp;
+    int64_t T_tokens = 0;                          // the longest projection sets grid.x
+    for (int i = 0; i < n; ++i) if (b.tokens[i] > T_tokens) T_tokens = b.tokens[i];
     const int64_t tiles = (T_tokens + tt - 1) / tt;
     dim3 grid((unsigned)tiles, (unsigned)n, 1);
     switch (rp) {
-        case 8:  fma_forward_kernel<T, 8><<<grid, kThreads, 0, stream>>>(b, T_tokens); break;
-        case 16: fma_forward_kernel<T, 16><<<grid, kThreads, 0, stream>>>(b, T_tokens); break;
-        case 32: fma_forward_kernel<T, 32><<<grid, kThreads, 0, stream>>>(b, T_tokens); break;
-        default: fma_forward_kernel<T, 64><<<grid, kThreads, 0, stream>>>(b, T_tokens); break;
+        case 8:  fma_forward_kernel<T, 8><<<grid, kThreads, 0, stream>>>(b); break;
+        case 16: fma_forward_kernel<T, 16><<<grid, kThreads, 0, stream>>>(b); break;
+        case 32: fma_forward_kernel<T, 32><<<grid, kThreads, 0, stream>>>(b); break;
+        default: fma_forward_kernel<T, 64><<<grid, kThreads, 0, stream>>>(b); break;
     }
     count_launch();
     return cudaGetLastError();
@@ -300,20 +304,20 @@ int padded_rank(int r) { return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64; }
 
 }  // namespace
 
-int launch_forward_fma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream)
+int launch_forward_fma(const lordba_proj *projs, const int64_t *tokens, int n, int dtype, cudaStream_t stream)
 {
-    if (T == 0 || n == 0) return LORDBA_OK;
+    if (n == 0) return LORDBA_OK;
     // Group projections of equal padded rank into launches of at most kMaxBatch.
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
         FmaBatch b;
         int m = 0;
         for (int i = 0; i <= n; ++i) {
-            const bool take = (i < n) && padded_rank(projs[i].r) == rp;
-            if (take) b.p[m++] = projs[i];
+            const bool take = (i < n) && tokens[i] > 0 && padded_rank(projs[i].r) == rp;
+            if (take) { b.tokens[m] = tokens[i]; b.p[m++] = projs[i]; }
             if (m == kMaxBatch || (i == n && m > 0)) {
                 const cudaError_t e = (dtype == LORDBA_F32)
-                                          ? launch_rank<float>(b, m, T, rp, stream)
-                                          : launch_rank<__nv_bfloat16>(b, m, T, rp, stream);
+                                          ? launch_rank<float>(b, m, rp, stream)
+                                          : launch_rank<__nv_bfloat16>(b, m, rp, stream);
                 if (e != cudaSuccess) return LORDBA_ECUDA;
                 m = 0;
             }

@@ -82,6 +82,7 @@ struct alignas(64) MmaProj {
     const float *s_r;
     __nv_bfloat16 *y;
     int64_t ldy;
+    int64_t T;             // token rows of this projection (projections of a launch may differ)
     int d_in, d_out, r;
     int y_vec32;           // y rows are 32-byte aligned: 256-bit stores
 };
@@ -91,7 +92,6 @@ struct MmaBatch {
 };
 
 struct MmaParams {
-    int64_t T;
     int rows;          // token rows per CTA tile (<= 16)
     int cwy;           // columns per y item: a multiple of 64, <= 1024 (x items are 1024 wide)
     int slots;         // ring depth
@@ -285,8 +285,8 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     const int rows = prm.rows, cwy = prm.cwy, S = prm.slots;
     constexpr int cwx = NW * kGroup;
     const int64_t t0 = (int64_t)blockIdx.x * rows;
-    if (t0 >= prm.T) return;
-    const int nt = (int)((prm.T - t0 < rows) ? (prm.T - t0) : rows);
+    if (t0 >= P.T) return;
+    const int nt = (int)((P.T - t0 < rows) ? (P.T - t0) : rows);
     const int r = P.r;
     const int d_in = P.d_in, d_out = P.d_out;
     const SmemPlan plan = make_plan(NW, RP, r, S, ELL);
@@ -749,10 +749,10 @@ bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
     return encode_fn() != nullptr;
 }
 
-int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream,
+int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, int dtype, cudaStream_t stream,
                        bool batch_checked)
 {
-    if (n == 0 || T == 0) return LORDBA_OK;
+    if (n == 0) return LORDBA_OK;
     if (dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
     int *status = device_status_word();
     if (!status) return LORDBA_ECUDA;
@@ -763,11 +763,14 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
     for (int ell = 1; ell <= 2; ++ell)
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
         const lordba_proj *sel[kMaxBatch];
+        int64_t sel_T[kMaxBatch];
         int m = 0, max_r = 0;
         int64_t min_dout = (int64_t)1 << 40;
         for (int i = 0; i <= n; ++i) {
-            const bool take = (i < n) && padded_rank(projs[i].r) == rp && ((projs[i].flags >> 8) & 0xf) + 1 == ell;
+            const bool take = (i < n) && tokens[i] > 0 && padded_rank(projs[i].r) == rp &&
+                              ((projs[i].flags >> 8) & 0xf) + 1 == ell;
             if (take) {
+                sel_T[m] = tokens[i];
                 sel[m++] = &projs[i];
                 if (projs[i].r > max_r) max_r = projs[i].r;
                 if (projs[i].d_out < min_dout) min_dout = projs[i].d_out;
@@ -775,24 +778,28 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
             if (m == kMaxBatch || (i == n && m > 0)) {
                 // Tile height: the smallest number of full waves of 16-row tiles, then the rows
                 // per tile that spread the tokens evenly over those waves.
-                const int64_t min_tiles = (int64_t)m * ((T + kTile - 1) / kTile);
+                int64_t min_tiles = 0, sum_T = 0;
+                for (int k = 0; k < m; ++k) { min_tiles += (sel_T[k] + kTile - 1) / kTile; sum_T += sel_T[k]; }
                 const int64_t waves = (min_tiles + sms - 1) / sms;
-                int64_t tiles_target = waves * sms / m;
-                if (tiles_target < 1) tiles_target = 1;
-                int64_t rows = (T + tiles_target - 1) / tiles_target;
+                int64_t rows = (sum_T + waves * sms - 1) / (waves * sms);
                 if (rows > kTile) rows = kTile;
                 if (rows < 1) rows = 1;
-                const int64_t tiles = (T + rows - 1) / rows;
+                int64_t tiles = 0, all_tiles = 0;      // widest projection (grid.x), and the sum
+                for (int k = 0; k < m; ++k) {
+                    const int64_t tk = (sel_T[k] + rows - 1) / rows;
+                    all_tiles += tk;
+                    if (tk > tiles) tiles = tk;
+                }
                 // Few tokens: split the y items over several CTAs per tile (each repeats the
                 // first product), with narrower items so that there is something to split.
-                int64_t want_splits = sms / (tiles * m);
+                int64_t want_splits = sms / all_tiles;
                 if (want_splits < 1) want_splits = 1;
                 // Two small CTAs per SM when there is a second CTA to pair with: more than one
                 // wave of tiles, or a call that may overlap its neighbours.  One's start-up and
                 // first-load latency then hide behind the other's streaming.  A lone single-wave
                 // call keeps one CTA with 16 consumer warps per SM.
                 const bool overlaps_neighbours = (launches == 0) ? all_overlap : batch_checked;
-                const int nw = (tiles * m > sms || overlaps_neighbours) ? 8 : kMaxWarps;
+                const int nw = (all_tiles > sms || overlaps_neighbours) ? 8 : kMaxWarps;
                 const int max_chunk = nw * kGroup;
                 const int smem_budget = (nw == kMaxWarps) ? kSmemBudget : kSmemBudgetHalf;
                 int cw = max_chunk;
@@ -807,8 +814,8 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                     const lordba_proj &q = *sel[k];
                     MmaProj &t = b.p[k];
                     // sign bytes: d r / 8 per carrier, as rows of 16 words; an item holds cw r / 512 rows
-                    if (!make_data_map(&t.x_map, q.x, T, q.d_in, q.ldx, nw) ||
-                        !make_data_map(&t.y_map, q.y, T, q.d_out, q.ldy, cw / kGroup) ||
+                    if (!make_data_map(&t.x_map, q.x, sel_T[k], q.d_in, q.ldx, nw) ||
+                        !make_data_map(&t.y_map, q.y, sel_T[k], q.d_out, q.ldy, cw / kGroup) ||
                         !make_scale_map(&t.si_map, q.s_in, q.d_in, ell, nw) ||
                         !make_scale_map(&t.so_map, q.s_out, q.d_out, ell, cw / kGroup) ||
                         !make_linear_map(&t.pa_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_A, 16,
@@ -819,11 +826,12 @@ int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cu
                     t.s_r = q.s_r;
                     t.y = static_cast<__nv_bfloat16 *>(q.y);
                     t.ldy = q.ldy;
+                    t.T = sel_T[k];
                     t.d_in = (int)q.d_in; t.d_out = (int)q.d_out; t.r = q.r;
                     t.y_vec32 = (reinterpret_cast<uintptr_t>(q.y) % 32 == 0 && q.ldy % 16 == 0) ? 1 : 0;
                 }
                 MmaParams prm;
-                prm.T = T; prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
+                prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
                 prm.wait_prev = !overlaps_neighbours;
                 ++launches;
                 prm.trace = nullptr;

@@ -33,7 +33,8 @@ int launch_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int role, 
 
 // --- forward_fma.cu ----------------------------------------------------------
 // n projections (validated by the caller), same T and dtype.  Any shape.
-int launch_forward_fma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream);
+// tokens[i]: token rows of projection i (entries may differ; zero entries are skipped).
+int launch_forward_fma(const lordba_proj *projs, const int64_t *tokens, int n, int dtype, cudaStream_t stream);
 
 // --- forward_tc.cu -----------------------------------------------------------
 // True when the tcgen05/TMA kernel can take this projection (bf16, 16-byte
@@ -48,7 +49,7 @@ bool mma_supported(const lordba_proj &p, int64_t T, int dtype);
 // batch_checked: the projections are known to be independent of one another, so the launches of
 // this call may overlap each other; LORDBA_PROJ_OVERLAP on every projection lets the first
 // launch overlap the previous call as well.
-int launch_forward_mma(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream,
+int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, int dtype, cudaStream_t stream,
                        bool batch_checked);
 
 }  // namespace lordba

@@ -54,6 +54,8 @@ _SIGNATURES = {
     "lordba_adapter_forward_ex": (ctypes.c_int, [ctypes.POINTER(Proj), _i64, ctypes.c_int, _vp]),
     "lordba_adapter_forward_batched": (ctypes.c_int, [ctypes.POINTER(Proj), ctypes.c_int, _i64,
                                                        ctypes.c_int, _vp]),
+    "lordba_adapter_forward_segments": (ctypes.c_int, [ctypes.POINTER(Proj), ctypes.POINTER(_i64), ctypes.c_int,
+                                                       ctypes.c_int, _vp]),
     "lordba_host_workspace_bytes": (ctypes.c_size_t, [_i64, _i64, _i64, ctypes.c_int]),
     "lordba_adapter_forward_host": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int,
                                                                ctypes.c_int, _vp, ctypes.c_size_t, _vp]),
@@ -233,6 +235,16 @@ def adapter_forward_batched(projs: Sequence[Proj], T: int, dtype: int, stream=No
     arr = (Proj * len(projs))(*projs)
     _check(load().lordba_adapter_forward_batched(arr, len(projs), T, dtype, _stream(stream)),
            "lordba_adapter_forward_batched")
+
+
+def adapter_forward_segments(segs: Sequence[Proj], tokens: Sequence[int], dtype: int, stream=None) -> None:
+    """Multi-adapter batch: segment i = tokens[i] rows starting at segs[i].x / .y with its own adapter."""
+    if len(segs) != len(tokens):
+        raise ValueError("one token count per segment")
+    arr = (Proj * len(segs))(*segs)
+    tok = (_i64 * len(tokens))(*[int(t) for t in tokens])
+    _check(load().lordba_adapter_forward_segments(arr, tok, len(segs), dtype, _stream(stream)),
+           "lordba_adapter_forward_segments")
 
 
 def host_workspace_bytes(T: int, d_in: int, d_out: int, dtype: int) -> int:

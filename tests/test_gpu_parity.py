@@ -400,3 +400,38 @@ def test_multi_envelope_with_one_envelope_equals_plain_call(oracle):
     lordba.adapter_forward_ell(a.x, a.packed_A, a.packed_B, t(s_in), t(s_r), t(s_out), a.y, 16)
     lordba.adapter_forward(b.x, b.packed_A, b.packed_B, t(s_in[0]), t(s_r[0]), t(s_out[0]), b.y, 16)
     assert torch.equal(a.y, b.y)
+
+
+# ---------------------------------------------------------------- multi-adapter batches (segments)
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d_in,d_out,r,lengths", [(1024, 768, 16, (100, 17, 0, 583)), (4096, 4096, 16, (256,) * 8),
+                                                    (520, 392, 8, (1, 2, 3)), (2048, 1024, 32, (130, 130))])
+def test_segments_each_with_its_own_adapter(oracle, dtype, d_in, d_out, r, lengths):
+    """One x / y matrix, consecutive row segments, a different adapter per segment (the last
+    segment reuses the first adapter): every segment must match the oracle run on its rows."""
+    if dtype == "f32" and d_in == 4096:
+        pytest.skip("full-size case is checked in bf16 only")
+    T = sum(lengths)
+    base = workloads.make_projection(d_in, d_out, r, T, dtype, seed=300 + r)
+    n_adapters = max(1, len(lengths) - 1)
+    adapters = [workloads.make_projection(d_in, d_out, r, 1, dtype, seed=310 + i) for i in range(n_adapters)]
+    dev = torch.device("cuda:0")
+    x = np_to_torch(base.x, dtype, dev)
+    y = np_to_torch(base.y, dtype, dev)
+    dads = [DeviceProj(a) for a in adapters]
+    segs, want = [], base.y_f64().copy()
+    start = 0
+    for i, n in enumerate(lengths):
+        a, da = adapters[i % n_adapters], dads[i % n_adapters]
+        lo = min(start, T - 1)                      # an empty segment still needs a well-formed pointer
+        segs.append(lordba.make_proj(x[lo:lo + max(n, 1)], da.packed_A, da.packed_B, da.s_in, da.s_r, da.s_out,
+                                     y[lo:lo + max(n, 1)], r))
+        if n:
+            rows = slice(start, start + n)
+            want[rows] = oracle.adapter_forward(base.x_f64()[rows], a.A_sign, a.B_sign, a.s_in.astype(np.float64),
+                                                a.s_r.astype(np.float64), a.s_out.astype(np.float64),
+                                                base.y_f64()[rows])
+        start += n
+    lordba.adapter_forward_segments(segs, lengths, lordba.BF16 if dtype == "bf16" else lordba.F32)
+    assert_close(torch_to_f64(y), want, dtype, "segments %s %s" % (lengths, dtype))

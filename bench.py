@@ -483,6 +483,52 @@ def run_workload(args):
     return 0
 
 
+def run_dense_lora_context(args):
+    """Context only, not the product: the dense bf16 LoRA side branch y += (x A^T) B^T of the same
+    rank as two torch.matmul calls (library GEMMs), timed the same way as the attention workload."""
+    import torch
+    dev = torch.device("cuda", 0)
+    r, Tn, H = args.rank, args.tokens, workloads.HIDDEN
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7)
+    A = (0.02 * torch.randn(r, H, device=dev, generator=gen)).to(torch.bfloat16)
+    Bm = (0.02 * torch.randn(H, r, device=dev, generator=gen)).to(torch.bfloat16)
+    set_bytes = 2 * Tn * H * ELEM
+    n_sets = int(np.ceil(8 * L2_BYTES / set_bytes))
+    xs = [torch.randn(Tn, H, device=dev, generator=gen).to(torch.bfloat16) for _ in range(n_sets)]
+    ys = [torch.randn(Tn, H, device=dev, generator=gen).to(torch.bfloat16) for _ in range(n_sets)]
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        def step(i):
+            ys[i].addmm_(torch.matmul(xs[i], A.t()), Bm.t())
+        for i in range(n_sets):
+            step(i)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(n_sets):
+                step(i)
+        reps = max(1, args.steps // n_sets)
+        for _ in range(max(1, args.warmup // n_sets)):
+            graph.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+    steps = reps * n_sets
+    ms = e0.elapsed_time(e1)
+    alg = 3 * Tn * H * ELEM + 2 * r * H * ELEM * 2 // 2
+    print(json.dumps({"metric": "context: dense bf16 LoRA side branch (torch.matmul), r=%d, T=%d, 4096->4096" % (r, Tn),
+                      "impl": "torch library GEMMs", "value": Tn * steps / (ms * 1e-3), "unit": UNIT,
+                      "ms_per_step": ms / steps, "steps": steps,
+                      "roofline": {"bound": "hbm", "achieved": alg / (ms * 1e-3 / steps) / 1e9, "unit": "GB/s"}}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -494,7 +540,7 @@ def main():
     ap.add_argument("--traffic", type=float, default=NCU_DRAM_BYTES_PER_LAUNCH,
                     help="ncu DRAM bytes per launch to report in roofline.traffic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full", "multi"],
+    ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full", "multi", "lora-dense"],
                     help="attn = the headline configuration (default); the others are supplementary: one "
                          "MLP projection, a layer's seven projections in one batched call (prefill, or "
                          "decode with --tokens 1..64), or all 224 projections in one call")
@@ -509,6 +555,8 @@ def main():
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload == "lora-dense":
+        return run_dense_lora_context(args)
     if args.workload != "attn" or args.ell != 1 or args.rank != R or args.tokens != T:
         return run_workload(args)
     return run_gpu(args)

@@ -435,3 +435,32 @@ def test_segments_each_with_its_own_adapter(oracle, dtype, d_in, d_out, r, lengt
         start += n
     lordba.adapter_forward_segments(segs, lengths, lordba.BF16 if dtype == "bf16" else lordba.F32)
     assert_close(torch_to_f64(y), want, dtype, "segments %s %s" % (lengths, dtype))
+
+
+# ---------------------------------------------------------------- the adjoint is the same path with the roles swapped
+
+def test_adjoint_is_a_forward_with_swapped_carriers(oracle):
+    """dX = ((dY D_gamma) B2^T D_beta) B1^T D_alpha (the backward of Eq. 8 with respect to X) is the
+    forward of the adapter (A' = B_sign^T, B' = A_sign^T, s_in' = s_out, s_out' = s_in).  Checked
+    two ways: against the oracle run on the swapped adapter, and through <dy, f(x)> = <f*(dy), x>."""
+    T, d_in, d_out, r = 200, 1024, 768, 16
+    p = workloads.make_projection(d_in, d_out, r, T, "bf16", seed=400)
+    dy = workloads.to_bf16_bits(np.random.default_rng(401).standard_normal((T, d_out), dtype=np.float32))
+    dev = torch.device("cuda:0")
+    A_t = np.ascontiguousarray(p.B_sign.T)          # r x d_out: plays A_sign
+    B_t = np.ascontiguousarray(p.A_sign.T)          # d_in x r: plays B_sign
+    pa = lordba.pack_signs(torch.from_numpy(A_t).to(dev), 0)
+    pb = lordba.pack_signs(torch.from_numpy(B_t).to(dev), 1)
+    dy_dev = np_to_torch(dy, "bf16", dev)
+    dx = torch.zeros(T, d_in, dtype=torch.bfloat16, device=dev)
+    t = lambda v: torch.from_numpy(v).to(dev)
+    lordba.adapter_forward(dy_dev, pa, pb, t(p.s_out), t(p.s_r), t(p.s_in), dx, r)
+    dy64 = workloads.bf16_bits_to_f32(dy).astype(np.float64)
+    want = oracle.adapter_forward(dy64, A_t, B_t, p.s_out.astype(np.float64), p.s_r.astype(np.float64),
+                                  p.s_in.astype(np.float64), np.zeros((T, d_in)))
+    assert_close(torch_to_f64(dx), want, "bf16", "adjoint")
+    # inner-product identity with the oracle's forward of the original adapter (float64 on both sides)
+    fx = oracle.adapter_forward(p.x_f64(), p.A_sign, p.B_sign, p.s_in.astype(np.float64), p.s_r.astype(np.float64),
+                                p.s_out.astype(np.float64), np.zeros((T, d_out)))
+    lhs, rhs = float((dy64 * fx).sum()), float((want * p.x_f64()).sum())
+    assert abs(lhs - rhs) <= 1e-9 * max(abs(lhs), abs(rhs))

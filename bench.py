@@ -397,13 +397,17 @@ def run_workload(args):
         return (torch.randint(0, 2, (rows, cols), device=dev, generator=gen, dtype=torch.int8) * 2 - 1)
 
     esh = (args.ell,) if args.ell > 1 else ()      # (ell, d) scales: a multi-envelope adapter (Eq. 4)
+    io_t, io_code = {"bf16": (torch.bfloat16, lordba.BF16), "f16": (torch.float16, lordba.F16)}[args.dtype]
+    # an adapter exported with half-precision scales: values rounded to float16, declared to the library
+    exported = (lambda s: s.to(torch.float16).to(torch.float32)) if args.scales_f16 else (lambda s: s)
+    base_flags = lordba.PROJ_SCALES_F16 if args.scales_f16 else 0
     adapters = []
     for di, do in shapes:
         adapters.append(dict(
             pa=lordba.pack_signs(rand_signs(r, di), 0), pb=lordba.pack_signs(rand_signs(do, r), 1),
-            s_in=torch.exp(0.5 * torch.randn(*esh, di, device=dev, generator=gen)),
-            s_r=64.0 * (0.02 * torch.randn(*esh, r, device=dev, generator=gen)).abs(),
-            s_out=torch.exp(0.5 * torch.randn(*esh, do, device=dev, generator=gen))))
+            s_in=exported(torch.exp(0.5 * torch.randn(*esh, di, device=dev, generator=gen))),
+            s_r=exported(64.0 * (0.02 * torch.randn(*esh, r, device=dev, generator=gen)).abs()),
+            s_out=exported(torch.exp(0.5 * torch.randn(*esh, do, device=dev, generator=gen)))))
     set_bytes = sum(Tn * (di + do) * ELEM for di, do in shapes)
     alg_bytes = sum(workloads.algorithmic_bytes(Tn, di, do, r, ELEM) + 4 * (args.ell - 1) * (di + r + do)
                     for di, do in shapes)
@@ -412,23 +416,23 @@ def run_workload(args):
         n_sets = 1                       # one set already exceeds the L2: every step re-reads it from DRAM
     sets = []
     for _ in range(n_sets):
-        sets.append([(torch.randn(Tn, di, device=dev, generator=gen, dtype=torch.float32).to(torch.bfloat16),
-                      torch.randn(Tn, do, device=dev, generator=gen, dtype=torch.float32).to(torch.bfloat16))
+        sets.append([(torch.randn(Tn, di, device=dev, generator=gen, dtype=torch.float32).to(io_t),
+                      torch.randn(Tn, do, device=dev, generator=gen, dtype=torch.float32).to(io_t))
                      for di, do in shapes])
     overlap_ok = n_sets > 1 and not args.no_overlap
 
     def step(i):
-        flags = lordba.PROJ_OVERLAP if (overlap_ok and i % n_sets != 0) else 0
+        flags = base_flags | (lordba.PROJ_OVERLAP if (overlap_ok and i % n_sets != 0) else 0)
         bufs = sets[i % n_sets]
         projs = [lordba.make_proj(x, a["pa"], a["pb"], a["s_in"], a["s_r"], a["s_out"], y, r, flags)
                  for (x, y), a in zip(bufs, adapters)]
         if n_seg:
             # multi-adapter batch: n_seg segments of Tn tokens, one adapter each, one call
-            lordba.adapter_forward_segments(projs, [Tn] * n_seg, lordba.BF16)
+            lordba.adapter_forward_segments(projs, [Tn] * n_seg, io_code)
         elif len(projs) == 1:
-            lordba.adapter_forward_ex(projs[0], Tn, lordba.BF16)
+            lordba.adapter_forward_ex(projs[0], Tn, io_code)
         else:
-            lordba.adapter_forward_batched(projs, Tn, lordba.BF16)
+            lordba.adapter_forward_batched(projs, Tn, io_code)
 
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
@@ -469,8 +473,9 @@ def run_workload(args):
                   % (args.workload, r, args.ell, Tn, len(shapes)),
         "value": Tn * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
         "warmup": reps_w * n_graph, "ms_per_step": ms / steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
         "config": {"workload": args.workload, "projections": len(shapes), "rank": r, "tokens": Tn,
+                   "scales": "float16 values, declared (LORDBA_PROJ_SCALES_F16)" if args.scales_f16 else "float32",
                    "l2": "%d buffer set(s) of %.0f MB" % (n_sets, set_bytes / 1e6),
                    "launch": "CUDA graph of %d steps replayed" % n_graph,
                    "step_dependency": "declared independent" if overlap_ok else "each step waits for the previous one"},
@@ -549,6 +554,10 @@ def main():
     ap.add_argument("--rank", type=int, default=R)
     ap.add_argument("--ell", type=int, default=1, help="envelopes per adapter (supplementary workloads only)")
     ap.add_argument("--tokens", type=int, default=T)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16"],
+                    help="element type of x and y (supplementary workloads; the default workload is bf16)")
+    ap.add_argument("--scales-f16", action="store_true",
+                    help="scales rounded to float16 values and declared so (an adapter exported in fp16)")
     ap.add_argument("--no-overlap", action="store_true",
                     help="every step waits for the previous one to finish (no LORDBA_PROJ_OVERLAP)")
     args = ap.parse_args()
@@ -557,7 +566,8 @@ def main():
         return run_reference(args)
     if args.workload == "lora-dense":
         return run_dense_lora_context(args)
-    if args.workload != "attn" or args.ell != 1 or args.rank != R or args.tokens != T:
+    if (args.workload != "attn" or args.ell != 1 or args.rank != R or args.tokens != T or args.dtype != "bf16" or
+            args.scales_f16):
         return run_workload(args)
     return run_gpu(args)
 

@@ -55,7 +55,11 @@ extern "C" {
 
 typedef enum {
     LORDBA_F32 = 0,   /* x and y are float32                                   */
-    LORDBA_BF16 = 1   /* x and y are bfloat16; all accumulation is in float32  */
+    LORDBA_BF16 = 1,  /* x and y are bfloat16; all accumulation is in float32  */
+    LORDBA_F16 = 2    /* x and y are IEEE half (the precision the method exports its adapters in:
+                         Sec. "Training and export", fp16 scales and activations); accumulation
+                         in float32.  s_in is used as a pair of halves here: |s_in| must stay below
+                         65504, and entries below 2^-14 are used with fewer than 22 bits */
 } lordba_dtype;
 
 typedef enum {
@@ -91,7 +95,7 @@ typedef struct lordba_proj {
     void           *y;          /* [device] T x d_out, pitch ldy, updated in place */
     int64_t d_in, d_out, ldx, ldy;
     int32_t r;
-    int32_t flags;              /* LORDBA_PROJ_OVERLAP and / or LORDBA_PROJ_ELL(ell); other bits 0 */
+    int32_t flags;              /* LORDBA_PROJ_OVERLAP, LORDBA_PROJ_SCALES_F16, LORDBA_PROJ_ELL(ell); other bits 0 */
 } lordba_proj;
 
 /*
@@ -118,6 +122,25 @@ typedef struct lordba_proj {
  * kernel acts on the flag; elsewhere it is accepted and ignored.
  */
 #define LORDBA_PROJ_OVERLAP 1
+
+/*
+ * lordba_proj.flags: the caller states that every entry of s_in is exactly representable as an
+ * IEEE half, which is the case for an adapter exported with fp16 scales (the method trains the
+ * scales in fp32 and casts them to fp16 at export) and widened by lordba_scales_from_f16.  With
+ * LORDBA_F16 activations the streaming kernel then forms x * s_in in one tensor-core pass
+ * instead of two; with a false statement the low bits of s_in beyond a half are ignored, nothing
+ * else.  Other kernels and dtypes accept the flag and ignore it.
+ */
+#define LORDBA_PROJ_SCALES_F16 2
+
+/*
+ * Widens n IEEE-half scales (the storage format of an exported adapter, 2 bytes per scale as in
+ * the method's footprint count, Eq. 5) to the float32 arrays that the forward calls take.  Once
+ * per adapter, like packing.  src: [device] n halves, 2-byte aligned; dst: [device] n floats.
+ * Exact (every half is a float).  Asynchronous on stream.  n = 0 is a no-op; n < 0 or a null
+ * pointer with n > 0 is LORDBA_EINVAL.
+ */
+int lordba_scales_from_f16(const uint16_t *src, float *dst, int64_t n, void *stream);
 
 /* Number of uint32 words of a packed carrier (layout above); -1 on bad arguments. */
 int64_t lordba_packed_words(int64_t rows, int64_t cols, int role);
@@ -153,7 +176,7 @@ int lordba_adapter_forward_f32(const float *x, const uint32_t *packed_A, const u
 
 /*
  * Multi-envelope form of the two calls above (Eq. 4, ell >= 1), dense rows: s_in is ell x d_in,
- * s_r ell x r, s_out ell x d_out.  dtype: LORDBA_BF16 or LORDBA_F32.
+ * s_r ell x r, s_out ell x d_out.  dtype: LORDBA_BF16, LORDBA_F16 or LORDBA_F32.
  */
 int lordba_adapter_forward_ell(const void *x, const uint32_t *packed_A, const uint32_t *packed_B,
                                const float *s_in, const float *s_r, const float *s_out, void *y,

@@ -43,11 +43,13 @@ bool overlaps(const void *a, size_t na, const void *b, size_t nb)
     return a0 < b0 + nb && b0 < a0 + na;
 }
 
+bool known_dtype(int dtype) { return dtype == LORDBA_F32 || dtype == LORDBA_BF16 || dtype == LORDBA_F16; }
+
 int validate_proj(const lordba_proj &p, int64_t T, int dtype)
 {
-    if (dtype != LORDBA_F32 && dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    if (!known_dtype(dtype)) return LORDBA_EUNSUPPORTED;
     if (T < 0 || p.d_in < 1 || p.d_out < 1 || p.ldx < p.d_in || p.ldy < p.d_out) return LORDBA_EINVAL;
-    if ((p.flags & ~(LORDBA_PROJ_OVERLAP | 0xf00)) != 0) return LORDBA_EINVAL;
+    if ((p.flags & ~(LORDBA_PROJ_OVERLAP | LORDBA_PROJ_SCALES_F16 | 0xf00)) != 0) return LORDBA_EINVAL;
     if (((p.flags >> 8) & 0xf) + 1 > LORDBA_MAX_ELL) return LORDBA_EUNSUPPORTED;
     if (p.r < 1 || p.r > kMaxRank) return LORDBA_EUNSUPPORTED;
     if (T == 0) return LORDBA_OK;   // nothing is touched: the pointers may be anything
@@ -146,6 +148,15 @@ int lordba_pack_signs(const int8_t *signs, int64_t rows, int64_t cols, int role,
     if (!signs || !packed) return LORDBA_EINVAL;
     if (!aligned(packed, 4)) return LORDBA_EALIGN;
     return launch_pack(signs, rows, cols, role, packed, static_cast<cudaStream_t>(stream));
+}
+
+int lordba_scales_from_f16(const uint16_t *src, float *dst, int64_t n, void *stream)
+{
+    if (n < 0) return LORDBA_EINVAL;
+    if (n == 0) return LORDBA_OK;
+    if (!src || !dst) return LORDBA_EINVAL;
+    if (!aligned(src, 2) || !aligned(dst, 4)) return LORDBA_EALIGN;
+    return launch_widen_scales(src, dst, n, static_cast<cudaStream_t>(stream));
 }
 
 int lordba_unpack_signs(const uint32_t *packed, int64_t rows, int64_t cols, int role, int8_t *signs,
@@ -259,7 +270,7 @@ int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
                                 int64_t d_out, int r, int dtype, void *workspace,
                                 size_t workspace_bytes, void *stream)
 {
-    if (dtype != LORDBA_F32 && dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    if (!known_dtype(dtype)) return LORDBA_EUNSUPPORTED;
     if (T < 0 || d_in < 1 || d_out < 1) return LORDBA_EINVAL;
     if (!x_host || !y_host || !workspace) return LORDBA_EINVAL;
     if (!aligned(workspace, 256)) return LORDBA_EALIGN;
@@ -319,7 +330,7 @@ int lordba_adapter_forward_host_static(const void *x_host, const uint32_t *packe
                                        const float *s_out, void *y_host, int64_t T, int64_t d_in,
                                        int64_t d_out, int r, int dtype, void *stream)
 {
-    if (dtype != LORDBA_F32 && dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    if (!known_dtype(dtype)) return LORDBA_EUNSUPPORTED;
     if (T < 0 || d_in < 1 || d_out < 1) return LORDBA_EINVAL;
     const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
     // sizes that cannot fit are refused before any multiplication can overflow

@@ -12,6 +12,7 @@
 // the SM.  This kernel takes every shape, pitch and alignment; it is the only
 // kernel for float32 activations (no reduced-precision step anywhere).
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "lordba_internal.h"
 
@@ -60,6 +61,23 @@ __device__ __forceinline__ void load8(const __nv_bfloat16 *row, int64_t c0, int6
     }
 }
 
+__device__ __forceinline__ void load8(const __half *row, int64_t c0, int64_t n, bool vec, float out[8])
+{
+    if (vec && c0 + 8 <= n) {
+        const uint4 a = __ldcs(reinterpret_cast<const uint4 *>(row + c0));
+        const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[e]));
+            out[2 * e] = f.x;
+            out[2 * e + 1] = f.y;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out[e] = (c0 + e < n) ? __half2float(row[c0 + e]) : 0.0f;
+    }
+}
+
 __device__ __forceinline__ void store8(float *row, int64_t c0, int64_t n, bool vec, const float v[8])
 {
     if (vec && c0 + 8 <= n) {
@@ -90,6 +108,26 @@ __device__ __forceinline__ void store8(__nv_bfloat16 *row, int64_t c0, int64_t n
 #pragma unroll
         for (int e = 0; e < 8; ++e)
             if (c0 + e < n) row[c0 + e] = __float2bfloat16_rn(v[e]);
+    }
+}
+
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi)
+{
+    const __half2 h = __floats2half2_rn(lo, hi);              // .x = lo (low half), .y = hi
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+__device__ __forceinline__ void store8(__half *row, int64_t c0, int64_t n, bool vec, const float v[8])
+{
+    if (vec && c0 + 8 <= n) {
+        uint4 o;
+        o.x = pack_f16x2(v[0], v[1]); o.y = pack_f16x2(v[2], v[3]);
+        o.z = pack_f16x2(v[4], v[5]); o.w = pack_f16x2(v[6], v[7]);
+        __stcs(reinterpret_cast<uint4 *>(row + c0), o);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if (c0 + e < n) row[c0 + e] = __float2half_rn(v[e]);
     }
 }
 
@@ -315,9 +353,9 @@ int launch_forward_fma(const lordba_proj *projs, const int64_t *tokens, int n, i
             const bool take = (i < n) && tokens[i] > 0 && padded_rank(projs[i].r) == rp;
             if (take) { b.tokens[m] = tokens[i]; b.p[m++] = projs[i]; }
             if (m == kMaxBatch || (i == n && m > 0)) {
-                const cudaError_t e = (dtype == LORDBA_F32)
-                                          ? launch_rank<float>(b, m, rp, stream)
-                                          : launch_rank<__nv_bfloat16>(b, m, rp, stream);
+                const cudaError_t e = (dtype == LORDBA_F32)    ? launch_rank<float>(b, m, rp, stream)
+                                      : (dtype == LORDBA_F16) ? launch_rank<__half>(b, m, rp, stream)
+                                                              : launch_rank<__nv_bfloat16>(b, m, rp, stream);
                 if (e != cudaSuccess) return LORDBA_ECUDA;
                 m = 0;
             }

@@ -48,6 +48,7 @@
 // the kernel runs to its end.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <cstdlib>
 #include <cstring>
@@ -80,7 +81,7 @@ struct alignas(64) MmaProj {
     CUtensorMap pa_map;    // u32 (16, d_in r / 512), box 16 x 2r: the sign bytes of an x item
     CUtensorMap pb_map;    // u32 (16, d_out r / 512), box 16 x (cwy r / 512)
     const float *s_r;
-    __nv_bfloat16 *y;
+    uint16_t *y;           // 16-bit elements: bfloat16 or half
     int64_t ldy;
     int64_t T;             // token rows of this projection (projections of a launch may differ)
     int d_in, d_out, r;
@@ -220,6 +221,15 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 "
+                 "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
@@ -235,7 +245,22 @@ __device__ __forceinline__ void split2(float v0, float v1, uint32_t &hi, uint32_
     lo = pack2(v0 - lo_f(hi), v1 - hi_f(hi));
 }
 
-// Sign bits (bit 1 = +1) -> sign-flip masks of bf16 pairs.  b holds sign bits in its low byte
+// The same for IEEE halves.  The low parts go subnormal for |v| below about 2^-3 and then keep an
+// absolute precision of 2^-25: still beyond what a half-precision output can show.
+__device__ __forceinline__ uint32_t pack2h(float lo, float hi)
+{
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+__device__ __forceinline__ float2 unpack2h(uint32_t w) { return __half22float2(*reinterpret_cast<const __half2 *>(&w)); }
+__device__ __forceinline__ void split2h(float v0, float v1, uint32_t &hi, uint32_t &lo)
+{
+    hi = pack2h(v0, v1);
+    const float2 h = unpack2h(hi);
+    lo = pack2h(v0 - h.x, v1 - h.y);
+}
+
+// Sign bits (bit 1 = +1) -> sign-flip masks of bf16 (or half) pairs.  b holds sign bits in its low byte
 // (nothing above bit 7); pair p takes bits 2p and 2p+1.  b * (2^(15-2p) + 2^(30-2p)) is two
 // disjoint shifted copies of b that put bit 2p at position 15 and bit 2p+1 at position 31; the
 // caller keeps only those two positions, inverted (a 0 bit flips the sign).
@@ -266,11 +291,20 @@ __device__ __forceinline__ uint64_t b_row_bits(const uint8_t *bits, int j_local,
     return v;
 }
 
+// Element type of x and y, and how s_in enters the first product.
+enum IoKind {
+    kIoBf16 = 0,      // bfloat16; s_in as a bf16 hi + lo pair (two passes over the tensor cores)
+    kIoF16 = 1,       // IEEE half; s_in as a half hi + lo pair (two passes)
+    kIoF16Exact = 2   // IEEE half; s_in stated to be exact in half precision: one pass
+};
+
 // RP: rank padded to 8, 16, 32 or 64.
-template <int RP, int NW, int ELL>
+template <int RP, int NW, int ELL, int IO>
 __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 2)
 mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant__ MmaParams prm)
 {
+    constexpr bool kHalf = (IO != kIoBf16);     // x, y and the first product's operands are halves
+    constexpr bool kLoPass = (IO != kIoF16Exact);
     constexpr int R8 = RP / 8;                 // 8-row blocks of A_sign = n-blocks of the first product
     constexpr int KS = (RP + 15) / 16;         // k-steps of the second product per z part
     constexpr int ZP = KS * 8;                 // bf16 pairs per token row of z
@@ -410,15 +444,20 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     {
                         const float2 sc = *reinterpret_cast<const float2 *>(slot + plan.off_scale +
                                                                             4 * (env * cwx + gcol + 2 * lane));
-                        split2(sc.x, sc.y, ph, pl);
+                        if (kHalf) split2h(sc.x, sc.y, ph, pl);
+                        else split2(sc.x, sc.y, ph, pl);
                     }
                     uint32_t hA[4], hB[4], lA[4], lB[4];
 #pragma unroll
                     for (int p = 0; p < 4; ++p) {
                         hA[p] = __shfl_sync(0xffffffffu, ph, 8 * q + p);
                         hB[p] = __shfl_sync(0xffffffffu, ph, 8 * q + 4 + p);
-                        lA[p] = __shfl_sync(0xffffffffu, pl, 8 * q + p);
-                        lB[p] = __shfl_sync(0xffffffffu, pl, 8 * q + 4 + p);
+                        if (kLoPass) {
+                            lA[p] = __shfl_sync(0xffffffffu, pl, 8 * q + p);
+                            lB[p] = __shfl_sync(0xffffffffu, pl, 8 * q + 4 + p);
+                        } else {
+                            lA[p] = lB[p] = 0u;
+                        }
                     }
                     // k-step outermost, rank blocks innermost: consecutive MMAs go to different
                     // accumulators, so none waits for the one before it
@@ -430,10 +469,21 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                         for (int a = 0; a < R8; ++a) {
                             const uint32_t b = (ks < 2) ? (bytes[a] & 0xffu) : (bytes[a] >> 8);
                             const uint32_t m0 = pair_bits(b, 2 * (ks & 1)), m1 = pair_bits(b, 2 * (ks & 1) + 1);
-                            mma_bf16(acc[env][0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
-                                     with_signs(h0, m0), with_signs(h1, m1));
-                            mma_bf16(acc[env][kSplitAcc ? 1 : 0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
-                                     with_signs(l0, m0), with_signs(l1, m1));
+                            if (!kHalf) {
+                                mma_bf16(acc[env][0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                         with_signs(h0, m0), with_signs(h1, m1));
+                                mma_bf16(acc[env][kSplitAcc ? 1 : 0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                         with_signs(l0, m0), with_signs(l1, m1));
+                            } else if (kLoPass) {
+                                mma_f16(acc[env][0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                        with_signs(h0, m0), with_signs(h1, m1));
+                                mma_f16(acc[env][kSplitAcc ? 1 : 0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                        with_signs(l0, m0), with_signs(l1, m1));
+                            } else {
+                                // one pass: alternate k-steps between the two accumulator sets
+                                mma_f16(acc[env][kSplitAcc ? (ks & 1) : 0][a], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3],
+                                        with_signs(h0, m0), with_signs(h1, m1));
+                            }
                         }
                     }
                 }
@@ -502,8 +552,8 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         };
         uint32_t zh[KS][4], zl[KS][4];
         if (ELL == 1) load_z(0, zh, zl);
-        __nv_bfloat16 *yrow0 = P.y + (t0 + g) * P.ldy;
-        __nv_bfloat16 *yrow1 = yrow0 + 8 * P.ldy;
+        uint16_t *yrow0 = P.y + (t0 + g) * P.ldy;
+        uint16_t *yrow1 = yrow0 + 8 * P.ldy;
         const bool vec32 = P.y_vec32 != 0;
 
         for (; it < n_items; ++it) {
@@ -548,8 +598,14 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                         const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            vs[half][2 * i] = lo_f(yw[i]);
-                            vs[half][2 * i + 1] = hi_f(yw[i]);
+                            if (kHalf) {
+                                const float2 f = unpack2h(yw[i]);
+                                vs[half][2 * i] = f.x;
+                                vs[half][2 * i + 1] = f.y;
+                            } else {
+                                vs[half][2 * i] = lo_f(yw[i]);
+                                vs[half][2 * i + 1] = hi_f(yw[i]);
+                            }
                         }
                     }
 #pragma unroll
@@ -593,12 +649,13 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     for (int half = 0; half < 2; ++half)
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            out[half][4 * cc + i] = pack2(vs[half][2 * i], vs[half][2 * i + 1]);
+                            out[half][4 * cc + i] = kHalf ? pack2h(vs[half][2 * i], vs[half][2 * i + 1])
+                                                          : pack2(vs[half][2 * i], vs[half][2 * i + 1]);
                 }
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     if (half == 0 ? v0 : v1) {
-                        __nv_bfloat16 *dst = (half == 0 ? yrow0 : yrow1) + col0 + gcol + 16 * q;
+                        uint16_t *dst = (half == 0 ? yrow0 : yrow1) + col0 + gcol + 16 * q;
                         const uint32_t oa[4] = {out[half][0], out[half][1], out[half][2], out[half][3]};
                         const uint32_t ob[4] = {out[half][4], out[half][5], out[half][6], out[half][7]};
                         if (vec32) {
@@ -702,13 +759,13 @@ int sm_count()
     return n;
 }
 
-template <int RP, int NW, int ELL>
+template <int RP, int NW, int ELL, int IO>
 cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem, cudaStream_t stream)
 {
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, []() {
-        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW, ELL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW, ELL, IO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSmemBudget);
     });
     if (attr_rc != cudaSuccess) return attr_rc;
@@ -727,14 +784,39 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP, NW, ELL>, b, prm);
+    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP, NW, ELL, IO>, b, prm);
+}
+
+template <int NW, int ELL, int IO>
+cudaError_t launch_rank(int rp, const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem, cudaStream_t stream)
+{
+    switch (rp) {
+        case 8:  return launch_one<8, NW, ELL, IO>(b, prm, grid, smem, stream);
+        case 16: return launch_one<16, NW, ELL, IO>(b, prm, grid, smem, stream);
+        case 32: return launch_one<32, NW, ELL, IO>(b, prm, grid, smem, stream);
+        default:
+            // two envelopes at rank 64 do not fit the register budget: mma_supported() keeps them out
+            if (ELL == 1) return launch_one<64, NW, 1, IO>(b, prm, grid, smem, stream);
+            return cudaErrorInvalidValue;
+    }
+}
+
+template <int IO>
+cudaError_t launch_io(int rp, int nw, int ell, const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem,
+                      cudaStream_t stream)
+{
+    if (ell == 1)
+        return nw == kMaxWarps ? launch_rank<kMaxWarps, 1, IO>(rp, b, prm, grid, smem, stream)
+                               : launch_rank<8, 1, IO>(rp, b, prm, grid, smem, stream);
+    return nw == kMaxWarps ? launch_rank<kMaxWarps, 2, IO>(rp, b, prm, grid, smem, stream)
+                           : launch_rank<8, 2, IO>(rp, b, prm, grid, smem, stream);
 }
 
 }  // namespace
 
 bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
 {
-    if (dtype != LORDBA_BF16 || T < 1 || T > (1 << 30)) return false;
+    if ((dtype != LORDBA_BF16 && dtype != LORDBA_F16) || T < 1 || T > (1 << 30)) return false;
     const int ell = ((p.flags >> 8) & 0xf) + 1;
     if (ell > 2 || (ell == 2 && p.r > 32)) return false;    // more envelopes, or two at high rank: FMA kernel
     if (p.r % 8 != 0 || p.r < 8 || p.r > kMaxRank) return false;
@@ -753,13 +835,21 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                        bool batch_checked)
 {
     if (n == 0) return LORDBA_OK;
-    if (dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    if (dtype != LORDBA_BF16 && dtype != LORDBA_F16) return LORDBA_EUNSUPPORTED;
     int *status = device_status_word();
     if (!status) return LORDBA_ECUDA;
     const int sms = sm_count();
     bool all_overlap = true;          // the caller's promise covers the call only if every projection carries it
     for (int i = 0; i < n; ++i) all_overlap = all_overlap && (projs[i].flags & LORDBA_PROJ_OVERLAP);
     int launches = 0;
+    // one launch per (element / scale kind, envelopes, padded rank) present in the call
+    const int io_first = (dtype == LORDBA_BF16) ? kIoBf16 : kIoF16;
+    const int io_last = (dtype == LORDBA_BF16) ? kIoBf16 : kIoF16Exact;
+    auto io_of = [&](const lordba_proj &q) {
+        if (dtype == LORDBA_BF16) return (int)kIoBf16;
+        return (q.flags & LORDBA_PROJ_SCALES_F16) ? (int)kIoF16Exact : (int)kIoF16;
+    };
+    for (int io = io_first; io <= io_last; ++io)
     for (int ell = 1; ell <= 2; ++ell)
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
         const lordba_proj *sel[kMaxBatch];
@@ -768,7 +858,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
         int64_t min_dout = (int64_t)1 << 40;
         for (int i = 0; i <= n; ++i) {
             const bool take = (i < n) && tokens[i] > 0 && padded_rank(projs[i].r) == rp &&
-                              ((projs[i].flags >> 8) & 0xf) + 1 == ell;
+                              ((projs[i].flags >> 8) & 0xf) + 1 == ell && io_of(projs[i]) == io;
             if (take) {
                 sel_T[m] = tokens[i];
                 sel[m++] = &projs[i];
@@ -824,7 +914,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                                          q.d_out * q.r / 512, cw * q.r / 512))
                         return LORDBA_ECUDA;
                     t.s_r = q.s_r;
-                    t.y = static_cast<__nv_bfloat16 *>(q.y);
+                    t.y = static_cast<uint16_t *>(q.y);
                     t.ldy = q.ldy;
                     t.T = sel_T[k];
                     t.d_in = (int)q.d_in; t.d_out = (int)q.d_out; t.r = q.r;
@@ -845,34 +935,10 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                 if (plan.total > kSmemBudget) return LORDBA_ECUDA;
                 prm.slots = slots;
                 const dim3 grid((unsigned)tiles, (unsigned)m, (unsigned)splits);
-                cudaError_t e;
-                if (ell == 1 && nw == kMaxWarps) {
-                    switch (rp) {
-                        case 8:  e = launch_one<8, 16, 1>(b, prm, grid, plan.total, stream); break;
-                        case 16: e = launch_one<16, 16, 1>(b, prm, grid, plan.total, stream); break;
-                        case 32: e = launch_one<32, 16, 1>(b, prm, grid, plan.total, stream); break;
-                        default: e = launch_one<64, 16, 1>(b, prm, grid, plan.total, stream); break;
-                    }
-                } else if (ell == 1) {
-                    switch (rp) {
-                        case 8:  e = launch_one<8, 8, 1>(b, prm, grid, plan.total, stream); break;
-                        case 16: e = launch_one<16, 8, 1>(b, prm, grid, plan.total, stream); break;
-                        case 32: e = launch_one<32, 8, 1>(b, prm, grid, plan.total, stream); break;
-                        default: e = launch_one<64, 8, 1>(b, prm, grid, plan.total, stream); break;
-                    }
-                } else if (nw == kMaxWarps) {
-                    switch (rp) {
-                        case 8:  e = launch_one<8, 16, 2>(b, prm, grid, plan.total, stream); break;
-                        case 16: e = launch_one<16, 16, 2>(b, prm, grid, plan.total, stream); break;
-                        default: e = launch_one<32, 16, 2>(b, prm, grid, plan.total, stream); break;
-                    }
-                } else {
-                    switch (rp) {
-                        case 8:  e = launch_one<8, 8, 2>(b, prm, grid, plan.total, stream); break;
-                        case 16: e = launch_one<16, 8, 2>(b, prm, grid, plan.total, stream); break;
-                        default: e = launch_one<32, 8, 2>(b, prm, grid, plan.total, stream); break;
-                    }
-                }
+                const cudaError_t e =
+                    io == kIoBf16 ? launch_io<kIoBf16>(rp, nw, ell, b, prm, grid, plan.total, stream)
+                    : io == kIoF16 ? launch_io<kIoF16>(rp, nw, ell, b, prm, grid, plan.total, stream)
+                                   : launch_io<kIoF16Exact>(rp, nw, ell, b, prm, grid, plan.total, stream);
                 if (e != cudaSuccess) return LORDBA_ECUDA;
                 count_launch();
                 m = 0; max_r = 0; min_dout = (int64_t)1 << 40;

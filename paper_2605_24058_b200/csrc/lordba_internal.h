@@ -28,6 +28,7 @@ int *device_status_word();
 // --- pack.cu ---------------------------------------------------------------
 int launch_pack(const int8_t *signs, int64_t rows, int64_t cols, int role, uint32_t *packed,
                 cudaStream_t stream);
+int launch_widen_scales(const uint16_t *src, float *dst, int64_t n, cudaStream_t stream);
 int launch_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int role, int8_t *signs,
                   cudaStream_t stream);
 

@@ -5,6 +5,8 @@
 // Role 0 (A carrier, r x d_in) is block-major: for every block of 64 columns,
 // r consecutive 64-bit groups (two words each, low word first), one per row.
 // sign(0) = +1: an entry packs as bit 0 only when it is negative.
+#include <cuda_fp16.h>
+
 #include "lordba_internal.h"
 
 namespace lordba {
@@ -59,6 +61,15 @@ unpack_kernel(const uint32_t *__restrict__ packed, int64_t rows, int64_t cols, i
     }
 }
 
+// Exported adapters store their scales as IEEE halves; the forward kernels take float32.
+__global__ void __launch_bounds__(kPackThreads)
+widen_scales_kernel(const __half *__restrict__ src, float *__restrict__ dst, int64_t n)
+{
+    const int64_t stride = (int64_t)gridDim.x * kPackThreads;
+    for (int64_t e = (int64_t)blockIdx.x * kPackThreads + threadIdx.x; e < n; e += stride)
+        dst[e] = __half2float(src[e]);
+}
+
 int grid_for(int64_t work_items, int per_block)
 {
     int64_t blocks = (work_items + per_block - 1) / per_block;
@@ -78,6 +89,15 @@ int launch_pack(const int8_t *signs, int64_t rows, int64_t cols, int role, uint3
     if (words == 0) return LORDBA_OK;
     pack_kernel<<<grid_for(words, kPackThreads / 32), kPackThreads, 0, stream>>>(signs, prow, pcols, role,
                                                                                 words, packed);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? LORDBA_OK : LORDBA_ECUDA;
+}
+
+int launch_widen_scales(const uint16_t *src, float *dst, int64_t n, cudaStream_t stream)
+{
+    if (n == 0) return LORDBA_OK;
+    widen_scales_kernel<<<grid_for(n, kPackThreads), kPackThreads, 0, stream>>>(
+        reinterpret_cast<const __half *>(src), dst, n);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LORDBA_OK : LORDBA_ECUDA;
 }

@@ -16,9 +16,10 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "liblordba.so")
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 VARIANT_AUTO, VARIANT_FMA, VARIANT_TC, VARIANT_MMA = 0, 1, 2, 3
 PROJ_OVERLAP = 1
+PROJ_SCALES_F16 = 2
 MAX_ELL = 8
 
 
@@ -47,6 +48,7 @@ _SIGNATURES = {
     "lordba_packed_words": (_i64, [_i64, _i64, ctypes.c_int]),
     "lordba_pack_signs": (ctypes.c_int, [_vp, _i64, _i64, ctypes.c_int, _vp, _vp]),
     "lordba_unpack_signs": (ctypes.c_int, [_vp, _i64, _i64, ctypes.c_int, _vp, _vp]),
+    "lordba_scales_from_f16": (ctypes.c_int, [_vp, _vp, _i64, _vp]),
     "lordba_adapter_forward": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int, _vp]),
     "lordba_adapter_forward_f32": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int, _vp]),
     "lordba_adapter_forward_ell": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int, ctypes.c_int,
@@ -116,7 +118,9 @@ def _dtype_code(t: torch.Tensor) -> int:
         return F32
     if t.dtype == torch.bfloat16:
         return BF16
-    raise TypeError("x and y must be float32 or bfloat16, got %s" % t.dtype)
+    if t.dtype == torch.float16:
+        return F16
+    raise TypeError("x and y must be float32, bfloat16 or float16, got %s" % t.dtype)
 
 
 def _need_cuda(*tensors: torch.Tensor) -> None:
@@ -156,6 +160,17 @@ def unpack_signs(packed: torch.Tensor, rows: int, cols: int, role: int, stream=N
     return signs
 
 
+def scales_from_f16(scales: torch.Tensor, stream=None) -> torch.Tensor:
+    """float16 scales of an exported adapter (device) -> the float32 tensor the forward calls take."""
+    _need_cuda(scales)
+    if scales.dtype != torch.float16 or not scales.is_contiguous():
+        raise ValueError("scales must be a contiguous float16 tensor")
+    out = torch.empty(scales.shape, dtype=torch.float32, device=scales.device)
+    _check(load().lordba_scales_from_f16(scales.data_ptr(), out.data_ptr(), scales.numel(), _stream(stream)),
+           "lordba_scales_from_f16")
+    return out
+
+
 def make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, flags: int = 0) -> Proj:
     """Fill a ``lordba_proj`` from 2-D (possibly row-strided) x, y and 1-D parameter tensors."""
     _need_cuda(x, packed_A, packed_B, s_in, s_r, s_out, y)
@@ -184,14 +199,16 @@ def make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, flags: int = 0
 
 
 def adapter_forward(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, stream=None,
-                    overlap: bool = False) -> None:
+                    overlap: bool = False, scales_f16: bool = False) -> None:
     """y += adapter(x) in place, through lordba_adapter_forward{,_f32} (dense rows)
-    or lordba_adapter_forward_ex (row-strided x / y, or overlap=True: the caller's promise
-    LORDBA_PROJ_OVERLAP that this call is independent of the run of calls before it)."""
-    p = make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r, PROJ_OVERLAP if overlap else 0)
+    or lordba_adapter_forward_ex (row-strided x / y, float16, or a flag: overlap=True is the
+    caller's promise LORDBA_PROJ_OVERLAP that this call is independent of the run of calls before
+    it, scales_f16=True the statement LORDBA_PROJ_SCALES_F16 that s_in holds float16 values)."""
+    flags = (PROJ_OVERLAP if overlap else 0) | (PROJ_SCALES_F16 if scales_f16 else 0)
+    p = make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r, flags)
     T = x.shape[0]
     lib = load()
-    dense = x.is_contiguous() and y.is_contiguous() and not overlap
+    dense = x.is_contiguous() and y.is_contiguous() and flags == 0
     if dense and x.dtype == torch.bfloat16:
         rc = lib.lordba_adapter_forward(p.x, p.packed_A, p.packed_B, p.s_in, p.s_r, p.s_out, p.y,
                                         T, p.d_in, p.d_out, r, _stream(stream))

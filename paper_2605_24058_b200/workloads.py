@@ -40,7 +40,7 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 @dataclass
 class Projection:
     """One adapted projection's inputs.  ``x``/``y`` are float32 arrays for
-    dtype "f32" and uint16 bfloat16 bit patterns for dtype "bf16"."""
+    dtype "f32", uint16 bfloat16 bit patterns for dtype "bf16" and float16 arrays for "f16"."""
     name: str
     d_in: int
     d_out: int
@@ -70,16 +70,19 @@ class Projection:
 
 def make_projection(d_in: int, d_out: int, r: int, T: int, dtype: str, seed: int,
                     scales: str = "llama", outlier_frac: float = 0.0,
-                    outlier_gain: float = 20.0, name: str = "proj") -> Projection:
+                    outlier_gain: float = 20.0, name: str = "proj",
+                    scales_f16: bool = False) -> Projection:
     """Draw one projection's inputs.
 
     scales="tiny":  s_in, s_r, s_out = exp(N(0, 0.5))            (the tiny fp32 case)
     scales="llama": s_in, s_out = exp(N(0, 0.5)); s_r = 64*|N(0, 0.02)|
     (0.5 and 0.02 are standard deviations; 64 = sqrt(4096) for every shape.)
     outlier_frac > 0 multiplies that fraction of input channels of x by outlier_gain.
+    scales_f16 rounds the three scale vectors to float16 values (an adapter exported in fp16);
+    they stay float32 arrays.
     """
-    if dtype not in ("f32", "bf16"):
-        raise ValueError("dtype must be 'f32' or 'bf16'")
+    if dtype not in ("f32", "bf16", "f16"):
+        raise ValueError("dtype must be 'f32', 'bf16' or 'f16'")
     rng = np.random.default_rng(seed)
     x = rng.standard_normal((T, d_in), dtype=np.float32)
     if outlier_frac > 0.0:
@@ -100,8 +103,13 @@ def make_projection(d_in: int, d_out: int, r: int, T: int, dtype: str, seed: int
     if dtype == "bf16":
         x = to_bf16_bits(x)
         y = to_bf16_bits(y)
+    elif dtype == "f16":
+        x = x.astype(np.float16)            # IEEE round to nearest even
+        y = y.astype(np.float16)
+    if scales_f16:
+        s_in, s_r, s_out = (s.astype(np.float16).astype(np.float32) for s in (s_in, s_r, s_out))
     return Projection(name, d_in, d_out, r, T, dtype, x, y, A_sign, B_sign, s_in, s_r, s_out,
-                      {"seed": seed, "scales": scales, "outlier_frac": outlier_frac})
+                      {"seed": seed, "scales": scales, "outlier_frac": outlier_frac, "scales_f16": scales_f16})
 
 
 def config0() -> Projection:

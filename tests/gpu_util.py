@@ -20,11 +20,21 @@ BF16_RAW_BOUND_REGION = 5.0
 # 2^-12 rms(y') for everything before it (split bf16 operands, fp32 summation order).
 BF16_HALF_ULP = 2.0 ** -8
 BF16_PRE_ROUNDING = 2.0 ** -12
+# float16 I/O (no bound is stated for it; derived from the arithmetic): half an ulp of the exact
+# result for the one final rounding (2^-11 |y'|) plus 2^-13 rms(y') for everything before it.  The
+# inexact steps before the rounding are s_in as a pair of halves (2^-22 relative), float32
+# summation, and z = s_r u as a bfloat16 pair: up to 2^-17 relative per rank term, r terms in
+# quadrature, times s_out[j], whose tail is heavy.  Over the 8 M outputs of a full-size call the
+# largest such error was measured at 2^-15 rms(y'); the bound leaves a factor of four.
+F16_HALF_ULP = 2.0 ** -11
+F16_PRE_ROUNDING = 2.0 ** -13
 
 
 def np_to_torch(a: np.ndarray, dtype: str, device) -> torch.Tensor:
     if dtype == "bf16":
         return torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).to(device)
+    if dtype == "f16":
+        return torch.from_numpy(a.view(np.int16).copy()).view(torch.float16).to(device)
     return torch.from_numpy(a.copy()).to(device)
 
 
@@ -59,13 +69,16 @@ class DeviceProj:
             self.packed_A = torch.from_numpy(oracle.pack_signs(p.A_sign, 0).view(np.int32)).to(dev)
             self.packed_B = torch.from_numpy(oracle.pack_signs(p.B_sign, 1).view(np.int32)).to(dev)
 
+    def flags(self) -> int:
+        return lordba.PROJ_SCALES_F16 if self.p.meta.get("scales_f16") else 0
+
     def proj(self) -> lordba.Proj:
         return lordba.make_proj(self.x, self.packed_A, self.packed_B, self.s_in, self.s_r,
-                                self.s_out, self.y, self.p.r)
+                                self.s_out, self.y, self.p.r, self.flags())
 
     def forward(self):
         lordba.adapter_forward(self.x, self.packed_A, self.packed_B, self.s_in, self.s_r,
-                               self.s_out, self.y, self.p.r)
+                               self.s_out, self.y, self.p.r, scales_f16=bool(self.flags()))
 
     def reset_y(self):
         self.y.copy_(np_to_torch(self.p.y, self.p.dtype, self.y.device))
@@ -88,6 +101,12 @@ def assert_close(got: np.ndarray, want: np.ndarray, dtype: str, what: str = "", 
     if dtype == "f32":
         bound = F32_REL_INF * np.abs(ref).max()
         assert err.max() <= bound, "%s: max err %.3e > %.3e" % (what, err.max(), bound)
+    elif dtype == "f16":
+        rms = float(np.sqrt(np.mean(ref * ref)))
+        tight = F16_HALF_ULP * np.abs(want) + F16_PRE_ROUNDING * rms
+        bad = err > tight
+        assert not bad.any(), "%s: %d elements beyond the f16 rounding bound, worst %.3e vs %.3e" % (
+            what, int(bad.sum()), float(err[bad].max()), float(tight[bad].min()))
     else:
         rms = float(np.sqrt(np.mean(ref * ref)))
         bound = BF16_REL_RMS * rms

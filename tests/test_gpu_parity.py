@@ -192,7 +192,7 @@ SHAPES = [
 
 
 @pytest.mark.parametrize("T,d_in,d_out,r", SHAPES)
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("vname,variant", VARIANTS)
 @skip_unsupported
 def test_shapes_every_element(oracle, T, d_in, d_out, r, dtype, vname, variant):
@@ -204,7 +204,7 @@ def test_shapes_every_element(oracle, T, d_in, d_out, r, dtype, vname, variant):
                  "shape %s %s %s" % ((T, d_in, d_out, r), dtype, vname))
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("ldx_pad,ldy_pad", [(8, 16), (3, 5), (64, 0), (0, 24)])
 @pytest.mark.parametrize("vname,variant", VARIANTS)
 @skip_unsupported
@@ -255,7 +255,7 @@ def test_empty_batch_and_zero_tokens():
 
 # ---------------------------------------------------------------- properties the method fixes
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("vname,variant", VARIANTS)
 @skip_unsupported
 def test_canonical_adapter_is_integer_exact(oracle, dtype, vname, variant):
@@ -267,8 +267,8 @@ def test_canonical_adapter_is_integer_exact(oracle, dtype, vname, variant):
     p = workloads.make_projection(d_in, d_out, r, T, dtype, seed=5, scales="tiny")
     xi = rng.integers(-2, 3, size=(T, d_in)).astype(np.float32)
     yi = rng.integers(-8, 9, size=(T, d_out)).astype(np.float32)
-    p.x = workloads.to_bf16_bits(xi) if dtype == "bf16" else xi
-    p.y = workloads.to_bf16_bits(yi) if dtype == "bf16" else yi
+    p.x = workloads.to_bf16_bits(xi) if dtype == "bf16" else xi.astype(np.float16) if dtype == "f16" else xi
+    p.y = workloads.to_bf16_bits(yi) if dtype == "bf16" else yi.astype(np.float16) if dtype == "f16" else yi
     p.s_in = np.ones(d_in, np.float32)
     p.s_out = np.ones(d_out, np.float32)
     p.s_r = np.full(r, 2.0 ** -6, np.float32)
@@ -277,6 +277,9 @@ def test_canonical_adapter_is_integer_exact(oracle, dtype, vname, variant):
         # keep only outputs that a bf16 can hold exactly (|v| * 64 an integer below 2^8)
         exact = np.abs(want * 64) <= 255
         assert exact.mean() > 0.2
+    elif dtype == "f16":
+        exact = np.abs(want * 64) <= 2047            # 11 significant bits
+        assert exact.mean() > 0.9
     else:
         exact = np.ones_like(want, bool)
     d = DeviceProj(p)
@@ -285,7 +288,7 @@ def test_canonical_adapter_is_integer_exact(oracle, dtype, vname, variant):
     assert np.array_equal(got[exact], want[exact])
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("vname,variant", VARIANTS)
 @skip_unsupported
 def test_zero_rank_scale_leaves_y_untouched_and_runs_are_deterministic(oracle, dtype, vname, variant):
@@ -379,11 +382,11 @@ def _ell_inputs(d_in, d_out, r, T, dtype, ell, seed):
     return base, s_in, s_r, s_out
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("T,d_in,d_out,r,ell", [(70, 256, 192, 8, 2), (300, 1024, 768, 16, 2), (33, 200, 136, 24, 3),
                                                 (150, 4096, 1024, 16, 4), (2048, 4096, 4096, 16, 2)])
 def test_multi_envelope_forward(oracle, dtype, T, d_in, d_out, r, ell):
-    if dtype == "f32" and T > 1000:
+    if dtype != "bf16" and T > 1000:
         pytest.skip("full-size case is checked in bf16 only")
     base, s_in, s_r, s_out = _ell_inputs(d_in, d_out, r, T, dtype, ell, seed=90 + ell + r)
     d = DeviceProj(base)
@@ -467,3 +470,83 @@ def test_adjoint_is_a_forward_with_swapped_carriers(oracle):
                                 p.s_out.astype(np.float64), np.zeros((T, d_out)))
     lhs, rhs = float((dy64 * fx).sum()), float((want * p.x_f64()).sum())
     assert abs(lhs - rhs) <= 1e-9 * max(abs(lhs), abs(rhs))
+
+
+# ---------------------------------------------------------------- the export precision: float16
+
+def test_scales_from_f16_is_exact():
+    """Every half widens to the same float: subnormals, zeros, infinities and the largest finite value included."""
+    rng = np.random.default_rng(5)
+    bits = rng.integers(0, 1 << 16, size=5000, dtype=np.uint16)
+    bits[:8] = [0x0000, 0x8000, 0x0001, 0x03ff, 0x0400, 0x7bff, 0x7c00, 0xfc00]
+    h = bits.view(np.float16)
+    keep = ~np.isnan(h)                          # NaN payloads are not compared
+    dev = torch.from_numpy(bits.view(np.int16).copy()).view(torch.float16).cuda()
+    got = lordba.scales_from_f16(dev).cpu().numpy()
+    want = h.astype(np.float32)
+    assert got.dtype == np.float32
+    assert np.array_equal(got[keep].view(np.uint32), want[keep].view(np.uint32))
+    assert np.isnan(got[~keep]).all()
+    assert lordba.scales_from_f16(dev[:0]).numel() == 0
+
+
+@pytest.mark.parametrize("r", [8, 16, 32, 64])
+@pytest.mark.parametrize("scales_f16", [False, True])
+def test_f16_activations_attention_full_size(oracle, r, scales_f16):
+    """The attention projection at T = 2048 with float16 x and y: float32 scales (s_in as a pair of
+    halves) and an adapter exported with float16 scales (one pass, flagged), every element."""
+    p = workloads.make_projection(4096, 4096, r, 2048, "f16", seed=1000 + r, scales_f16=scales_f16)
+    d = DeviceProj(p)
+    assert d.flags() == (lordba.PROJ_SCALES_F16 if scales_f16 else 0)
+    d.forward()
+    assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "f16", "f16 attn r=%d exported=%s" % (r, scales_f16))
+
+
+def test_f16_exported_adapter_loaded_from_half_storage(oracle):
+    """An adapter stored with half-precision scales: widened by the library, used flagged and
+    unflagged; both agree with the oracle run on the same half values."""
+    p = workloads.make_projection(1024, 1536, 16, 333, "f16", seed=77, scales_f16=True)
+    d = DeviceProj(p)
+    for name in ("s_in", "s_r", "s_out"):
+        stored = torch.from_numpy(getattr(p, name).astype(np.float16).view(np.int16).copy()).view(torch.float16).cuda()
+        widened = lordba.scales_from_f16(stored)
+        assert torch.equal(widened, getattr(d, name))
+        setattr(d, name, widened)
+    want = oracle_forward(oracle, p)
+    for flagged in (True, False):
+        d.reset_y()
+        lordba.adapter_forward(d.x, d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, d.y, p.r, scales_f16=flagged)
+        assert_close(torch_to_f64(d.y), want, "f16", "exported adapter, flagged=%s" % flagged)
+
+
+@pytest.mark.parametrize("c", [2.0 ** -8, 2.0 ** 6])
+def test_f16_scale_gauge(oracle, c):
+    """(c s_in, s_r / c, s_out) is the same adapter (c a power of two): small and large s_in
+    stay within the float16 bound although s_in enters the tensor cores as halves."""
+    p = workloads.make_projection(2048, 1024, 16, 200, "f16", seed=91)
+    want = oracle_forward(oracle, p)
+    p.s_in = (p.s_in * np.float32(c)).astype(np.float32)
+    p.s_r = (p.s_r / np.float32(c)).astype(np.float32)
+    d = DeviceProj(p)
+    d.forward()
+    assert_close(torch_to_f64(d.y), want, "f16", "gauge c=%g" % c)
+
+
+def test_f16_mixed_batch_and_segments(oracle):
+    """One batched call with flagged and unflagged projections of different rank, and a segmented call."""
+    ps = [workloads.make_projection(di, do, r, 150, "f16", seed=300 + i, scales_f16=ex)
+          for i, (di, do, r, ex) in enumerate([(512, 768, 16, True), (512, 768, 16, False), (1024, 256, 64, True),
+                                               (200, 136, 24, False)])]
+    ds = [DeviceProj(p) for p in ps]
+    lordba.adapter_forward_batched([d.proj() for d in ds], 150, lordba.F16)
+    for p, d in zip(ps, ds):
+        assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "f16", "f16 batched " + p.name)
+    for d in ds:
+        d.reset_y()
+    tokens = [150, 0, 77, 150]
+    lordba.adapter_forward_segments([d.proj() for d in ds], tokens, lordba.F16)
+    for p, d, n in zip(ps, ds, tokens):
+        got = torch_to_f64(d.y)
+        want = oracle_forward(oracle, p)
+        assert_close(got[:n], want[:n], "f16", "f16 segment " + p.name, scale_from=want)
+        assert np.array_equal(got[n:], p.y_f64()[n:])

@@ -1,5 +1,5 @@
-// Streaming tensor-core kernel of the LoRDBA adapter forward (bf16 activations),
-// Eq. 8 / Eq. 9:
+// Streaming tensor-core kernel of the LoRDBA adapter forward (bf16 or float16
+// activations), Eq. 8 / Eq. 9:
 //
 //   y[t,:] += s_out * ( B_sign ( s_r * ( A_sign ( s_in * x[t,:] ) ) ) )
 //
@@ -37,6 +37,12 @@
 //     parts, so both products carry ~16 mantissa bits into the float32
 //     accumulators.  MMAs are issued k-step outermost, so that consecutive
 //     ones go to different accumulators.
+//   * float16 activations (the precision the method exports adapters in) use
+//     the same kernel with half operands in the first product: s_in as a half
+//     hi/lo pair, or, when the caller states that s_in holds half-precision
+//     values (an adapter exported with fp16 scales), as one half, which halves
+//     the tensor-core work of that product.  z stays a bf16 pair (its range is
+//     not bounded by 65504) and the second product is unchanged.
 //
 // Warps split the d_in axis for the first product (fixed-order reduction
 // through shared memory, hence deterministic) and the d_out axis for the
@@ -714,7 +720,8 @@ bool encode(CUtensorMap *map, CUtensorMapDataType type, int rank, const void *ba
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Row-major T x d bf16 matrix (row pitch ld elements, d % 64 == 0) seen as the 3-D tensor
+// Row-major T x d matrix of 16-bit elements (bf16 or half: the map only moves them; row pitch ld
+// elements, d % 64 == 0) seen as the 3-D tensor
 // (column in group: 64, row: T, column group: d / 64); a box is 64 x 16 rows x `groups`.
 bool make_data_map(CUtensorMap *map, const void *base, int64_t T, int64_t d, int64_t ld, int groups)
 {

@@ -228,9 +228,9 @@ def run_gpu(args):
     # Consecutive steps work on different buffer sets, so every step but the first of a graph is
     # declared independent of the ones before it (LORDBA_PROJ_OVERLAP): its loads may start while
     # the previous step's last tiles are still being written.
-    def step(i):
+    def step(i, dependent=False):
         lordba.adapter_forward(xs[i % n_sets], packed_A, packed_B, s_in, s_r, s_out, ys[i % n_sets], R,
-                               overlap=(i % n_sets != 0) and not args.no_overlap)
+                               overlap=(i % n_sets != 0) and not args.no_overlap and not dependent)
 
     # correctness of the configuration being timed: sampled rows against the oracle (rank 0)
     parity = None
@@ -301,6 +301,24 @@ def run_gpu(args):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1)
 
+        # the same steps as a chain: no step declared independent, each kernel waits for the one
+        # before it (what a caller pays when every call consumes the previous call's output)
+        dep_steps = int(max(n_sets, min(args.steps, 2000) // n_sets * n_sets))
+        dep_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(dep_graph, stream=stream):
+            for i in range(n_sets):
+                step(i, dependent=True)
+        for _ in range(3):
+            dep_graph.replay()
+        stream.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        for _ in range(dep_steps // n_sets):
+            dep_graph.replay()
+        d1.record(stream)
+        stream.synchronize()
+        dep_ms = d0.elapsed_time(d1) / dep_steps
+
         # end to end through the host-buffer entry point: H2D x, H2D y, kernel, D2H y per step
         ws = torch.empty(lordba.host_workspace_bytes(T, D_IN, D_OUT, lordba.BF16), dtype=torch.uint8,
                          device=dev)
@@ -328,7 +346,7 @@ def run_gpu(args):
     if status != 0:
         raise RuntimeError("device status word is %d after the timed region" % status)
 
-    ms, e2e_ms = max_over_ranks([ms, e2e_ms], dev if world > 1 else None)
+    ms, e2e_ms, dep_ms = max_over_ranks([ms, e2e_ms, dep_ms], dev if world > 1 else None)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -361,6 +379,9 @@ def run_gpu(args):
                     "d2h_bytes_per_step": T * D_OUT * ELEM, "steps": e2e_steps},
             "gpu_launches": int(round(launches_per_step * args.steps)),
             "clocks": sampler.summary(),
+            # the same workload with every step waiting for the one before it (not the headline)
+            "dependent_steps": {"ms_per_step": dep_ms, "value": world * T / (dep_ms * 1e-3), "unit": UNIT,
+                                "roofline_frac": alg_bytes / (dep_ms * 1e-3) / 1e9 / peak, "steps": dep_steps},
         }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(p)

@@ -301,6 +301,16 @@ def run_gpu(args):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1)
 
+        # spread of the step time: every replay of the graph (n_sets steps) timed on its own
+        n_spread = int(max(5, min(100, args.steps // n_sets)))
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_spread + 1)]
+        marks[0].record(stream)
+        for k in range(n_spread):
+            graph.replay()
+            marks[k + 1].record(stream)
+        stream.synchronize()
+        spread_us = np.array([marks[k].elapsed_time(marks[k + 1]) for k in range(n_spread)]) * 1e3 / n_sets
+
         # the same steps as a chain: no step declared independent, each kernel waits for the one
         # before it (what a caller pays when every call consumes the previous call's output)
         dep_steps = int(max(n_sets, min(args.steps, 2000) // n_sets * n_sets))
@@ -379,6 +389,10 @@ def run_gpu(args):
                     "d2h_bytes_per_step": T * D_OUT * ELEM, "steps": e2e_steps},
             "gpu_launches": int(round(launches_per_step * args.steps)),
             "clocks": sampler.summary(),
+            # per-step time over single graph replays (this rank): the timed region's figure is the mean
+            "step_us_spread": {"p10": float(np.percentile(spread_us, 10)), "median": float(np.median(spread_us)),
+                               "p90": float(np.percentile(spread_us, 90)), "replays": n_spread,
+                               "steps_per_replay": n_sets},
             # the same workload with every step waiting for the one before it (not the headline)
             "dependent_steps": {"ms_per_step": dep_ms, "value": world * T / (dep_ms * 1e-3), "unit": UNIT,
                                 "roofline_frac": alg_bytes / (dep_ms * 1e-3) / 1e9 / peak, "steps": dep_steps},

@@ -276,6 +276,16 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint6
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// The same with the descriptors as (low, high) words: the issuing thread keeps the high words
+// and the base of the low words in registers and only adds a 16-byte-unit offset per MMA.
+__device__ __forceinline__ void mma_bf16_words(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                               uint32_t b_hi, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %6, 0;\n"
+                 "mov.b64 da, {%1, %2};\nmov.b64 db, {%3, %4};\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -473,56 +483,69 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             }
         } else if (warp == 1) {
             // ================= MMA issuer =================
+            // One thread; its per-chunk latency bounds the whole pipeline (measured: with slot and
+            // phase recomputed from `it` by division and the descriptors rebuilt per MMA, a chunk
+            // cost this thread ~1100 cycles in stage 1 and ~1800 in stage 2, more than the loads).
+            // So: ring positions are carried, descriptor words are precomputed, loops are unrolled.
             if (lane == 0) {
                 const uint32_t idesc1 = instr_desc(kTileM, 2 * r);
                 const uint32_t idesc2 = instr_desc(kTileM, kChunk);
+                const int ksteps2 = kp / 16;
+                // descriptor words (see smem_desc): low = address >> 4 | (lbo >> 4) << 16,
+                // high = sbo >> 4 | version | layout << 29
+                // (a shared address carries the CTA's rank in the cluster above bit 18: masked off)
+                const uint32_t base18 = sm_base & 0x3ffffu;
+                const uint32_t x_lo = (base18 >> 4) | (1u << 16), x_hi = 64u | (1u << 14) | (2u << 29);
+                const uint32_t op_lo = ((base18 + plan.off_ops) >> 4) | (8u << 16);
+                const uint32_t w1_hi = 64u | (1u << 14);
+                const uint32_t z_hi = (uint32_t)(kt8 * 8) | (1u << 14);
+                const uint32_t zhi_lo = ((base18 + plan.off_zhi) >> 4) | (8u << 16);
+                const uint32_t zlo_lo = ((base18 + plan.off_zlo) >> 4) | (8u << 16);
+                const uint32_t slot_units = (uint32_t)plan.slot_stride >> 4, op_units = (uint32_t)plan.op_bytes >> 4;
+                uint32_t s = it % S, ph = (it / S) & 1u, o = it % kOps, oph = (it / kOps) & 1u;
                 for (int c = kb; c < ke; ++c, ++it) {
-                    const int s = it % S; const uint32_t ph = (it / S) & 1u;
-                    const int o = it % kOps; const uint32_t oph = (it / kOps) & 1u;
                     mbar_wait<false>(wctx, bar_full(s), ph, kDevMmaWaitTimeout);
                     mbar_wait<false>(wctx, bar_op_full(o), oph, kDevMmaWaitTimeout);
                     TC_TRACE(1, it, 0);
                     tc_fence_after();
-                    const uint32_t a0 = sm_base + s * plan.slot_stride;       // x tile, 128B swizzle
-                    const uint32_t b0 = sm_base + plan.off_ops + o * plan.op_bytes;   // W1, no swizzle
+                    const uint32_t a_lo = x_lo + s * slot_units;          // x tile, 128B swizzle
+                    const uint32_t b_lo = op_lo + o * op_units;           // W1, no swizzle
 #pragma unroll
-                    for (int ks = 0; ks < kChunk / 16; ++ks) {
-                        const uint64_t ad = smem_desc(a0 + ks * 32, 16, 1024, 2);
-                        const uint64_t bd = smem_desc(b0 + ks * 256, 128, 1024, 0);
-                        mma_bf16(tmem_base + kTmemU, ad, bd, idesc1, (c > kb || ks > 0) ? 1u : 0u);
-                    }
+                    for (int ks = 0; ks < kChunk / 16; ++ks)
+                        mma_bf16_words(tmem_base + kTmemU, a_lo + 2u * ks, x_hi, b_lo + 16u * ks, w1_hi, idesc1,
+                                       (c > kb || ks > 0) ? 1u : 0u);
                     mma_commit(bar_empty(s));
                     mma_commit(bar_op_empty(o));
+                    if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
+                    if (++o == (uint32_t)kOps) { o = 0; oph ^= 1u; }
                 }
                 mma_commit(bar_u_full);
                 mbar_wait<true>(wctx, bar_z_full, tphase, kDevMmaWaitTimeout);
                 TC_TRACE(1, it, 2);
                 fence_proxy_async();
                 tc_fence_after();
-                const uint32_t zhi = sm_base + plan.off_zhi, zlo = sm_base + plan.off_zlo;
-                const uint32_t z_sbo = kt8 * 128;
+                uint32_t vb = vit & 1u, vph = (vit >> 1) & 1u;
                 for (int c = nb; c < ne; ++c, ++it, ++vit) {
-                    const int vb = vit & 1u; const uint32_t vph = (vit >> 1) & 1u;
-                    const int o = it % kOps; const uint32_t oph = (it / kOps) & 1u;
                     mbar_wait<false>(wctx, bar_op_full(o), oph, kDevMmaWaitTimeout);   // the y box is not needed here
                     TC_TRACE(1, it, 0);
                     mbar_wait<false>(wctx, bar_v_empty(vb), vph ^ 1u, kDevMmaWaitTimeout);
                     TC_TRACE(1, it, 1);
                     tc_fence_after();
-                    const uint32_t b0 = sm_base + plan.off_ops + o * plan.op_bytes;   // W2, no swizzle
+                    const uint32_t b_lo = op_lo + o * op_units;           // W2, no swizzle
                     const uint32_t d = tmem_base + kTmemV + vb * kChunk;
-                    uint32_t acc = 0;
-                    for (int half = 0; half < 2; ++half) {
-                        const uint32_t za = half ? zlo : zhi;
-                        for (int ks = 0; ks < kp / 16; ++ks) {
-                            const uint64_t ad = smem_desc(za + ks * 256, 128, z_sbo, 0);
-                            const uint64_t bd = smem_desc(b0 + ks * 256, 128, z_sbo, 0);
-                            mma_bf16(d, ad, bd, idesc2, acc);
-                            acc = 1;
-                        }
-                    }
+#pragma unroll
+                    for (int ks = 0; ks < kMaxRank / 16; ++ks)
+                        if (ks < ksteps2)
+                            mma_bf16_words(d, zhi_lo + 16u * ks, z_hi, b_lo + 16u * ks, z_hi, idesc2, ks > 0 ? 1u : 0u);
+#pragma unroll
+                    for (int ks = 0; ks < kMaxRank / 16; ++ks)
+                        if (ks < ksteps2)
+                            mma_bf16_words(d, zlo_lo + 16u * ks, z_hi, b_lo + 16u * ks, z_hi, idesc2, 1u);
                     mma_commit(bar_v_full(vb));
                     mma_commit(bar_op_empty(o));
+                    if (++o == (uint32_t)kOps) { o = 0; oph ^= 1u; }
+                    vph ^= vb;              // the phase flips when the buffer index wraps from 1 to 0
+                    vb ^= 1u;
                 }
             }
         } else if (warp < 2 + kGenThreads / 32) {

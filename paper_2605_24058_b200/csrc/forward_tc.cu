@@ -102,7 +102,7 @@ __host__ __device__ inline int aux_operand_bytes(int r, int kp)
     return w1 > w2 ? w1 : w2;
 }
 
-__host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile_rows)
+__host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile_rows, int cluster)
 {
     SmemPlan s;
     // The MMA reads 128 rows (16 KiB) from the start of a slot whatever tile_rows is; what lies
@@ -120,7 +120,8 @@ __host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile
     s.off_zhi = s.off_ops + kOps * s.op_bytes;
     s.off_zlo = s.off_zhi + s.z_bytes;
     s.off_rx = s.off_zlo + s.z_bytes;
-    s.off_bar = s.off_rx + kTileM * r * 4;
+    // the exchange buffer for partial u exists only when a cluster splits the feature axes
+    s.off_bar = s.off_rx + (cluster > 1 ? kTileM * r * 4 : 0);
     s.off_misc = s.off_bar + (3 * slots + 2 * kOps + 8) * 8;
     s.total = s.off_misc + 16;
     const int last_read_end = (slots - 1) * s.slot_stride + kTileM * kChunk * 2;
@@ -360,7 +361,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     const int r = B.r, kp = B.kp, S = B.slots, C = B.cluster;
     const int tile_rows = B.tile_rows;
     if (threadIdx.x == 0) TC_TRACE(4, 0, 0);
-    const SmemPlan plan = make_plan(r, kp, S, tile_rows);
+    const SmemPlan plan = make_plan(r, kp, S, tile_rows, C);
     const uint32_t box_bytes = (uint32_t)tile_rows * kChunk * 2;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t crank = cluster_ctarank();
@@ -402,8 +403,8 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
         mbar_init(bar_rx_full, (uint32_t)(2 * tile_rows));   // one arrive per (token row, column half)
         mbar_init(bar_v_full(0), 1);
         mbar_init(bar_v_full(1), 1);
-        mbar_init(bar_v_empty(0), kEpiThreads);
-        mbar_init(bar_v_empty(1), kEpiThreads);
+        mbar_init(bar_v_empty(0), kEpiThreads / 2);      // the epilogue group that reads the buffer
+        mbar_init(bar_v_empty(1), kEpiThreads / 2);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -648,6 +649,34 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             if (e == 0) TC_TRACE(3, it, 5);
             __syncwarp();
             tc_fence_after();
+            if (C == 1) {
+                // no exchange: this thread's pieces of u go straight to z = s_r * u as bf16 hi + lo
+                if (warp_has_rows) {
+                    for (int p = chalf; p < r8; p += 2) {
+                        float h[8], l[8];
+                        tmem_ld8(tlane + kTmemU + p * 8, h);          // warp-collective
+                        tmem_ld8(tlane + kTmemU + r + p * 8, l);
+                        tmem_wait_ld();
+                        if (row_valid) {
+                            uint32_t zh[4], zl[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float z0 = (h[2 * q] + l[2 * q]) * __ldg(P.s_r + p * 8 + 2 * q);
+                                const float z1 = (h[2 * q + 1] + l[2 * q + 1]) * __ldg(P.s_r + p * 8 + 2 * q + 1);
+                                const float h0 = bf16_round(z0), h1 = bf16_round(z1);
+                                zh[q] = pack2_bf16(h0, h1);
+                                zl[q] = pack2_bf16(z0 - h0, z1 - h1);
+                            }
+                            const uint32_t off = (uint32_t)((row >> 3) * (kt8 * 128) + p * 128 + (row & 7) * 16);
+                            *reinterpret_cast<uint4 *>(sm + plan.off_zhi + off) = make_uint4(zh[0], zh[1], zh[2], zh[3]);
+                            *reinterpret_cast<uint4 *>(sm + plan.off_zlo + off) = make_uint4(zl[0], zl[1], zl[2], zl[3]);
+                            fence_proxy_async();
+                            mbar_arrive(bar_z_full);
+                        }
+                    }
+                    tc_fence_before();
+                }
+            } else {
             if (warp_has_rows) {
                 const uint32_t owner = row_valid ? (uint32_t)(row / rows_per) : 0u;
                 const int row_local = row - (int)owner * rows_per;
@@ -704,11 +733,19 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     for (int dst = 0; dst < C; ++dst) mbar_arrive_remote(mapa(bar_z_full, dst));
                 }
             }
-            // ---- after stage 2: y tile (already in the slot) += s_out * V, in place, then TMA store
+            }
+            // ---- after stage 2: y tile (already in the slot) += s_out * V, in place, then TMA store.
+            // The two groups of four warps (one TMEM lane quadrant each) take alternate chunks, so
+            // that one group's TMEM load, barrier and store latencies overlap the other's
+            // arithmetic; chunk parity is also the accumulator buffer, so group g always reads
+            // buffer g.  A thread handles all 64 columns of its token row.
+            const int egroup = chalf;
+            const bool store_thread = (e & (kEpiThreads / 2 - 1)) == 0;
             int prev_slot = -1;
             for (int c = nb; c < ne; ++c, ++it, ++vit) {
+                if ((int)(vit & 1u) != egroup) continue;
                 const int s = it % S; const uint32_t ph = (it / S) & 1u;
-                const int vb = vit & 1u; const uint32_t vph = (vit >> 1) & 1u;
+                const int vb = egroup; const uint32_t vph = (vit >> 1) & 1u;
                 mbar_wait<false>(wctx, bar_v_full(vb), vph, kDevEpilogueWaitTimeout);
                 if (e == 0) TC_TRACE(3, it, 0);
                 mbar_wait<false>(wctx, bar_full(s), ph, kDevEpilogueWaitTimeout);
@@ -717,32 +754,37 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 uint8_t *ytile = sm + s * plan.slot_stride;
                 const float *so = reinterpret_cast<const float *>(ytile + plan.slot_data);
                 if (warp_has_rows) {
-                    uint32_t v[32];
-                    tmem_ld32(tlane + kTmemV + vb * kChunk + chalf * 32, v);   // warp-collective
-                    tmem_wait_ld();
-                    tc_fence_before();
-                    mbar_arrive(bar_v_empty(vb));
-                    if (e == 0) TC_TRACE(3, it, 1);
-                    if (row_valid) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int ch = chalf * 4 + q;                  // 16-byte chunk of the row
-                            uint4 *py = reinterpret_cast<uint4 *>(ytile + row * 128 + ((ch ^ (row & 7)) * 16));
-                            const uint4 yv = *py;
-                            const float4 s0 = *reinterpret_cast<const float4 *>(so + ch * 8);
-                            const float4 s1 = *reinterpret_cast<const float4 *>(so + ch * 8 + 4);
-                            const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
-                            const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-                            uint32_t ow[4];
+                    for (int hh = 0; hh < 2; ++hh) {
+                        uint32_t v[32];
+                        tmem_ld32(tlane + kTmemV + vb * kChunk + hh * 32, v);   // warp-collective
+                        tmem_wait_ld();
+                        if (hh == 1) {
+                            tc_fence_before();
+                            mbar_arrive(bar_v_empty(vb));
+                            if (e == 0) TC_TRACE(3, it, 1);
+                        }
+                        if (row_valid) {
 #pragma unroll
-                            for (int k2 = 0; k2 < 4; ++k2) {
-                                const float y0 = __uint_as_float(yw[k2] << 16);
-                                const float y1 = __uint_as_float(yw[k2] & 0xffff0000u);
-                                const float o0 = fmaf(sc[2 * k2], __uint_as_float(v[q * 8 + 2 * k2]), y0);
-                                const float o1 = fmaf(sc[2 * k2 + 1], __uint_as_float(v[q * 8 + 2 * k2 + 1]), y1);
-                                ow[k2] = pack2_bf16(o0, o1);
+                            for (int q = 0; q < 4; ++q) {
+                                const int ch = hh * 4 + q;                     // 16-byte chunk of the row
+                                uint4 *py = reinterpret_cast<uint4 *>(ytile + row * 128 + ((ch ^ (row & 7)) * 16));
+                                const uint4 yv = *py;
+                                const float4 s0 = *reinterpret_cast<const float4 *>(so + ch * 8);
+                                const float4 s1 = *reinterpret_cast<const float4 *>(so + ch * 8 + 4);
+                                const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
+                                const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                                uint32_t ow[4];
+#pragma unroll
+                                for (int k2 = 0; k2 < 4; ++k2) {
+                                    const float y0 = __uint_as_float(yw[k2] << 16);
+                                    const float y1 = __uint_as_float(yw[k2] & 0xffff0000u);
+                                    const float o0 = fmaf(sc[2 * k2], __uint_as_float(v[q * 8 + 2 * k2]), y0);
+                                    const float o1 = fmaf(sc[2 * k2 + 1], __uint_as_float(v[q * 8 + 2 * k2 + 1]), y1);
+                                    ow[k2] = pack2_bf16(o0, o1);
+                                }
+                                *py = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                             }
-                            *py = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                         }
                     }
                 } else {
@@ -750,9 +792,9 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 }
                 if (e == 0) TC_TRACE(3, it, 2);
                 fence_proxy_async();
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-                if (e == 0) {
-                    TC_TRACE(3, it, 3);
+                asm volatile("bar.sync %0, %1;" ::"r"(1 + 3 * egroup), "n"(kEpiThreads / 2) : "memory");
+                if (store_thread) {
+                    if (e == 0) TC_TRACE(3, it, 3);
                     tma_store_2d(&P.y_map, sm_base + s * plan.slot_stride, c * kChunk, t0);
                     bulk_commit();
                     if (prev_slot >= 0) {
@@ -760,10 +802,10 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                         mbar_arrive(bar_empty(prev_slot));
                     }
                     prev_slot = s;
-                    TC_TRACE(3, it, 4);
+                    if (e == 0) TC_TRACE(3, it, 4);
                 }
             }
-            if (e == 0 && prev_slot >= 0) {
+            if (store_thread && prev_slot >= 0) {
                 bulk_wait_read_0();
                 mbar_arrive(bar_empty(prev_slot));
             }
@@ -771,7 +813,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     }
 
     // ---- teardown -------------------------------------------------------------------------------
-    if (tid == 64 + kGenThreads) bulk_wait_all();       // the thread that issued the stores
+    if (tid == 64 + kGenThreads || tid == 64 + kGenThreads + kEpiThreads / 2) bulk_wait_all();   // the threads that issued the stores
     if (*abort_flag) {
         // give copies that may still be in flight time to land before the CTA goes away
         const long long start = clock64();
@@ -876,12 +918,12 @@ bool plan_launch(int r, int kp, int cluster, int tile_rows, LaunchShape *out)
 {
     int slots = 0;
     for (int s = kMaxSlots; s >= 2; --s) {
-        if (make_plan(r, kp, s, tile_rows).total + 1024 <= kSmemBudget) { slots = s; break; }
+        if (make_plan(r, kp, s, tile_rows, cluster).total + 1024 <= kSmemBudget) { slots = s; break; }
     }
     const int forced = env_int("LORDBA_TC_SLOTS", 0);
     if (forced >= 2 && forced <= slots) slots = forced;
     if (slots < 2) return false;
-    const int smem = make_plan(r, kp, slots, tile_rows).total + 1024;
+    const int smem = make_plan(r, kp, slots, tile_rows, cluster).total + 1024;
     const int n = max_active_clusters(cluster, smem);
     if (n < 1) return false;
     out->cluster = cluster; out->tile_rows = tile_rows; out->slots = slots; out->smem = smem;

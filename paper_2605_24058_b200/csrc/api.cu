@@ -105,7 +105,7 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, 
     }
     if (variant != LORDBA_VARIANT_AUTO && !fma.empty()) return LORDBA_EUNSUPPORTED;
     if (!fast.empty()) {
-        const int rc = use_tc ? launch_forward_tc(fast.data(), (int)fast.size(), T, dtype, stream)
+        const int rc = use_tc ? launch_forward_tc(fast.data(), (int)fast.size(), T, dtype, stream, batch_checked)
                               : launch_forward_mma(fast.data(), fast_rows.data(), (int)fast.size(), dtype, stream,
                                                    batch_checked);
         if (rc != LORDBA_OK) return rc;

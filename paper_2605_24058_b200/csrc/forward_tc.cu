@@ -48,7 +48,7 @@ constexpr int kGenGroups = 2;             // the groups take alternate chunks, s
 constexpr int kGenThreads = kGenGroups * kGenGroupThreads;   // warps 2-9
 constexpr int kEpiThreads = 256;          // warps 6-13
 constexpr int kThreads = 64 + kGenThreads + kEpiThreads;
-constexpr int kMaxTcBatch = 24;
+constexpr int kMaxTcBatch = 96;          // 96 x 320 bytes of descriptors: inside the 32 KiB of kernel parameters
 constexpr int kTmemCols = 256;
 constexpr int kTmemU = 0;               // stage-1 accumulator columns [0, 2r)
 constexpr int kTmemV = 128;             // stage-2 accumulators: [128,192) and [192,256)
@@ -78,6 +78,7 @@ struct TcBatch {
     int cluster;           // CTAs per cluster
     int slots;             // ring depth
     int tile_rows;         // tokens per tile (multiple of cluster, <= 128); rows above it are padding
+    int wait_prev;         // 1: the previous kernel of the stream must be complete before any global access
     int *status;
     long long *trace;      // development builds only
 };
@@ -360,6 +361,14 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
 
     const int r = B.r, kp = B.kp, S = B.slots, C = B.cluster;
     const int tile_rows = B.tile_rows;
+    // Programmatic dependent launch, same protocol as the streaming kernel.  A launch that must
+    // see what ran before it sets up, waits for it, and only then lets its successor in.  A launch
+    // that is independent of its predecessor (a later group of projections of the same batched
+    // call) lets its successor in at once, works without waiting, and waits just before it exits,
+    // so that "this grid is complete" still implies "everything before it is complete".  With
+    // one CTA per SM the successor's CTAs start as this grid's CTAs leave: no idle tail between
+    // the launches of one call.
+    if (!B.wait_prev) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) TC_TRACE(4, 0, 0);
     const SmemPlan plan = make_plan(r, kp, S, tile_rows, C);
     const uint32_t box_bytes = (uint32_t)tile_rows * kChunk * 2;
@@ -423,6 +432,11 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     cluster_sync_all();
     const uint32_t tmem_base = *tmem_slot;
     if (tid == 0) TC_TRACE(4, 0, 1);
+    if (B.wait_prev) {
+        // nothing before this line touched global memory
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
 
     const int rows_per = tile_rows / C;      // token rows of a tile owned by each CTA of the cluster
 
@@ -828,6 +842,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
+    if (!B.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ------------------------------------------------------------------------------------- host side
@@ -994,7 +1009,8 @@ bool tc_supported(const lordba_proj &p, int64_t T, int dtype)
     return encode_fn() != nullptr;
 }
 
-int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream)
+int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream,
+                      bool batch_checked)
 {
     if (n == 0 || T == 0) return LORDBA_OK;
     if (dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
@@ -1002,6 +1018,7 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
     if (!status) return LORDBA_ECUDA;
 
     // one launch per rank value and per kMaxTcBatch projections
+    int launches = 0;
     for (int r = 8; r <= kMaxRank; r += 8) {
         int i = 0;
         while (i < n) {
@@ -1052,6 +1069,10 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
             b.cluster = shape.cluster;
             b.slots = shape.slots;
             b.tile_rows = shape.tile_rows;
+            // the projections of a checked batch are independent of one another: every launch
+            // after the first may overlap its predecessor
+            b.wait_prev = (launches == 0 || !batch_checked) ? 1 : 0;
+            ++launches;
             int n_clusters = b.total_tiles < shape.max_clusters ? b.total_tiles : shape.max_clusters;
             if (env_int("LORDBA_TC_DEBUG", 0))
                 std::fprintf(stderr, "[lordba tc] r=%d proj=%d tiles=%d rows=%d cluster=%d slots=%d smem=%d "
@@ -1064,10 +1085,12 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
             cfg.blockDim = dim3(kThreads, 1, 1);
             cfg.dynamicSmemBytes = shape.smem;
             cfg.stream = stream;
-            cudaLaunchAttribute attr;
-            attr.id = cudaLaunchAttributeClusterDimension;
-            attr.val.clusterDim.x = shape.cluster; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-            cfg.attrs = &attr; cfg.numAttrs = 1;
+            cudaLaunchAttribute attr[2];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = shape.cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[1].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr; cfg.numAttrs = 2;
             if (cudaLaunchKernelEx(&cfg, tc_forward_kernel, b) != cudaSuccess) {
                 cudaGetLastError();
                 return LORDBA_ECUDA;

@@ -41,7 +41,8 @@ int launch_forward_fma(const lordba_proj *projs, const int64_t *tokens, int n, i
 // True when the tcgen05/TMA kernel can take this projection (bf16, 16-byte
 // aligned rows, rank a multiple of 8).
 bool tc_supported(const lordba_proj &p, int64_t T, int dtype);
-int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream);
+int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cudaStream_t stream,
+                      bool batch_checked);
 
 // --- forward_mma.cu ----------------------------------------------------------
 // True when the register-streaming mma.sync kernel can take this projection

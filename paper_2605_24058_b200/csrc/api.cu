@@ -82,7 +82,7 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, 
     }
     // Split the list: what the chosen tensor-core kernel can take, and the rest.  Left to itself
     // the library takes the tcgen05 kernel where it was measured ahead of the streaming one: ranks
-    // above 32 with at least two waves of full 128-token tiles.  (That kernel wants one token
+    // above 16 with at least two waves of full 128-token tiles.  (That kernel wants one token
     // count for all projections.)
     bool use_tc = (variant == LORDBA_VARIANT_TC);
     if (use_tc && tokens) return LORDBA_EUNSUPPORTED;
@@ -90,7 +90,7 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, 
         int64_t big_rank_tiles = 0;
         bool all_big = n > 0;
         for (int i = 0; i < n; ++i) {
-            all_big = all_big && projs[i].r > 32 && tc_supported(projs[i], T, dtype);
+            all_big = all_big && projs[i].r > 16 && tc_supported(projs[i], T, dtype);
             big_rank_tiles += T / 128;
         }
         use_tc = all_big && big_rank_tiles >= 2 * 148;

@@ -211,8 +211,10 @@ struct WaitCtx {
 template <bool kClusterScope>
 __device__ __forceinline__ bool mbar_wait(const WaitCtx &w, uint32_t bar, uint32_t parity, int code)
 {
-    if (*w.abort_flag) return false;
+    // fast path first: the abort flag is looked at only when the phase is not complete yet (after
+    // an abort some barriers never complete, and the loop below then returns within 64 polls)
     if (kClusterScope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+    if (*w.abort_flag) return false;
     const long long start = clock64();
     uint32_t spins = 0;
     for (;;) {

@@ -66,13 +66,13 @@ struct alignas(64) TcProj {
     int d_in, d_out;
     int nk, nn;            // 64-column chunks of d_in / d_out
     int words_a;           // uint32 words per row of packed_A
-    int tile_begin;        // first work item of this projection
 };
 
 struct TcBatch {
     TcProj p[kMaxTcBatch];
     int n_proj;
     int total_tiles;
+    int tiles_per_proj;    // every projection of a launch has the same token count
     int r;                 // rank, multiple of 8
     int kp;                // r rounded up to 16 (K extent of the stage-2 MMA)
     int cluster;           // CTAs per cluster
@@ -448,10 +448,9 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     uint32_t tile_n = 0;    // tiles done by this cluster (phase of the per-tile barriers)
 
     for (int item = cid; item < B.total_tiles; item += n_clusters, ++tile_n) {
-        int pi = 0;
-        while (pi + 1 < B.n_proj && item >= B.p[pi + 1].tile_begin) ++pi;
+        const int pi = item / B.tiles_per_proj;      // no search through the (large) parameter block
         const TcProj &P = B.p[pi];
-        const int t0 = (item - P.tile_begin) * tile_rows;
+        const int t0 = (item - pi * B.tiles_per_proj) * tile_rows;
         int kb, ke, nb, ne;
         split_range(P.nk, C, (int)crank, kb, ke);
         split_range(P.nn, C, (int)crank, nb, ne);
@@ -1055,10 +1054,10 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
                 t.nk = (int)((q.d_in + kChunk - 1) / kChunk);
                 t.nn = (int)((q.d_out + kChunk - 1) / kChunk);
                 t.words_a = (int)((q.d_in + 31) / 32);
-                t.tile_begin = k * tiles_per_proj;
             }
             b.n_proj = m;
             b.total_tiles = m * tiles_per_proj;
+            b.tiles_per_proj = tiles_per_proj;
             b.r = r;
             b.kp = kp;
             b.status = status;

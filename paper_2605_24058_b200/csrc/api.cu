@@ -82,18 +82,20 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, 
     }
     // Split the list: what the chosen tensor-core kernel can take, and the rest.  Left to itself
     // the library takes the tcgen05 kernel where it was measured ahead of the streaming one: ranks
-    // above 16 with at least two waves of full 128-token tiles.  (That kernel wants one token
-    // count for all projections.)
+    // above 32 from 32 tiles of 128 tokens (one projection at T = 4096, a layer at T = 2048), ranks
+    // 24 and 32 from two waves of such tiles.  (That kernel wants one token count for all
+    // projections.)
     bool use_tc = (variant == LORDBA_VARIANT_TC);
     if (use_tc && tokens) return LORDBA_EUNSUPPORTED;
     if (variant == LORDBA_VARIANT_AUTO && !tokens) {
-        int64_t big_rank_tiles = 0;
-        bool all_big = n > 0;
+        int64_t tiles = 0;
+        bool all_ok = n > 0, all_high = true;
         for (int i = 0; i < n; ++i) {
-            all_big = all_big && projs[i].r > 16 && tc_supported(projs[i], T, dtype);
-            big_rank_tiles += T / 128;
+            all_ok = all_ok && projs[i].r > 16 && tc_supported(projs[i], T, dtype);
+            all_high = all_high && projs[i].r > 32;
+            tiles += T / 128;
         }
-        use_tc = all_big && big_rank_tiles >= 2 * 148;
+        use_tc = all_ok && tiles >= (all_high ? 32 : 2 * 148);
     }
     std::vector<lordba_proj> fast, fma;
     std::vector<int64_t> fast_rows, fma_rows;

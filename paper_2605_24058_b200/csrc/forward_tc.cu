@@ -10,20 +10,28 @@
 //
 //   warp 0      TMA producer: 128 x 64 bf16 boxes of x, then of y, into a ring of
 //               128B-swizzled shared-memory slots (cp.async.bulk.tensor, mbarrier tx).
-//   warps 2-5   operand generators: expand packed sign bits into bf16 MMA operands
-//               next to each slot.  Stage 1: W1[k,i] = A_sign[k,i]*s_in[i] as a
+//   warps 2-9   operand generators (two groups of four warps on alternate chunks):
+//               expand packed sign bits into bf16 MMA operands in a ring of their own.  Stage 1: W1[k,i] = A_sign[k,i]*s_in[i] as a
 //               hi/lo bf16 pair (rows 0..r-1 hi, r..2r-1 lo) so that s_in keeps
 //               ~16 mantissa bits.  Stage 2: W2[j,k] = B_sign[j,k] (+-1, exact).
 //   warp 1      MMA issuer (one thread): tcgen05.mma kind::f16, M=128.
 //               Stage 1: U[128 x 2r] += X[128 x 64] * W1^T, accumulated in TMEM
 //               over the CTA's K chunks.  Stage 2, per 64 output columns:
 //               V[128 x 64] = Zhi * W2^T + Zlo * W2^T (z split hi/lo as well).
-//   warps 6-9   epilogue: TMEM -> registers.  After stage 1: u = U_hi + U_lo,
-//               partial sums are pushed to the cluster CTA that owns the row,
+//   warps 10-17 epilogue: TMEM -> registers.  After stage 1: u = U_hi + U_lo; with
+//               a cluster the partial sums are pushed to the CTA that owns the row,
 //               reduced there in a fixed order, scaled by s_r, split into bf16
-//               hi/lo and pushed back into every CTA's stage-2 operand buffer.
-//               After stage 2: y tile (already in the slot) += s_out * V in fp32,
-//               rounded once to bf16 in place, TMA-stored from the same slot.
+//               hi/lo and pushed back into every CTA's stage-2 operand buffer; a
+//               lone CTA writes z = s_r * u straight into its own buffer.
+//               After stage 2 (two groups of four warps on alternate chunks): y
+//               tile (already in the slot) += s_out * V in fp32, rounded once to
+//               bf16 in place, TMA-stored from the same slot.
+//
+// The roles are decoupled by mbarriers only, so each one's per-chunk latency is
+// a ceiling for the whole pipeline; the single MMA-issuing thread in particular
+// carries its ring positions and descriptor words instead of recomputing them.
+// Consecutive launches of one batched call overlap through programmatic
+// dependent launch (B.wait_prev = 0 for all but the first).
 //
 // Every mbarrier wait is bounded: after ~1 s it records a code in the device
 // status word, raises the CTA's abort flag (all later waits return at once) and
@@ -259,13 +267,10 @@ __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk
 __device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-// Shared-memory matrix descriptor (tcgen05): start address, leading / stride byte offsets
-// (all >> 4), descriptor version 1, layout type in bits 61..63 (0 = no swizzle, 2 = 128B swizzle).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout)
-{
-    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
-           (1ull << 46) | ((uint64_t)layout << 61);
-}
+// Shared-memory matrix descriptor (tcgen05), 64 bits: start address >> 4 in bits 0..13, leading
+// byte offset >> 4 in bits 16..29, stride byte offset >> 4 in bits 32..45, descriptor version 1 at
+// bit 46, layout type in bits 61..63 (0 = no swizzle, 2 = 128B swizzle).  The MMA issuer builds the
+// two 32-bit words itself.
 
 // Instruction descriptor, kind::f16: D = fp32, A = B = bf16, both K-major, M x N tile.
 __device__ __forceinline__ uint32_t instr_desc(int m, int n)
@@ -273,14 +278,7 @@ __device__ __forceinline__ uint32_t instr_desc(int m, int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                         uint32_t accumulate)
-{
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// The same with the descriptors as (low, high) words: the issuing thread keeps the high words
+// tcgen05.mma with the descriptors as (low, high) words: the issuing thread keeps the high words
 // and the base of the low words in registers and only adds a 16-byte-unit offset per MMA.
 __device__ __forceinline__ void mma_bf16_words(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
                                                uint32_t b_hi, uint32_t idesc, uint32_t accumulate)
@@ -507,7 +505,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 const uint32_t idesc1 = instr_desc(kTileM, 2 * r);
                 const uint32_t idesc2 = instr_desc(kTileM, kChunk);
                 const int ksteps2 = kp / 16;
-                // descriptor words (see smem_desc): low = address >> 4 | (lbo >> 4) << 16,
+                // descriptor words (layout above): low = address >> 4 | (lbo >> 4) << 16,
                 // high = sbo >> 4 | version | layout << 29
                 // (a shared address carries the CTA's rank in the cluster above bit 18: masked off)
                 const uint32_t base18 = sm_base & 0x3ffffu;

@@ -1,4 +1,4 @@
-// Tensor-core kernel of the LoRDBA adapter forward (bf16 activations), sm_100a:
+// Tensor-core kernel of the LoRDBA adapter forward (bf16 or float16 activations), sm_100a:
 //
 //   y[t,:] += s_out * ( B_sign ( s_r * ( A_sign ( s_in * x[t,:] ) ) ) )        (Eq. 8 / Eq. 9)
 //
@@ -38,6 +38,7 @@
 // the kernel runs to its normal teardown, which frees TMEM.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <cstdio>
 #include <cstdlib>
@@ -63,6 +64,14 @@ constexpr int kTmemV = 128;             // stage-2 accumulators: [128,192) and [
 constexpr int kSmemBudget = 227 * 1024;
 constexpr long long kWaitLimitCycles = 1500000000LL;
 
+// Element type of x and y, and how s_in enters the first product (same meaning as in the
+// streaming kernel).
+enum IoKind {
+    kIoBf16 = 0,      // bfloat16; W1 = +-s_in as bf16 hi rows and lo rows (N = 2r)
+    kIoF16 = 1,       // IEEE half; W1 as half hi rows and lo rows (N = 2r)
+    kIoF16Exact = 2   // IEEE half; s_in stated to be exact in half precision: hi rows only (N = r)
+};
+
 struct alignas(64) TcProj {
     CUtensorMap x_map;
     CUtensorMap y_map;
@@ -86,6 +95,7 @@ struct TcBatch {
     int cluster;           // CTAs per cluster
     int slots;             // ring depth
     int tile_rows;         // tokens per tile (multiple of cluster, <= 128); rows above it are padding
+    int io;                // element type of x / y and form of s_in: see IoKind
     int wait_prev;         // 1: the previous kernel of the stream must be complete before any global access
     int *status;
     long long *trace;      // development builds only
@@ -272,10 +282,12 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 // bit 46, layout type in bits 61..63 (0 = no swizzle, 2 = 128B swizzle).  The MMA issuer builds the
 // two 32-bit words itself.
 
-// Instruction descriptor, kind::f16: D = fp32, A = B = bf16, both K-major, M x N tile.
-__device__ __forceinline__ uint32_t instr_desc(int m, int n)
+// Instruction descriptor, kind::f16: D = fp32, A and B both bf16 (format 1) or both half (format
+// 0; the two never differ), both K-major, M x N tile.
+__device__ __forceinline__ uint32_t instr_desc(int m, int n, bool half_operands)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+    const uint32_t fmt = half_operands ? 0u : ((1u << 7) | (1u << 10));
+    return (1u << 4) | fmt | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // tcgen05.mma with the descriptors as (low, high) words: the issuing thread keeps the high words
@@ -326,6 +338,12 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi)
     return *reinterpret_cast<const uint32_t *>(&h);
 }
 __device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+__device__ __forceinline__ uint32_t pack2_f16(float lo, float hi)
+{
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+__device__ __forceinline__ float2 unpack2_f16(uint32_t w) { return __half22float2(*reinterpret_cast<const __half2 *>(&w)); }
 
 // 8 sign bits (bit 1 = +1) -> XOR masks over four bf16 pairs (a 0 bit flips the sign).  b times
 // (2^(15-2p) + 2^(30-2p)) is two disjoint shifted copies of the byte that put bit 2p at position
@@ -394,6 +412,8 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
 
     const int kt8 = kp / 8;                 // 16-byte chunks per row of a stage-2 operand
     const int r8 = r / 8;
+    const bool half_io = B.io != kIoBf16;       // x, y and W1 are IEEE halves
+    const bool lo_pass = B.io != kIoF16Exact;   // W1 and U carry low parts of s_in
     const uint32_t sign_bytes = 8u * r;     // sign bytes next to one 64-column chunk, either stage
 
     // ---- one-time setup ---------------------------------------------------------------------
@@ -502,8 +522,10 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             // cost this thread ~1100 cycles in stage 1 and ~1800 in stage 2, more than the loads).
             // So: ring positions are carried, descriptor words are precomputed, loops are unrolled.
             if (lane == 0) {
-                const uint32_t idesc1 = instr_desc(kTileM, 2 * r);
-                const uint32_t idesc2 = instr_desc(kTileM, kChunk);
+                // N of stage 1: hi and lo rows, or the hi rows alone rounded up to the next legal N
+                // (rows past r then hold stale operand data and feed accumulator columns nobody reads)
+                const uint32_t idesc1 = instr_desc(kTileM, lo_pass ? 2 * r : (r + 15) / 16 * 16, half_io);
+                const uint32_t idesc2 = instr_desc(kTileM, kChunk, false);      // z and W2 are always bf16
                 const int ksteps2 = kp / 16;
                 // descriptor words (layout above): low = address >> 4 | (lbo >> 4) << 16,
                 // high = sbo >> 4 | version | layout << 29
@@ -593,9 +615,15 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 uint32_t hi[4], lo[4];
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
-                    const float ah = bf16_round(sv[2 * p]), bh = bf16_round(sv[2 * p + 1]);
-                    hi[p] = pack2_bf16(ah, bh);
-                    lo[p] = pack2_bf16(sv[2 * p] - ah, sv[2 * p + 1] - bh);
+                    if (half_io) {
+                        hi[p] = pack2_f16(sv[2 * p], sv[2 * p + 1]);
+                        const float2 hf = unpack2_f16(hi[p]);
+                        lo[p] = pack2_f16(sv[2 * p] - hf.x, sv[2 * p + 1] - hf.y);
+                    } else {
+                        const float ah = bf16_round(sv[2 * p]), bh = bf16_round(sv[2 * p + 1]);
+                        hi[p] = pack2_bf16(ah, bh);
+                        lo[p] = pack2_bf16(sv[2 * p] - ah, sv[2 * p + 1] - bh);
+                    }
                 }
                 uint8_t *w1 = aux;
                 for (int k = kg0 * 8 + rsub; k < r; k += kGenGroupThreads / 8) {
@@ -603,8 +631,9 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     const int row_hi = k, row_lo = r + k;
                     *reinterpret_cast<uint4 *>(w1 + (row_hi >> 3) * 1024 + cc * 128 + (row_hi & 7) * 16) =
                         make_uint4(hi[0] ^ m.x, hi[1] ^ m.y, hi[2] ^ m.z, hi[3] ^ m.w);
-                    *reinterpret_cast<uint4 *>(w1 + (row_lo >> 3) * 1024 + cc * 128 + (row_lo & 7) * 16) =
-                        make_uint4(lo[0] ^ m.x, lo[1] ^ m.y, lo[2] ^ m.z, lo[3] ^ m.w);
+                    if (lo_pass)
+                        *reinterpret_cast<uint4 *>(w1 + (row_lo >> 3) * 1024 + cc * 128 + (row_lo & 7) * 16) =
+                            make_uint4(lo[0] ^ m.x, lo[1] ^ m.y, lo[2] ^ m.z, lo[3] ^ m.w);
                 }
                 fence_proxy_async();
                 mbar_arrive(bar_op_full(o));
@@ -668,7 +697,12 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     for (int p = chalf; p < r8; p += 2) {
                         float h[8], l[8];
                         tmem_ld8(tlane + kTmemU + p * 8, h);          // warp-collective
-                        tmem_ld8(tlane + kTmemU + r + p * 8, l);
+                        if (lo_pass) {
+                            tmem_ld8(tlane + kTmemU + r + p * 8, l);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) l[i] = 0.0f;
+                        }
                         tmem_wait_ld();
                         if (row_valid) {
                             uint32_t zh[4], zl[4];
@@ -698,7 +732,12 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 for (int p = chalf; p < r8; p += 2) {
                     float h[8], l[8];
                     tmem_ld8(tlane + kTmemU + p * 8, h);          // warp-collective
-                    tmem_ld8(tlane + kTmemU + r + p * 8, l);
+                    if (lo_pass) {
+                        tmem_ld8(tlane + kTmemU + r + p * 8, l);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) l[i] = 0.0f;
+                    }
                     tmem_wait_ld();
                     if (row_valid) {
                         uint32_t w[8];
@@ -790,11 +829,17 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                                 uint32_t ow[4];
 #pragma unroll
                                 for (int k2 = 0; k2 < 4; ++k2) {
-                                    const float y0 = __uint_as_float(yw[k2] << 16);
-                                    const float y1 = __uint_as_float(yw[k2] & 0xffff0000u);
+                                    float y0, y1;
+                                    if (half_io) {
+                                        const float2 yf = unpack2_f16(yw[k2]);
+                                        y0 = yf.x; y1 = yf.y;
+                                    } else {
+                                        y0 = __uint_as_float(yw[k2] << 16);
+                                        y1 = __uint_as_float(yw[k2] & 0xffff0000u);
+                                    }
                                     const float o0 = fmaf(sc[2 * k2], __uint_as_float(v[q * 8 + 2 * k2]), y0);
                                     const float o1 = fmaf(sc[2 * k2 + 1], __uint_as_float(v[q * 8 + 2 * k2 + 1]), y1);
-                                    ow[k2] = pack2_bf16(o0, o1);
+                                    ow[k2] = half_io ? pack2_f16(o0, o1) : pack2_bf16(o0, o1);
                                 }
                                 *py = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                             }
@@ -994,7 +1039,7 @@ bool choose_shape(int r, int kp, int n_proj, int64_t T, int min_chunks, LaunchSh
 
 bool tc_supported(const lordba_proj &p, int64_t T, int dtype)
 {
-    if (dtype != LORDBA_BF16 || T < 1) return false;
+    if ((dtype != LORDBA_BF16 && dtype != LORDBA_F16) || T < 1) return false;
     if (((p.flags >> 8) & 0xf) != 0) return false;          // multi-envelope adapters: other kernels
     if (p.r % 8 != 0 || p.r < 8 || p.r > kMaxRank) return false;
     if (p.d_in < kChunk || p.d_out < kChunk) return false;
@@ -1012,12 +1057,17 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
                       bool batch_checked)
 {
     if (n == 0 || T == 0) return LORDBA_OK;
-    if (dtype != LORDBA_BF16) return LORDBA_EUNSUPPORTED;
+    if (dtype != LORDBA_BF16 && dtype != LORDBA_F16) return LORDBA_EUNSUPPORTED;
     int *status = device_status_word();
     if (!status) return LORDBA_ECUDA;
+    auto io_of = [&](const lordba_proj &q) {
+        if (dtype == LORDBA_BF16) return (int)kIoBf16;
+        return (q.flags & LORDBA_PROJ_SCALES_F16) ? (int)kIoF16Exact : (int)kIoF16;
+    };
 
-    // one launch per rank value and per kMaxTcBatch projections
+    // one launch per element / scale kind, rank value and kMaxTcBatch projections
     int launches = 0;
+    for (int io = (dtype == LORDBA_BF16 ? kIoBf16 : kIoF16); io <= (dtype == LORDBA_BF16 ? kIoBf16 : kIoF16Exact); ++io)
     for (int r = 8; r <= kMaxRank; r += 8) {
         int i = 0;
         while (i < n) {
@@ -1025,7 +1075,7 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
             const lordba_proj *sel[kMaxTcBatch];
             int m = 0, min_chunks = 1 << 30;
             for (; i < n && m < kMaxTcBatch; ++i) {
-                if (projs[i].r != r) continue;
+                if (projs[i].r != r || io_of(projs[i]) != io) continue;
                 sel[m++] = &projs[i];
                 const int nk = (int)((projs[i].d_in + kChunk - 1) / kChunk);
                 const int nn = (int)((projs[i].d_out + kChunk - 1) / kChunk);
@@ -1058,6 +1108,7 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
             b.tiles_per_proj = tiles_per_proj;
             b.r = r;
             b.kp = kp;
+            b.io = io;
             b.status = status;
 #ifdef LORDBA_TC_TRACE
             {

@@ -550,3 +550,31 @@ def test_f16_mixed_batch_and_segments(oracle):
         want = oracle_forward(oracle, p)
         assert_close(got[:n], want[:n], "f16", "f16 segment " + p.name, scale_from=want)
         assert np.array_equal(got[n:], p.y_f64()[n:])
+
+
+@pytest.mark.parametrize("r,scales_f16", [(64, False), (64, True), (24, True), (40, False)])
+def test_f16_layer_on_the_tcgen05_kernel(oracle, r, scales_f16):
+    """One decoder layer's seven projections with float16 activations, as the library runs them
+    by itself and with the tcgen05 kernel pinned (full 128-token tiles plus a ragged last one):
+    both forms of s_in (a pair of halves; one half, declared), ranks that are and are not
+    multiples of 16.  Sampled rows: first tile, last (ragged) tile, random rows."""
+    T = 2048 + 40
+    rng = np.random.default_rng(11 + r)
+    rows = np.unique(np.concatenate([np.arange(16), np.arange(T - 48, T), rng.integers(0, T, size=24)]))
+    projs = [workloads.make_projection(di, do, r, T, "f16", seed=5000 + 7 * r + i, name=n, scales_f16=scales_f16,
+                                       outlier_frac=0.01)
+             for i, (n, di, do) in enumerate(workloads.LAYER_PROJECTIONS)]
+    devs = [DeviceProj(p) for p in projs]
+    lordba.adapter_forward_batched([d.proj() for d in devs], T, lordba.F16)
+    rows_t = torch.from_numpy(rows).cuda()
+    for p, d in zip(projs, devs):
+        assert_close(torch_to_f64(d.y[rows_t]), oracle_forward(oracle, p, rows=rows), "f16",
+                     "f16 layer r=%d %s" % (r, p.name))
+    # and with the tcgen05 kernel pinned (the library's own choice only for ranks above 32 here)
+    for d in devs:
+        d.reset_y()
+    lordba.set_variant(lordba.VARIANT_TC)
+    lordba.adapter_forward_batched([d.proj() for d in devs], T, lordba.F16)
+    for p, d in zip(projs, devs):
+        assert_close(torch_to_f64(d.y[rows_t]), oracle_forward(oracle, p, rows=rows), "f16",
+                     "f16 layer, tcgen05 pinned, r=%d %s" % (r, p.name))

@@ -367,8 +367,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         }
     }
-    auto issue_item = [&](int it) {       // one thread
-        const int s = it % S;
+    auto issue_item = [&](int it, int s) {       // one thread; s = it % S
         const bool is_x = it < n_x;
         const int cw = is_x ? cwx : cwy;
         const int col0 = is_x ? it * cwx : (yc_begin + (it - n_x)) * cwy;
@@ -384,16 +383,20 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     };
     const int n_first = n_items < S ? n_items : S;
     if (tid == kConsumerThreads)
-        for (int it = 0; it < n_first; ++it) issue_item(it);
+        for (int it = 0; it < n_first; ++it) issue_item(it, it);     // n_first <= S
     __syncthreads();
     if (tid == 0) MMA_TRACE(1);
 
     if (warp == kConsumerWarps) {
         // ================= producer warp: one lane refills the slots as they are released ========
         if (lane == 0) {
+            // item n_first is the first to reuse a slot: slot 0, first release phase
+            int s = 0;
+            uint32_t eph = 0;
             for (int it = n_first; it < n_items; ++it) {
-                if (!mbar_wait(wctx, bar_empty(it % S), ((it / S) - 1) & 1u, kDevTmaWaitTimeout)) break;
-                issue_item(it);
+                if (!mbar_wait(wctx, bar_empty(s), eph, kDevTmaWaitTimeout)) break;
+                issue_item(it, s);
+                if (++s == S) { s = 0; eph ^= 1u; }
             }
         }
     } else {
@@ -418,9 +421,10 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     for (int e = 0; e < 4; ++e) acc[env][h][a][e] = 0.0f;
 
         int it = 0;
+        int s = 0;                 // ring slot of item `it` and the phase of its barrier, carried
+        uint32_t sph = 0;          // along instead of recomputed by division
         for (; it < n_x; ++it) {
-            const int s = it % S;
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), (it / S) & 1u, kDevMmaWaitTimeout));
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), sph, kDevMmaWaitTimeout));
             const int cwv = (d_in - it * cwx < cwx) ? (d_in - it * cwx) : cwx;
             if (tid == 0) MMA_TRACE(20 + it);
             if (gcol < cwv && ok) {
@@ -497,6 +501,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
             if (tid == 0) MMA_TRACE(40 + it);
+            if (++s == S) { s = 0; sph ^= 1u; }
         }
 
         // ---- reduce u over the warps in a fixed order, z = s_r * u, split into bf16 hi + lo ---
@@ -563,8 +568,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         const bool vec32 = P.y_vec32 != 0;
 
         for (; it < n_items; ++it) {
-            const int s = it % S;
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), (it / S) & 1u, kDevEpilogueWaitTimeout));
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), sph, kDevEpilogueWaitTimeout));
             const int col0 = (yc_begin + (it - n_x)) * cwy;
             const int cwv = (d_out - col0 < cwy) ? (d_out - col0) : cwy;
             if (tid == 0) MMA_TRACE(20 + it);
@@ -676,6 +680,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
             if (tid == 0) MMA_TRACE(40 + it);
+            if (++s == S) { s = 0; sph ^= 1u; }
         }
     }
     if (tid == 0) MMA_TRACE(61);

@@ -359,6 +359,15 @@ __device__ __forceinline__ uint4 sign_masks(uint32_t b)
     return m;
 }
 
+// Slot of the data ring and phase of its barriers for chunk counter `it`: set once per tile (one
+// division), then stepped, so that no role divides per chunk.
+struct RingPos {
+    int s;
+    uint32_t ph;
+    __device__ __forceinline__ void set(uint32_t it, int slots) { s = (int)(it % (uint32_t)slots); ph = (it / (uint32_t)slots) & 1u; }
+    __device__ __forceinline__ void next(int slots) { if (++s == slots) { s = 0; ph ^= 1u; } }
+};
+
 // balanced contiguous split of n chunks over `parts` CTAs
 __device__ __forceinline__ void split_range(int n, int parts, int idx, int &begin, int &end)
 {
@@ -480,8 +489,10 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             // chunk's 64 columns, then the 64-column box of x (stage 1) or y (stage 2).  A ragged
             // last chunk (fewer than 64 valid columns) leaves the raw fetch to the generators.
             if (lane == 0) {
-                for (int c = kb; c < ke; ++c, ++it) {
-                    const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                RingPos rp;
+                rp.set(it, S);
+                for (int c = kb; c < ke; ++c, ++it, rp.next(S)) {
+                    const int s = rp.s; const uint32_t ph = rp.ph;
                     mbar_wait<false>(wctx, bar_empty(s), ph ^ 1u, kDevTmaWaitTimeout);
                     TC_TRACE(0, it, 0);
                     const uint32_t slot = sm_base + s * plan.slot_stride;
@@ -497,8 +508,8 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     mbar_arrive_expect_tx(bar_full(s), box_bytes);
                     tma_load_2d(slot, &P.x_map, c * kChunk, t0, bar_full(s));
                 }
-                for (int c = nb; c < ne; ++c, ++it) {
-                    const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                for (int c = nb; c < ne; ++c, ++it, rp.next(S)) {
+                    const int s = rp.s; const uint32_t ph = rp.ph;
                     mbar_wait<false>(wctx, bar_empty(s), ph ^ 1u, kDevTmaWaitTimeout);
                     TC_TRACE(0, it, 0);
                     const uint32_t slot = sm_base + s * plan.slot_stride;
@@ -591,9 +602,11 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             const int rsub = g & 7;                // row within an 8-row core matrix
             const int cc = (g >> 3) & 7;           // 16-byte chunk (8 columns) within the 64-column box
             const int kg0 = g >> 6;                // first 8-row group handled by this thread (stage 1)
-            for (int c = kb; c < ke; ++c, ++it) {
+            RingPos rp;
+            rp.set(it, S);
+            for (int c = kb; c < ke; ++c, ++it, rp.next(S)) {
                 if ((int)(it % kGenGroups) != group) continue;
-                const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                const int s = rp.s; const uint32_t ph = rp.ph;
                 mbar_wait<false>(wctx, bar_raw(s), ph, kDevTmaWaitTimeout);
                 if (g == 0) TC_TRACE(2, it, 0);
                 const int o = it % kOps;
@@ -639,9 +652,9 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 mbar_arrive(bar_op_full(o));
                 if (g == 0) TC_TRACE(2, it, 1);
             }
-            for (int c = nb; c < ne; ++c, ++it) {
+            for (int c = nb; c < ne; ++c, ++it, rp.next(S)) {
                 if ((int)(it % kGenGroups) != group) continue;
-                const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                const int s = rp.s; const uint32_t ph = rp.ph;
                 mbar_wait<false>(wctx, bar_raw(s), ph, kDevTmaWaitTimeout);
                 if (g == 0) TC_TRACE(2, it, 0);
                 const int o = it % kOps;
@@ -794,9 +807,11 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             const int egroup = chalf;
             const bool store_thread = (e & (kEpiThreads / 2 - 1)) == 0;
             int prev_slot = -1;
-            for (int c = nb; c < ne; ++c, ++it, ++vit) {
+            RingPos rp;
+            rp.set(it, S);
+            for (int c = nb; c < ne; ++c, ++it, ++vit, rp.next(S)) {
                 if ((int)(vit & 1u) != egroup) continue;
-                const int s = it % S; const uint32_t ph = (it / S) & 1u;
+                const int s = rp.s; const uint32_t ph = rp.ph;
                 const int vb = egroup; const uint32_t vph = (vit >> 1) & 1u;
                 mbar_wait<false>(wctx, bar_v_full(vb), vph, kDevEpilogueWaitTimeout);
                 if (e == 0) TC_TRACE(3, it, 0);

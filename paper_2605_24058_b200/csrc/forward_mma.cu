@@ -878,6 +878,19 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                 if (projs[i].d_out < min_dout) min_dout = projs[i].d_out;
             }
             if (m == kMaxBatch || (i == n && m > 0)) {
+                // CTAs start in grid order (all tiles of projection 0, then of projection 1, ...):
+                // projections with the most bytes per token go first, so that the last, partly
+                // filled wave consists of the cheapest tiles (stable insertion sort).
+                for (int a = 1; a < m; ++a) {
+                    const lordba_proj *pa = sel[a];
+                    const int64_t ta = sel_T[a], ka = pa->d_in + 2 * pa->d_out;
+                    int b = a - 1;
+                    while (b >= 0 && sel[b]->d_in + 2 * sel[b]->d_out < ka) {
+                        sel[b + 1] = sel[b]; sel_T[b + 1] = sel_T[b];
+                        --b;
+                    }
+                    sel[b + 1] = pa; sel_T[b + 1] = ta;
+                }
                 // Tile height: the smallest number of full waves of 16-row tiles, then the rows
                 // per tile that spread the tokens evenly over those waves.
                 int64_t min_tiles = 0, sum_T = 0;

@@ -435,14 +435,15 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 const uint4 xb0 = *reinterpret_cast<const uint4 *>(slot + off_r0 + pc1);
                 const uint4 xa1 = *reinterpret_cast<const uint4 *>(slot + off_r1 + pc0);
                 const uint4 xb1 = *reinterpret_cast<const uint4 *>(slot + off_r1 + pc1);
-                const uint2 *blk = reinterpret_cast<const uint2 *>(slot + plan.off_bits) + warp * r;
-                uint32_t bytes[R8];                                  // sign bytes of this lane's 16 columns
+                // the warp's block of the carrier: r rows of 64 sign bits; this lane's 16 columns are
+                // half-word q of a row
+                const uint16_t *blk = reinterpret_cast<const uint16_t *>(slot + plan.off_bits) + warp * r * 4 + q;
+                uint32_t bytes[R8];                                  // sign bits of this lane's 16 columns
 #pragma unroll
                 for (int a = 0; a < R8; ++a) {
                     int k = 8 * a + g;
                     if (k > r - 1) k = r - 1;                       // padded rank rows: result unused
-                    const uint2 sb = blk[k];                         // the row's 64 sign bits of this block
-                    bytes[a] = (((q & 2) ? sb.y : sb.x) >> (16 * (q & 1))) & 0xffffu;
+                    bytes[a] = blk[k * 4];
                 }
                 const uint32_t xk[4][4] = {{xa0.x, xa1.x, xa0.y, xa1.y}, {xa0.z, xa1.z, xa0.w, xa1.w},
                                            {xb0.x, xb1.x, xb0.y, xb1.y}, {xb0.z, xb1.z, xb0.w, xb1.w}};

@@ -1098,6 +1098,16 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
                 if (nn < min_chunks) min_chunks = nn;
             }
             if (m == 0) continue;
+            // Tiles go to the persistent CTAs round-robin in index order: projections in order of
+            // falling cost per tile (a y chunk costs about 1.7 x chunks), so that a CTA's later
+            // tiles are cheaper than its earlier ones and the loads even out (stable insertion sort).
+            auto tile_cost = [](const lordba_proj *q) { return 10 * q->d_in + 17 * q->d_out; };
+            for (int a = 1; a < m; ++a) {
+                const lordba_proj *pa = sel[a];
+                int b = a - 1;
+                while (b >= 0 && tile_cost(sel[b]) < tile_cost(pa)) { sel[b + 1] = sel[b]; --b; }
+                sel[b + 1] = pa;
+            }
             const int kp = (r + 15) / 16 * 16;
             LaunchShape shape;
             if (!choose_shape(r, kp, m, T, min_chunks, &shape)) return LORDBA_ECUDA;

@@ -40,10 +40,12 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "lordba_internal.h"
 
@@ -1084,29 +1086,56 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
     int launches = 0;
     for (int io = (dtype == LORDBA_BF16 ? kIoBf16 : kIoF16); io <= (dtype == LORDBA_BF16 ? kIoBf16 : kIoF16Exact); ++io)
     for (int r = 8; r <= kMaxRank; r += 8) {
-        int i = 0;
-        while (i < n) {
-            // collect the next projections of this rank
+        // all projections of this kind and rank, in order of falling cost per tile (a y chunk
+        // costs about 1.7 x chunks): tiles go to the persistent CTAs round-robin in index order,
+        // so a CTA's later tiles are cheaper than its earlier ones, and the last launch of the
+        // call holds the cheapest projections
+        std::vector<const lordba_proj *> all;
+        for (int i = 0; i < n; ++i)
+            if (projs[i].r == r && io_of(projs[i]) == io) all.push_back(&projs[i]);
+        if (all.empty()) continue;
+        std::stable_sort(all.begin(), all.end(), [](const lordba_proj *a, const lordba_proj *b) {
+            return 10 * a->d_in + 17 * a->d_out > 10 * b->d_in + 17 * b->d_out;
+        });
+        // Launch sizes.  The launches of a call run back to back (each one's CTAs start as the
+        // previous one's leave), so only the last one's tail is exposed: it gets the number of
+        // projections whose 128-token tiles fill whole waves of the SMs best, the others share
+        // the rest evenly.
+        std::vector<int> sizes;
+        {
+            const int total = (int)all.size();
+            if (total <= kMaxTcBatch) {
+                sizes.push_back(total);
+            } else {
+                const int64_t tpp = (T + kTileM - 1) / kTileM;
+                int dev = 0, sms = 0;
+                if (cudaGetDevice(&dev) != cudaSuccess ||
+                    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+                    sms = 148;
+                const int64_t ctas = sms;
+                int last = kMaxTcBatch;
+                double best_fill = 0.0;
+                for (int cand = kMaxTcBatch; cand >= kMaxTcBatch / 3; --cand) {
+                    const int64_t tiles = cand * tpp, waves = (tiles + ctas - 1) / ctas;
+                    const double fill = (double)tiles / (double)(waves * ctas);
+                    if (fill > best_fill + 1e-9) { best_fill = fill; last = cand; }
+                }
+                const int rest = total - last, parts = (rest + kMaxTcBatch - 1) / kMaxTcBatch;
+                for (int k = 0; k < parts; ++k) sizes.push_back(rest / parts + (k < rest % parts ? 1 : 0));
+                sizes.push_back(last);
+            }
+        }
+        size_t next = 0;
+        for (size_t li = 0; li < sizes.size(); ++li) {
             const lordba_proj *sel[kMaxTcBatch];
-            int m = 0, min_chunks = 1 << 30;
-            for (; i < n && m < kMaxTcBatch; ++i) {
-                if (projs[i].r != r || io_of(projs[i]) != io) continue;
-                sel[m++] = &projs[i];
-                const int nk = (int)((projs[i].d_in + kChunk - 1) / kChunk);
-                const int nn = (int)((projs[i].d_out + kChunk - 1) / kChunk);
+            const int m = sizes[li];
+            int min_chunks = 1 << 30;
+            for (int k = 0; k < m; ++k) {
+                sel[k] = all[next++];
+                const int nk = (int)((sel[k]->d_in + kChunk - 1) / kChunk);
+                const int nn = (int)((sel[k]->d_out + kChunk - 1) / kChunk);
                 if (nk < min_chunks) min_chunks = nk;
                 if (nn < min_chunks) min_chunks = nn;
-            }
-            if (m == 0) continue;
-            // Tiles go to the persistent CTAs round-robin in index order: projections in order of
-            // falling cost per tile (a y chunk costs about 1.7 x chunks), so that a CTA's later
-            // tiles are cheaper than its earlier ones and the loads even out (stable insertion sort).
-            auto tile_cost = [](const lordba_proj *q) { return 10 * q->d_in + 17 * q->d_out; };
-            for (int a = 1; a < m; ++a) {
-                const lordba_proj *pa = sel[a];
-                int b = a - 1;
-                while (b >= 0 && tile_cost(sel[b]) < tile_cost(pa)) { sel[b + 1] = sel[b]; --b; }
-                sel[b + 1] = pa;
             }
             const int kp = (r + 15) / 16 * 16;
             LaunchShape shape;

@@ -75,7 +75,8 @@ typedef enum {
 /* Kernel families the forward entry points can be pinned to (default AUTO). */
 typedef enum {
     LORDBA_VARIANT_AUTO = 0,  /* the library's choice: streaming kernel where the shape allows  */
-                              /* it (tcgen05 kernel for rank > 32 with many tiles), else FMA   */
+                              /* it; tcgen05 kernel for rank > 16 once a call holds enough     */
+                              /* 128-token tiles (rank > 32: 32 tiles, else two per SM); else FMA */
     LORDBA_VARIANT_FMA = 1,   /* CUDA-core float32 FMA kernel (always used for LORDBA_F32)  */
     LORDBA_VARIANT_TC = 2,    /* tcgen05/TMA cluster kernel; LORDBA_EUNSUPPORTED if the     */
                               /* shape or alignment rules it out                            */
@@ -118,7 +119,7 @@ typedef struct lordba_proj {
  * writes, and that nothing else was enqueued on the stream in between.  Example: the q, k and v
  * adapters of one layer read the same x and update three different y buffers; the first is
  * called without the flag (it must see the kernel that produced x), the other two with it.
- * Work enqueued after the run is ordered after all of it, as usual.  Only the streaming bf16
+ * Work enqueued after the run is ordered after all of it, as usual.  Only the streaming
  * kernel acts on the flag; elsewhere it is accepted and ignored.
  */
 #define LORDBA_PROJ_OVERLAP 1

@@ -50,6 +50,12 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_DRAM_BYTES_PER_LAUNCH = 33633792
 
 
+def ensure_library():
+    """Build liblordba.so in-tree if it is missing or stale (it is not under version control)."""
+    from paper_2605_24058_b200 import build
+    build.build_library()
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -205,6 +211,7 @@ def run_gpu(args):
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    ensure_library()
     lordba.load()
     if args.variant is not None:
         lordba.set_variant({"auto": 0, "fma": 1, "tc": 2, "mma": 3}[args.variant])
@@ -416,6 +423,7 @@ def run_workload(args):
 
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
+    ensure_library()
     lordba.load()
     if args.variant is not None:
         lordba.set_variant({"auto": 0, "fma": 1, "tc": 2, "mma": 3}[args.variant])

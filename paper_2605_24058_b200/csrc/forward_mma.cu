@@ -280,26 +280,33 @@ __device__ __forceinline__ uint32_t with_signs(uint32_t operand, uint32_t bits)
     return operand ^ (~bits & kSignBits);
 }
 
-// The r sign bits of row j_local of an item's slice of B_sign: r/8 bytes per row for r % 8 == 0;
-// for r = 1, 2 or 4 the rows are packed 8, 4 or 2 to a byte and what lies above a row's r bits
-// belongs to other rows (harmless: those ranks of z are zero).
+// The r sign bits of row j_local of an item's slice of B_sign, which is the dense bit stream of
+// the rows: r/8 whole bytes per row when r is a multiple of 8, else a row starts at bit j_local * r
+// and is gathered byte by byte.  Bits above the row's r belong to other rows and are harmless
+// (those ranks of z are zero).
 template <int RP>
 __device__ __forceinline__ uint64_t b_row_bits(const uint8_t *bits, int j_local, int r)
 {
-    if (RP == 8) {
-        if (r == 8) return bits[j_local];
-        const int bit = j_local * r;
-        return (uint32_t)bits[bit >> 3] >> (bit & 7);
+    if ((r & 7) == 0) {
+        if (RP == 8) return bits[j_local];
+        if (RP == 16) return reinterpret_cast<const uint16_t *>(bits)[j_local];
+        if (r == 32) return reinterpret_cast<const uint32_t *>(bits)[j_local];
+        if (r == 64) {
+            const uint2 v = reinterpret_cast<const uint2 *>(bits)[j_local];
+            return (uint64_t)v.x | ((uint64_t)v.y << 32);
+        }
+        const int nb = r >> 3;                       // 3, 5, 6 or 7 bytes
+        uint64_t v = 0;
+        for (int i = 0; i < nb; ++i) v |= (uint64_t)bits[j_local * nb + i] << (8 * i);
+        return v;
     }
-    if (RP == 16) return reinterpret_cast<const uint16_t *>(bits)[j_local];
-    if (r == 32) return reinterpret_cast<const uint32_t *>(bits)[j_local];
-    if (r == 64) {
-        const uint2 v = reinterpret_cast<const uint2 *>(bits)[j_local];
-        return (uint64_t)v.x | ((uint64_t)v.y << 32);
-    }
-    const int nb = r >> 3;                       // 3, 5, 6 or 7 bytes
+    const int bit = j_local * r, sh = bit & 7;
+    const uint8_t *p = bits + (bit >> 3);
+    const int nb = (sh + r + 7) >> 3;                // 1 .. 9 bytes hold the row
     uint64_t v = 0;
-    for (int i = 0; i < nb; ++i) v |= (uint64_t)bits[j_local * nb + i] << (8 * i);
+    for (int i = 0; i < nb && i < 8; ++i) v |= (uint64_t)p[i] << (8 * i);
+    v >>= sh;
+    if (nb > 8) v |= (uint64_t)p[8] << (64 - sh);    // sh > 0 here
     return v;
 }
 
@@ -590,7 +597,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 // 4 bits at bit 16 ks
                 typedef typename std::conditional<(RP > 32), uint64_t, uint32_t>::type bits_t;
                 bits_t rb[8];
-                if (RP == 16) {
+                if (RP == 16 && r == 16) {
                     // rows jb - (g&1) .. + 15 are 16 half-words: word i holds rows 2i (low) and 2i+1
                     const uint4 w0 = *reinterpret_cast<const uint4 *>(bits + 2 * (jb - (g & 1)));
                     const uint4 w1 = *reinterpret_cast<const uint4 *>(bits + 2 * (jb - (g & 1)) + 16);
@@ -838,9 +845,7 @@ bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
     if ((dtype != LORDBA_BF16 && dtype != LORDBA_F16) || T < 1 || T > (1 << 30)) return false;
     const int ell = ((p.flags >> 8) & 0xf) + 1;
     if (ell > 2 || (ell == 2 && p.r > 32)) return false;    // more envelopes, or two at high rank: FMA kernel
-    // ranks: multiples of 8, and the small powers of two (their B_sign rows do not straddle bytes)
-    const bool small_rank = (p.r == 1 || p.r == 2 || p.r == 4);
-    if ((p.r % 8 != 0 && !small_rank) || p.r < 1 || p.r > kMaxRank) return false;
+    if (p.r < 1 || p.r > kMaxRank) return false;
     // a carrier is copied as whole 64-byte rows of sign bytes
     if ((p.d_in * p.r) % 512 != 0 || (p.d_out * p.r) % 512 != 0) return false;
     // whole 64-column groups (the 3-D tensor view), 16-byte aligned rows
@@ -877,7 +882,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
         const lordba_proj *sel[kMaxBatch];
         int64_t sel_T[kMaxBatch];
-        int m = 0, max_r = 0, min_r = kMaxRank;
+        int m = 0, max_r = 0, min_cw = 128;
         int64_t min_dout = (int64_t)1 << 40;
         for (int i = 0; i <= n; ++i) {
             const bool take = (i < n) && tokens[i] > 0 && padded_rank(projs[i].r) == rp &&
@@ -886,7 +891,9 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                 sel_T[m] = tokens[i];
                 sel[m++] = &projs[i];
                 if (projs[i].r > max_r) max_r = projs[i].r;
-                if (projs[i].r < min_r) min_r = projs[i].r;
+                // narrowest y item of this projection: its sign bytes must be whole 64-byte rows
+                const int need_cw = (projs[i].r % 4 == 0) ? 128 : (projs[i].r % 2 == 0) ? 256 : 512;
+                if (need_cw > min_cw) min_cw = need_cw;
                 if (projs[i].d_out < min_dout) min_dout = projs[i].d_out;
             }
             if (m == kMaxBatch || (i == n && m > 0)) {
@@ -929,8 +936,6 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                 const int nw = (all_tiles > sms || overlaps_neighbours) ? 8 : kMaxWarps;
                 const int max_chunk = nw * kGroup;
                 const int smem_budget = (nw == kMaxWarps) ? kSmemBudget : kSmemBudgetHalf;
-                // narrowest y item: 128 columns, and a whole 64-byte row of sign bytes at any rank
-                const int min_cw = (min_r >= 4) ? 128 : 512 / min_r;
                 int cw = max_chunk;
                 while (cw > min_cw && (min_dout + cw - 1) / cw < want_splits) cw /= 2;
                 int64_t splits = (min_dout + cw - 1) / cw;
@@ -980,7 +985,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                                    : launch_io<kIoF16Exact>(rp, nw, ell, b, prm, grid, plan.total, stream);
                 if (e != cudaSuccess) return LORDBA_ECUDA;
                 count_launch();
-                m = 0; max_r = 0; min_r = kMaxRank; min_dout = (int64_t)1 << 40;
+                m = 0; max_r = 0; min_cw = 128; min_dout = (int64_t)1 << 40;
             }
         }
     }

@@ -188,8 +188,11 @@ SHAPES = [
     (129, 1000, 1032, 16), (130, 4096, 1376, 32), (257, 2048, 520, 64), (9, 64, 64, 64),
     (40, 11008, 128, 16), (260, 640, 11008, 8), (1, 4096, 4096, 16), (200, 4104, 4104, 24),
     (33, 72, 200, 40), (128, 128, 128, 16), (127, 192, 136, 8), (385, 1024, 768, 48),
-    # ranks below 8 that the streaming kernel takes (1, 2, 4: several B_sign rows per byte)
+    # ranks below 8 on shapes that the streaming kernel takes (several B_sign rows per byte)
     (300, 1024, 768, 4), (70, 512, 1536, 2), (33, 1024, 512, 1), (1100, 4096, 4096, 4), (9, 11008, 4096, 4),
+    # other ranks that are not multiples of 8 (B_sign rows start at any bit)
+    (150, 1024, 1024, 12), (77, 512, 1024, 3), (260, 4096, 512, 20), (40, 1024, 1024, 57), (64, 512, 512, 63),
+    (31, 2048, 1024, 6), (500, 4096, 4096, 28),
 ]
 
 

@@ -583,3 +583,16 @@ def test_f16_layer_on_the_tcgen05_kernel(oracle, r, scales_f16):
     for p, d in zip(projs, devs):
         assert_close(torch_to_f64(d.y[rows_t]), oracle_forward(oracle, p, rows=rows), "f16",
                      "f16 layer, tcgen05 pinned, r=%d %s" % (r, p.name))
+
+
+def test_f16_mixed_scale_kinds_on_the_tcgen05_kernel(oracle):
+    """One batched call, tcgen05 kernel pinned: projections with declared float16 scales and with
+    float32 scales go out as separate launches that may overlap; every element checked."""
+    T = 300
+    ps = [workloads.make_projection(di, do, 64, T, "f16", seed=7000 + i, scales_f16=ex)
+          for i, (di, do, ex) in enumerate([(1024, 768, True), (512, 1024, False), (768, 512, True), (1024, 1024, False)])]
+    ds = [DeviceProj(p) for p in ps]
+    lordba.set_variant(lordba.VARIANT_TC)
+    lordba.adapter_forward_batched([d.proj() for d in ds], T, lordba.F16)
+    for p, d in zip(ps, ds):
+        assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "f16", "f16 mixed tcgen05 " + str(p.meta["seed"]))

@@ -281,32 +281,25 @@ __device__ __forceinline__ uint32_t with_signs(uint32_t operand, uint32_t bits)
 }
 
 // The r sign bits of row j_local of an item's slice of B_sign, which is the dense bit stream of
-// the rows: r/8 whole bytes per row when r is a multiple of 8, else a row starts at bit j_local * r
-// and is gathered byte by byte.  Bits above the row's r belong to other rows and are harmless
+// the rows: one aligned load when r is 8, 16, 32 or 64, else a row starts at bit j_local * r and
+// is cut out of the words that hold it.  Bits above the row's r belong to other rows and are harmless
 // (those ranks of z are zero).
 template <int RP>
 __device__ __forceinline__ uint64_t b_row_bits(const uint8_t *bits, int j_local, int r)
 {
-    if ((r & 7) == 0) {
+    if (r == RP) {                                   // 8, 16, 32 or 64: one aligned load
         if (RP == 8) return bits[j_local];
         if (RP == 16) return reinterpret_cast<const uint16_t *>(bits)[j_local];
-        if (r == 32) return reinterpret_cast<const uint32_t *>(bits)[j_local];
-        if (r == 64) {
-            const uint2 v = reinterpret_cast<const uint2 *>(bits)[j_local];
-            return (uint64_t)v.x | ((uint64_t)v.y << 32);
-        }
-        const int nb = r >> 3;                       // 3, 5, 6 or 7 bytes
-        uint64_t v = 0;
-        for (int i = 0; i < nb; ++i) v |= (uint64_t)bits[j_local * nb + i] << (8 * i);
-        return v;
+        if (RP == 32) return reinterpret_cast<const uint32_t *>(bits)[j_local];
+        const uint2 v = reinterpret_cast<const uint2 *>(bits)[j_local];
+        return (uint64_t)v.x | ((uint64_t)v.y << 32);
     }
-    const int bit = j_local * r, sh = bit & 7;
-    const uint8_t *p = bits + (bit >> 3);
-    const int nb = (sh + r + 7) >> 3;                // 1 .. 9 bytes hold the row
-    uint64_t v = 0;
-    for (int i = 0; i < nb && i < 8; ++i) v |= (uint64_t)p[i] << (8 * i);
-    v >>= sh;
-    if (nb > 8) v |= (uint64_t)p[8] << (64 - sh);    // sh > 0 here
+    // two or three aligned words hold the row (the slice starts word-aligned; a word past its end
+    // is still inside the slot)
+    const int bit = j_local * r, sh = bit & 31;
+    const uint32_t *w = reinterpret_cast<const uint32_t *>(bits) + (bit >> 5);
+    uint64_t v = ((uint64_t)w[0] | ((uint64_t)w[1] << 32)) >> sh;
+    if (RP > 32 && sh > 0) v |= (uint64_t)w[2] << (64 - sh);
     return v;
 }
 

@@ -281,21 +281,21 @@ __device__ __forceinline__ uint32_t with_signs(uint32_t operand, uint32_t bits)
 }
 
 // The r sign bits of row j_local of an item's slice of B_sign, which is the dense bit stream of
-// the rows: one aligned load when r is 8, 16, 32 or 64, else a row starts at bit j_local * r and
-// is cut out of the words that hold it.  Bits above the row's r belong to other rows and are harmless
-// (those ranks of z are zero).
-template <int RP>
+// the rows.  GEN = false: r is 8, 16, 32 or 64 and a row is one aligned load.  GEN = true (any
+// other rank, its own instantiations so that the common ranks keep their code): a row starts at
+// bit j_local * r and is cut out of the two or three aligned words that hold it (the stream
+// starts word-aligned; a word past its end is still inside the slot).  Bits above the row's r
+// belong to other rows and are harmless: those ranks of z are zero.
+template <int RP, bool GEN>
 __device__ __forceinline__ uint64_t b_row_bits(const uint8_t *bits, int j_local, int r)
 {
-    if (r == RP) {                                   // 8, 16, 32 or 64: one aligned load
+    if (!GEN) {
         if (RP == 8) return bits[j_local];
         if (RP == 16) return reinterpret_cast<const uint16_t *>(bits)[j_local];
         if (RP == 32) return reinterpret_cast<const uint32_t *>(bits)[j_local];
         const uint2 v = reinterpret_cast<const uint2 *>(bits)[j_local];
         return (uint64_t)v.x | ((uint64_t)v.y << 32);
     }
-    // two or three aligned words hold the row (the slice starts word-aligned; a word past its end
-    // is still inside the slot)
     const int bit = j_local * r, sh = bit & 31;
     const uint32_t *w = reinterpret_cast<const uint32_t *>(bits) + (bit >> 5);
     uint64_t v = ((uint64_t)w[0] | ((uint64_t)w[1] << 32)) >> sh;
@@ -311,7 +311,7 @@ enum IoKind {
 };
 
 // RP: rank padded to 8, 16, 32 or 64.
-template <int RP, int NW, int ELL, int IO>
+template <int RP, int NW, int ELL, int IO, bool GEN>
 __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 2)
 mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant__ MmaParams prm)
 {
@@ -590,7 +590,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 // 4 bits at bit 16 ks
                 typedef typename std::conditional<(RP > 32), uint64_t, uint32_t>::type bits_t;
                 bits_t rb[8];
-                if (RP == 16 && r == 16) {
+                if (RP == 16 && !GEN) {
                     // rows jb - (g&1) .. + 15 are 16 half-words: word i holds rows 2i (low) and 2i+1
                     const uint4 w0 = *reinterpret_cast<const uint4 *>(bits + 2 * (jb - (g & 1)));
                     const uint4 w1 = *reinterpret_cast<const uint4 *>(bits + 2 * (jb - (g & 1)) + 16);
@@ -600,7 +600,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     for (int i = 0; i < 8; ++i) rb[i] = (bits_t)(w[i] >> sh);
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) rb[i] = (bits_t)(b_row_bits<RP>(bits, jb + 2 * i, r) >> (4 * q));
+                    for (int i = 0; i < 8; ++i) rb[i] = (bits_t)(b_row_bits<RP, GEN>(bits, jb + 2 * i, r) >> (4 * q));
                 }
                 // The lane's 16 columns are done as two halves of 8 (n-blocks 4cc .. 4cc+3) to keep
                 // the live registers low; the results of both halves leave in one 256-bit store.
@@ -778,13 +778,13 @@ int sm_count()
     return n;
 }
 
-template <int RP, int NW, int ELL, int IO>
+template <int RP, int NW, int ELL, int IO, bool GEN>
 cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem, cudaStream_t stream)
 {
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, []() {
-        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW, ELL, IO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW, ELL, IO, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSmemBudget);
     });
     if (attr_rc != cudaSuccess) return attr_rc;
@@ -803,32 +803,37 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP, NW, ELL, IO>, b, prm);
+    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP, NW, ELL, IO, GEN>, b, prm);
 }
 
-template <int NW, int ELL, int IO>
+template <int NW, int ELL, int IO, bool GEN>
 cudaError_t launch_rank(int rp, const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem, cudaStream_t stream)
 {
     switch (rp) {
-        case 8:  return launch_one<8, NW, ELL, IO>(b, prm, grid, smem, stream);
-        case 16: return launch_one<16, NW, ELL, IO>(b, prm, grid, smem, stream);
-        case 32: return launch_one<32, NW, ELL, IO>(b, prm, grid, smem, stream);
+        case 8:  return launch_one<8, NW, ELL, IO, GEN>(b, prm, grid, smem, stream);
+        case 16: return launch_one<16, NW, ELL, IO, GEN>(b, prm, grid, smem, stream);
+        case 32: return launch_one<32, NW, ELL, IO, GEN>(b, prm, grid, smem, stream);
         default:
             // two envelopes at rank 64 do not fit the register budget: mma_supported() keeps them out
-            if (ELL == 1) return launch_one<64, NW, 1, IO>(b, prm, grid, smem, stream);
+            if (ELL == 1) return launch_one<64, NW, 1, IO, GEN>(b, prm, grid, smem, stream);
             return cudaErrorInvalidValue;
     }
 }
 
 template <int IO>
-cudaError_t launch_io(int rp, int nw, int ell, const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem,
-                      cudaStream_t stream)
+cudaError_t launch_io(int rp, int nw, int ell, bool gen, const MmaBatch &b, const MmaParams &prm, dim3 grid,
+                      size_t smem, cudaStream_t stream)
 {
+    if (gen) {      // ranks other than 8 / 16 / 32 / 64: one envelope only (mma_supported())
+        if (ell != 1) return cudaErrorInvalidValue;
+        return nw == kMaxWarps ? launch_rank<kMaxWarps, 1, IO, true>(rp, b, prm, grid, smem, stream)
+                               : launch_rank<8, 1, IO, true>(rp, b, prm, grid, smem, stream);
+    }
     if (ell == 1)
-        return nw == kMaxWarps ? launch_rank<kMaxWarps, 1, IO>(rp, b, prm, grid, smem, stream)
-                               : launch_rank<8, 1, IO>(rp, b, prm, grid, smem, stream);
-    return nw == kMaxWarps ? launch_rank<kMaxWarps, 2, IO>(rp, b, prm, grid, smem, stream)
-                           : launch_rank<8, 2, IO>(rp, b, prm, grid, smem, stream);
+        return nw == kMaxWarps ? launch_rank<kMaxWarps, 1, IO, false>(rp, b, prm, grid, smem, stream)
+                               : launch_rank<8, 1, IO, false>(rp, b, prm, grid, smem, stream);
+    return nw == kMaxWarps ? launch_rank<kMaxWarps, 2, IO, false>(rp, b, prm, grid, smem, stream)
+                           : launch_rank<8, 2, IO, false>(rp, b, prm, grid, smem, stream);
 }
 
 }  // namespace
@@ -838,6 +843,7 @@ bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
     if ((dtype != LORDBA_BF16 && dtype != LORDBA_F16) || T < 1 || T > (1 << 30)) return false;
     const int ell = ((p.flags >> 8) & 0xf) + 1;
     if (ell > 2 || (ell == 2 && p.r > 32)) return false;    // more envelopes, or two at high rank: FMA kernel
+    if (ell == 2 && p.r != padded_rank(p.r)) return false;   // two envelopes: ranks 8, 16, 32 only
     if (p.r < 1 || p.r > kMaxRank) return false;
     // a carrier is copied as whole 64-byte rows of sign bytes
     if ((p.d_in * p.r) % 512 != 0 || (p.d_out * p.r) % 512 != 0) return false;
@@ -872,6 +878,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
     };
     for (int io = io_first; io <= io_last; ++io)
     for (int ell = 1; ell <= 2; ++ell)
+    for (int gen = 0; gen <= (ell == 1 ? 1 : 0); ++gen)
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
         const lordba_proj *sel[kMaxBatch];
         int64_t sel_T[kMaxBatch];
@@ -879,7 +886,8 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
         int64_t min_dout = (int64_t)1 << 40;
         for (int i = 0; i <= n; ++i) {
             const bool take = (i < n) && tokens[i] > 0 && padded_rank(projs[i].r) == rp &&
-                              ((projs[i].flags >> 8) & 0xf) + 1 == ell && io_of(projs[i]) == io;
+                              ((projs[i].flags >> 8) & 0xf) + 1 == ell && io_of(projs[i]) == io &&
+                              (projs[i].r != rp) == (gen != 0);
             if (take) {
                 sel_T[m] = tokens[i];
                 sel[m++] = &projs[i];
@@ -973,9 +981,9 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                 prm.slots = slots;
                 const dim3 grid((unsigned)tiles, (unsigned)m, (unsigned)splits);
                 const cudaError_t e =
-                    io == kIoBf16 ? launch_io<kIoBf16>(rp, nw, ell, b, prm, grid, plan.total, stream)
-                    : io == kIoF16 ? launch_io<kIoF16>(rp, nw, ell, b, prm, grid, plan.total, stream)
-                                   : launch_io<kIoF16Exact>(rp, nw, ell, b, prm, grid, plan.total, stream);
+                    io == kIoBf16 ? launch_io<kIoBf16>(rp, nw, ell, gen != 0, b, prm, grid, plan.total, stream)
+                    : io == kIoF16 ? launch_io<kIoF16>(rp, nw, ell, gen != 0, b, prm, grid, plan.total, stream)
+                                   : launch_io<kIoF16Exact>(rp, nw, ell, gen != 0, b, prm, grid, plan.total, stream);
                 if (e != cudaSuccess) return LORDBA_ECUDA;
                 count_launch();
                 m = 0; max_r = 0; min_cw = 128; min_dout = (int64_t)1 << 40;

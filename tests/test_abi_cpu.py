@@ -115,3 +115,33 @@ def test_bad_arguments_return_codes_without_launching(lib):
     assert lib.lordba_set_variant(lordba.VARIANT_FMA) == 0 and lordba.get_variant() == lordba.VARIANT_FMA
     assert lib.lordba_set_variant(lordba.VARIANT_AUTO) == 0
     assert lordba.launch_count() == before
+
+
+def test_float16_arguments_and_inputs_without_launching(lib):
+    """The float16 element type, the declared-scales flag and the scale widening entry: argument
+    checks that return before any launch, and the seeded float16 inputs."""
+    import numpy as np
+    from paper_2605_24058_b200 import lordba, workloads
+    EINVAL, EUNSUP, EALIGN = 1, 2, 3
+    call = lambda p, T=4, dt=lordba.F16: lib.lordba_adapter_forward_ex(ctypes.byref(p), T, dt, None)
+    assert call(_proj(lordba, flags=lordba.PROJ_SCALES_F16), T=0) == 0
+    assert call(_proj(lordba, flags=lordba.PROJ_SCALES_F16 | lordba.PROJ_OVERLAP), T=0) == 0
+    assert call(_proj(lordba, x=0x1001)) == EALIGN                    # 2-byte elements
+    assert call(_proj(lordba, flags=4), T=0) == EINVAL
+    assert lib.lordba_scales_from_f16(0x1000, 0x2000, -1, None) == EINVAL
+    assert lib.lordba_scales_from_f16(None, 0x2000, 4, None) == EINVAL
+    assert lib.lordba_scales_from_f16(0x1001, 0x2000, 4, None) == EALIGN
+    assert lib.lordba_scales_from_f16(0x1000, 0x2002, 4, None) == EALIGN
+    assert lib.lordba_scales_from_f16(None, None, 0, None) == 0
+    # inputs: float16 x / y are the float32 draws rounded to nearest even; exported scales are
+    # float16 values held in float32
+    a = workloads.make_projection(64, 128, 8, 5, "f32", seed=3)
+    b = workloads.make_projection(64, 128, 8, 5, "f16", seed=3, scales_f16=True)
+    assert b.x.dtype == np.float16 and b.y.dtype == np.float16
+    assert np.array_equal(b.x, a.x.astype(np.float16)) and np.array_equal(b.y, a.y.astype(np.float16))
+    for name in ("s_in", "s_r", "s_out"):
+        got, src = getattr(b, name), getattr(a, name)
+        assert got.dtype == np.float32
+        assert np.array_equal(got, src.astype(np.float16).astype(np.float32))
+    assert np.array_equal(a.A_sign, b.A_sign) and np.array_equal(a.B_sign, b.B_sign)
+    assert b.x_f64().dtype == np.float64 and np.array_equal(b.x_f64(), b.x.astype(np.float64))

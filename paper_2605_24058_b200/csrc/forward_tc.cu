@@ -84,7 +84,6 @@ struct alignas(64) TcProj {
     const float *s_out;
     int d_in, d_out;
     int nk, nn;            // 64-column chunks of d_in / d_out
-    int words_a;           // uint32 words per row of packed_A
 };
 
 struct TcBatch {
@@ -1155,7 +1154,6 @@ int launch_forward_tc(const lordba_proj *projs, int n, int64_t T, int dtype, cud
                 t.d_in = (int)q.d_in; t.d_out = (int)q.d_out;
                 t.nk = (int)((q.d_in + kChunk - 1) / kChunk);
                 t.nn = (int)((q.d_out + kChunk - 1) / kChunk);
-                t.words_a = (int)((q.d_in + 31) / 32);
             }
             b.n_proj = m;
             b.total_tiles = m * tiles_per_proj;

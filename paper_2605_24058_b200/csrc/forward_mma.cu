@@ -911,14 +911,11 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                     }
                     sel[b + 1] = pa; sel_T[b + 1] = ta;
                 }
-                // Tile height: the smallest number of full waves of 16-row tiles, then the rows
-                // per tile that spread the tokens evenly over those waves.
-                int64_t min_tiles = 0, sum_T = 0;
-                for (int k = 0; k < m; ++k) { min_tiles += (sel_T[k] + kTile - 1) / kTile; sum_T += sel_T[k]; }
-                const int64_t waves = (min_tiles + sms - 1) / sms;
-                int64_t rows = (sum_T + waves * sms - 1) / (waves * sms);
-                if (rows > kTile) rows = kTile;
-                if (rows < 1) rows = 1;
+                // Tile height: always the full 16 rows of an MMA tile.  Shorter tiles that spread a
+                // call evenly over whole waves of SMs (14 rows for T = 2048) were measured slower at
+                // every size from 8 to 4096 tokens: an MMA costs the same with 14 or 16 live rows,
+                // and fewer, fuller CTAs leave room for the neighbouring calls' CTAs.
+                const int64_t rows = kTile;
                 int64_t tiles = 0, all_tiles = 0;      // widest projection (grid.x), and the sum
                 for (int k = 0; k < m; ++k) {
                     const int64_t tk = (sel_T[k] + rows - 1) / rows;

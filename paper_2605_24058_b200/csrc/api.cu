@@ -83,7 +83,7 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, 
     // Split the list: what the chosen tensor-core kernel can take, and the rest.  Left to itself
     // the library takes the tcgen05 kernel where it was measured ahead of the streaming one: ranks
     // above 32 from 32 tiles of 128 tokens (one projection at T = 4096, a layer at T = 2048), ranks
-    // 24 and 32 from two waves of such tiles.  (That kernel wants one token count for all
+    // 24 and 32 from eight waves of such tiles (below that the streaming kernel is ahead).  (That kernel wants one token count for all
     // projections.)
     bool use_tc = (variant == LORDBA_VARIANT_TC);
     if (use_tc && tokens) return LORDBA_EUNSUPPORTED;
@@ -95,7 +95,7 @@ int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, 
             all_high = all_high && projs[i].r > 32;
             tiles += T / 128;
         }
-        use_tc = all_ok && tiles >= (all_high ? 32 : 2 * 148);
+        use_tc = all_ok && tiles >= (all_high ? 32 : 8 * 148);
     }
     std::vector<lordba_proj> fast, fma;
     std::vector<int64_t> fast_rows, fma_rows;

@@ -7,9 +7,10 @@
 // flops on them, so it is bound by HBM as long as the two sign products cost
 // next to nothing and the memory system always has requests queued.
 //
-//   * One CTA owns `rows` <= 16 consecutive tokens (chosen on the host so that
-//     the tiles of a call fill the SMs evenly) and needs no other CTA: the
-//     16 x r intermediate lives in registers and shared memory.
+//   * One CTA owns `rows` <= 16 consecutive tokens (the host passes 16, the
+//     height of an MMA tile: shorter tiles that fill the SMs more evenly were
+//     measured slower) and needs no other CTA: the 16 x r intermediate lives
+//     in registers and shared memory.
 //   * A producer warp streams the CTA's rows of x, then of y, through a ring of
 //     shared-memory slots, NW x 64 columns per item (NW = consumer warps), with
 //     ONE tensor copy per item: the row-major matrix is described to TMA as a

@@ -10,10 +10,23 @@ d_in = d_out = 4096, r = 16, T = 2048 tokens, bf16 activations, float32 scales.
 Prints ONE JSON line.  `value` is adapter-branch tokens/s with the inputs
 resident in HBM; consecutive steps rotate through buffer sets whose total size
 exceeds the L2 several times over, so every step reads x and y from DRAM.
+
+Timing.  Every timed step is a node of a replayed CUDA graph (no call is issued
+from Python inside a timed region): the K steps are the replays of an
+n-step graph (n = number of buffer sets) plus one graph holding the K mod n
+remainder.  The region "W warm-up steps, event, K steps, event" is repeated
+back to back (>= 30 times, and until the GPU has been busy for about 0.1 s so
+that the clock sampler sees it); `ms_per_step` is the median over the repeats
+and `repeat_spread` gives p10 / p90.
+
 `e2e` is the same metric through lordba_adapter_forward_host with pinned host
 buffers (H2D of x and y and D2H of y inside the timed region).  `roofline`
 relates the kernel's algorithmic bytes per launch to the measured HBM copy peak.
 `cpu_baseline` is the float64 oracle timed on this machine's host cores.
+`workloads` (one GPU only) times the other configurations the same way: the MLP
+projections, a layer's seven projections in one batched call, the full
+224-projection set over the rank sweep, decode calls, multi-envelope and
+multi-adapter calls, each with the kernel family the library chose.
 
 With --gpus N > 1 (under torchrun) every rank runs the same step on its own
 token shard of T tokens (weak scaling, no collective on the data path).
@@ -37,6 +50,8 @@ if ROOT not in sys.path:
 from paper_2605_24058_b200 import workloads  # noqa: E402
 
 METRIC = "adapter-branch tokens/s at r=16, T=2048 (LLaMA-2-7B attention projection 4096->4096, bf16)"
+WORKLOAD = ("config1: LLaMA-2-7B attention projection adapter, d_in=d_out=4096, r=16, "
+            "T=2048 tokens per GPU per step, bf16 x/y, fp32 scales")
 UNIT = "tokens/s"
 D_IN = D_OUT = workloads.HIDDEN
 R = 16
@@ -44,10 +59,12 @@ T = 2048
 ELEM = 2
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
+MIN_REPEATS = 30
+MIN_BUSY_S = 0.1
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel on this workload
-# (ncu capture summarised under profiles/; reads only, the write-back L2 defers the y writes past
-# the end of the kernel).  Set to None whenever the kernel changes after the capture.
-NCU_DRAM_BYTES_PER_LAUNCH = 33633792
+# (ncu capture summarised under profiles/).  None whenever the kernel has changed since the capture.
+NCU_DRAM_BYTES_PER_LAUNCH = None
+VARIANT_NAMES = {0: "auto", 1: "fma", 2: "tc", 3: "mma"}
 
 
 def ensure_library():
@@ -70,7 +87,7 @@ def measured_peak():
 class ClockSampler(threading.Thread):
     """Polls SM clock and throttle reasons through NVML (read-only) while the GPU is busy."""
 
-    def __init__(self, index: int, period_s: float = 0.004):
+    def __init__(self, index: int, period_s: float = 0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -162,14 +179,14 @@ def run_reference(args):
     time_oracle(p, tokens, max(0, args.warmup))
     dt, cores = time_oracle(p, tokens, args.steps)
     value = args.steps * tokens / dt
-    sample = "each step = the oracle over %d of the step's %d tokens" % (tokens, T)
+    sample = ("each step = the float64 oracle (bf16 inputs widened to f64) over %d of the step's %d tokens"
+              % (tokens, T))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": "config1: attn 4096->4096, r=16, T=2048, bf16 inputs widened to f64",
-                   "sample": sample},
+        "config": {"workload": WORKLOAD, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -178,7 +195,7 @@ def run_reference(args):
     return 0
 
 
-# ----------------------------------------------------------------------------- GPU arm
+# ----------------------------------------------------------------------------- timing helpers
 
 def max_over_ranks(values, device=None):
     """The slowest rank's timings: element-wise MAX over the ranks of the default process group
@@ -196,6 +213,232 @@ def aggregate_tokens_per_s(world, tokens_per_rank_step, steps, ms):
     """Whole-job throughput: what all ranks processed divided by the slowest rank's time."""
     return world * tokens_per_rank_step * steps / (ms * 1e-3)
 
+
+def split_steps(k: int, n: int):
+    """k steps as (full replays of an n-step graph, steps of the remainder graph)."""
+    return k // n, k % n
+
+
+def repeats_for(region_s: float, min_repeats: int = MIN_REPEATS, min_busy_s: float = MIN_BUSY_S,
+                max_repeats: int = 2000) -> int:
+    """How often a timed region is repeated: at least min_repeats, and until the GPU has been busy
+    for about min_busy_s (bounded)."""
+    if region_s <= 0.0:
+        return max_repeats
+    return int(max(min_repeats, min(max_repeats, np.ceil(min_busy_s / region_s))))
+
+
+class GraphSteps:
+    """Steps 0, 1, 2, ... of a workload as replayed CUDA graphs: one graph of n steps and, on
+    demand, graphs of the first m < n steps for remainders."""
+
+    def __init__(self, step, n: int, stream):
+        import torch
+        self.torch, self.step, self.n, self.stream = torch, step, n, stream
+        self.graphs = {}
+
+    def graph(self, m: int):
+        if m not in self.graphs:
+            g = self.torch.cuda.CUDAGraph()
+            with self.torch.cuda.graph(g, stream=self.stream):
+                for i in range(m):
+                    self.step(i)
+            self.graphs[m] = g
+        return self.graphs[m]
+
+    def prepare(self, k: int):
+        full, rem = split_steps(k, self.n)
+        if full:
+            self.graph(self.n)
+        if rem:
+            self.graph(rem)
+
+    def run(self, k: int):
+        """Enqueue exactly k steps, all of them graph nodes."""
+        full, rem = split_steps(k, self.n)
+        for _ in range(full):
+            self.graphs[self.n].replay()
+        if rem:
+            self.graphs[rem].replay()
+
+
+def time_regions(gs: GraphSteps, steps: int, warmup: int, repeats: int):
+    """`repeats` times back to back on the graphs' stream: `warmup` untimed steps, an event, `steps`
+    timed steps, an event.  The untimed steps keep the GPU busy while the timed graphs are
+    enqueued, so no launch latency sits between the first event and the first timed kernel.
+    Returns the milliseconds of every timed region."""
+    torch = gs.torch
+    gs.prepare(steps)
+    gs.prepare(warmup)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(repeats)]
+    for a, b in ev:
+        gs.run(warmup)
+        a.record(gs.stream)
+        gs.run(steps)
+        b.record(gs.stream)
+    gs.stream.synchronize()
+    return np.array([a.elapsed_time(b) for a, b in ev])
+
+
+def timed(gs: GraphSteps, steps: int, warmup: int, min_repeats: int = MIN_REPEATS, min_busy_s: float = MIN_BUSY_S):
+    """Probe the region once to size the repeat count, then time it.  Returns the per-region ms."""
+    probe = time_regions(gs, steps, warmup, 3)
+    region_s = float(np.median(probe)) * 1e-3 * (1.0 + warmup / max(1, steps))
+    return time_regions(gs, steps, warmup, repeats_for(region_s, min_repeats, min_busy_s))
+
+
+# ----------------------------------------------------------------------------- the other workloads
+
+def _variant_of(lordba, projs, tokens, code):
+    """Kernel families the library takes for a call (names, deduplicated, in order)."""
+    fams = lordba.query_variant(projs, tokens, code)
+    out = []
+    for f in fams:
+        name = VARIANT_NAMES.get(f, str(f))
+        if name not in out:
+            out.append(name)
+    return "+".join(out)
+
+
+class DeviceWorkload:
+    """Device-generated inputs of one supplementary workload: `shapes` projections of rank r (ell
+    envelopes) over Tn tokens, n_sets rotating sets of x / y buffers, one library call per step."""
+
+    def __init__(self, lordba, dev, shapes, r, Tn, ell=1, dtype="bf16", scales_f16=False, segments=0,
+                 overlap=True, seed=1234, mem_cap=40e9, shared=None):
+        import torch
+        self.torch, self.lordba = torch, lordba
+        self.shapes, self.r, self.Tn, self.ell, self.segments = shapes, r, Tn, ell, segments
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(seed)
+        io_t, self.code = {"bf16": (torch.bfloat16, lordba.BF16), "f16": (torch.float16, lordba.F16)}[dtype]
+        esh = (ell,) if ell > 1 else ()          # (ell, d) scales: a multi-envelope adapter (Eq. 4)
+        # an adapter exported with half-precision scales: values rounded to float16, declared to the library
+        exported = (lambda s: s.to(torch.float16).to(torch.float32)) if scales_f16 else (lambda s: s)
+        self.base_flags = lordba.PROJ_SCALES_F16 if scales_f16 else 0
+
+        def rand_signs(rows, cols):
+            return torch.randint(0, 2, (rows, cols), device=dev, generator=gen, dtype=torch.int8) * 2 - 1
+
+        self.adapters = []
+        for di, do in shapes:
+            self.adapters.append(dict(
+                pa=lordba.pack_signs(rand_signs(r, di), 0), pb=lordba.pack_signs(rand_signs(do, r), 1),
+                s_in=exported(torch.exp(0.5 * torch.randn(*esh, di, device=dev, generator=gen))),
+                s_r=exported(64.0 * (0.02 * torch.randn(*esh, r, device=dev, generator=gen)).abs()),
+                s_out=exported(torch.exp(0.5 * torch.randn(*esh, do, device=dev, generator=gen)))))
+        self.set_bytes = sum(Tn * (di + do) * ELEM for di, do in shapes)
+        self.alg_bytes = sum(workloads.algorithmic_bytes(Tn, di, do, r, ELEM) + 4 * (ell - 1) * (di + r + do)
+                             for di, do in shapes)
+        n_sets = int(max(1, min(np.ceil(8 * L2_BYTES / self.set_bytes), mem_cap // self.set_bytes)))
+        if self.set_bytes > 2 * L2_BYTES:
+            n_sets = 1                   # one set already exceeds the L2: every step re-reads it from DRAM
+        self.n_sets = n_sets
+        if shared is not None and shared.get("key") == (tuple(shapes), Tn, dtype, n_sets):
+            self.sets = shared["sets"]   # x / y do not depend on the adapters: reused across a rank sweep
+        else:
+            self.sets = [[(torch.randn(Tn, di, device=dev, generator=gen, dtype=torch.float32).to(io_t),
+                           torch.randn(Tn, do, device=dev, generator=gen, dtype=torch.float32).to(io_t))
+                          for di, do in shapes] for _ in range(n_sets)]
+            if shared is not None:
+                shared["key"], shared["sets"] = (tuple(shapes), Tn, dtype, n_sets), self.sets
+        self.overlap_ok = n_sets > 1 and overlap
+        self.n_graph = max(n_sets, 4)
+
+    def projs(self, i):
+        flags = self.base_flags | (self.lordba.PROJ_OVERLAP if (self.overlap_ok and i % self.n_sets != 0) else 0)
+        return [self.lordba.make_proj(x, a["pa"], a["pb"], a["s_in"], a["s_r"], a["s_out"], y, self.r, flags)
+                for (x, y), a in zip(self.sets[i % self.n_sets], self.adapters)]
+
+    def tokens(self):
+        return [self.Tn] * len(self.shapes)
+
+    def step(self, i):
+        projs = self.projs(i)
+        if self.segments:
+            # multi-adapter batch: segments of Tn tokens, one adapter each, one call
+            self.lordba.adapter_forward_segments(projs, self.tokens(), self.code)
+        elif len(projs) == 1:
+            self.lordba.adapter_forward_ex(projs[0], self.Tn, self.code)
+        else:
+            self.lordba.adapter_forward_batched(projs, self.Tn, self.code)
+
+    def variant(self):
+        return _variant_of(self.lordba, self.projs(1), self.tokens(), self.code)
+
+
+def time_workload(w: DeviceWorkload, stream, steps: int, warmup: int, min_repeats=MIN_REPEATS, min_busy_s=MIN_BUSY_S):
+    """Times one supplementary workload (graph replay, rotating buffers); returns the summary dict."""
+    torch, lordba = w.torch, w.lordba
+    with torch.cuda.stream(stream):
+        for i in range(min(w.n_graph, 4)):
+            w.step(i)
+        stream.synchronize()
+        gs = GraphSteps(w.step, w.n_graph, stream)
+        n0 = lordba.launch_count()
+        gs.graph(w.n_graph)
+        launches_per_step = (lordba.launch_count() - n0) / w.n_graph
+        ms = timed(gs, steps, warmup, min_repeats, min_busy_s)
+    if lordba.device_status() != 0:
+        raise RuntimeError("device status word set")
+    peak, peak_kind = measured_peak()
+    med = float(np.median(ms)) / steps
+    achieved = w.alg_bytes / (med * 1e-3) / 1e9
+    return {"us_per_call": med * 1e3, "p10_us": float(np.percentile(ms, 10)) / steps * 1e3,
+            "p90_us": float(np.percentile(ms, 90)) / steps * 1e3, "gbs": achieved, "frac": achieved / peak,
+            "peak_kind": "of " + peak_kind, "variant": w.variant(), "launches_per_call": launches_per_step,
+            "steps": steps, "repeats": int(len(ms)), "buffer_sets": w.n_sets, "alg_bytes": w.alg_bytes,
+            "step_dependency": "declared independent" if w.overlap_ok else "each call waits for the previous one"}
+
+
+def supplementary_workloads(lordba, dev, stream, sampler):
+    """Configs 2 to 4 and the widened rows, each as {us_per_call, gbs, frac, variant, ...}."""
+    import torch
+    H, F = workloads.HIDDEN, workloads.FFN
+    layer = [(di, do) for _, di, do in workloads.LAYER_PROJECTIONS]
+    full = layer * workloads.N_LAYERS
+    out = {}
+
+    def run(name, steps, warmup, shared=None, min_repeats=MIN_REPEATS, min_busy_s=0.03, **kw):
+        w = DeviceWorkload(lordba, dev, shared=shared, **kw)
+        sampler.recording = True
+        out[name] = time_workload(w, stream, steps, warmup, min_repeats, min_busy_s)
+        sampler.recording = False
+        del w
+        if shared is None:
+            torch.cuda.empty_cache()
+
+    # config 2: the MLP projections; config 1's shape when every call waits for the one before it
+    run("gate_T2048_r16", 20, 5, shapes=[(H, F)], r=16, Tn=2048)
+    run("down_T2048_r16", 20, 5, shapes=[(F, H)], r=16, Tn=2048)
+    run("attn_T2048_r16_dependent", 20, 5, shapes=[(H, H)], r=16, Tn=2048, overlap=False)
+    # a layer's seven projections in one batched call (prefill)
+    run("layer_T2048_r16", 8, 4, shapes=layer, r=16, Tn=2048)
+    run("layer_T4096_r16", 8, 4, shapes=layer, r=16, Tn=4096)
+    run("layer_T2048_r32", 8, 4, shapes=layer, r=32, Tn=2048)
+    run("layer_T2048_r64", 8, 4, shapes=layer, r=64, Tn=2048)
+    run("attn_T4096_r64", 20, 5, shapes=[(H, H)], r=64, Tn=4096)
+    run("attn_T2048_r32", 20, 5, shapes=[(H, H)], r=32, Tn=2048)
+    run("attn_T2048_r64", 20, 5, shapes=[(H, H)], r=64, Tn=2048)
+    # multi-envelope adapters (Eq. 4) and a multi-adapter batch (8 adapters x 256 tokens, one call)
+    run("attn_T2048_r16_ell2", 20, 5, shapes=[(H, H)], r=16, Tn=2048, ell=2)
+    run("attn_T2048_r16_ell4", 20, 5, shapes=[(H, H)], r=16, Tn=2048, ell=4)
+    run("attn_T2048_r4_ell2", 20, 5, shapes=[(H, H)], r=4, Tn=2048, ell=2)
+    run("multi_8x256_r16", 20, 5, shapes=[(H, H)] * 8, r=16, Tn=256, segments=8)
+    run("multi_8x256_r32", 20, 5, shapes=[(H, H)] * 8, r=32, Tn=256, segments=8)
+    # config 3: decode, one batched call per layer (latency bound: the figure is us per call)
+    for Tn in (1, 8, 32, 64):
+        run("decode_layer_T%d_r16" % Tn, 32, 8, shapes=layer, r=16, Tn=Tn)
+    # config 4: all 224 projections in one call over the rank sweep (one 15.8 GB buffer set, shared)
+    shared = {}
+    for r in (8, 16, 32, 64):
+        run("full_T2048_r%d" % r, 4, 2, shared=shared, min_repeats=8, min_busy_s=0.02, shapes=full, r=r, Tn=2048)
+    shared.clear()
+    torch.cuda.empty_cache()
+    return out
+
+
+# ----------------------------------------------------------------------------- GPU arm (headline)
 
 def run_gpu(args):
     import torch
@@ -244,7 +487,7 @@ def run_gpu(args):
     if rank == 0:
         import oracle
         # both launch shapes that the timed region uses: step 0 (waits for its predecessor) and
-        # step 1 (declared independent: the two-CTA-per-SM kernel)
+        # step 1 (declared independent)
         step(0)
         step(1)
         torch.cuda.synchronize()
@@ -267,74 +510,44 @@ def run_gpu(args):
                                    "rounding bound held: %s" % (k, parity, tight_ok))
             ys[k].copy_(y_host)
 
-    # one CUDA graph holds n_sets consecutive steps (one per buffer set): launches are then
-    # issued faster than the ~10 us kernels retire.
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     with torch.cuda.stream(stream):
         for i in range(n_sets):
             step(i)
         stream.synchronize()
+        gs = GraphSteps(step, n_sets, stream)
         n0 = lordba.launch_count()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
-            for i in range(n_sets):
-                step(i)
+        gs.graph(n_sets)
         launches_per_step = (lordba.launch_count() - n0) / n_sets
-
-        def run_steps(k):
-            full, rem = divmod(k, n_sets)
-            for _ in range(full):
-                graph.replay()
-            for i in range(rem):
-                step(i)
-
-        sampler = ClockSampler(local_rank)
-        sampler.start()
-        run_steps(args.warmup)
-        stream.synchronize()
+        gs.prepare(args.steps)
+        gs.prepare(args.warmup)
+        probe = time_regions(gs, args.steps, args.warmup, 3)
+        repeats = repeats_for(float(np.median(probe)) * 1e-3 * (1.0 + args.warmup / args.steps))
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         sampler.recording = True
-        e0.record(stream)
-        run_steps(args.steps)
-        e1.record(stream)
-        stream.synchronize()
+        region_ms = time_regions(gs, args.steps, args.warmup, repeats)
         sampler.recording = False
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-
-        # spread of the step time: every replay of the graph (n_sets steps) timed on its own
-        n_spread = int(max(5, min(100, args.steps // n_sets)))
-        marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_spread + 1)]
-        marks[0].record(stream)
-        for k in range(n_spread):
-            graph.replay()
-            marks[k + 1].record(stream)
-        stream.synchronize()
-        spread_us = np.array([marks[k].elapsed_time(marks[k + 1]) for k in range(n_spread)]) * 1e3 / n_sets
+        ms = float(np.median(region_ms))
 
         # the same steps as a chain: no step declared independent, each kernel waits for the one
         # before it (what a caller pays when every call consumes the previous call's output)
-        dep_steps = int(max(n_sets, min(args.steps, 2000) // n_sets * n_sets))
-        dep_graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(dep_graph, stream=stream):
-            for i in range(n_sets):
-                step(i, dependent=True)
-        for _ in range(3):
-            dep_graph.replay()
-        stream.synchronize()
-        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        d0.record(stream)
-        for _ in range(dep_steps // n_sets):
-            dep_graph.replay()
-        d1.record(stream)
-        stream.synchronize()
-        dep_ms = d0.elapsed_time(d1) / dep_steps
+        dep = GraphSteps(lambda i: step(i, dependent=True), n_sets, stream)
+        sampler.recording = True
+        dep_region = timed(dep, args.steps, args.warmup)
+        sampler.recording = False
+        dep_ms = float(np.median(dep_region)) / args.steps
+
+        # the same independent steps issued one by one from the host, no graph: a prepared call
+        # (tensor maps encoded once) against the plain entry point, in microseconds per call
+        eager = eager_loops(lordba, xs, ys, packed_A, packed_B, s_in, s_r, s_out, n_sets, stream)
 
         # end to end through the host-buffer entry point: H2D x, H2D y, kernel, D2H y per step
         ws = torch.empty(lordba.host_workspace_bytes(T, D_IN, D_OUT, lordba.BF16), dtype=torch.uint8,
@@ -351,13 +564,14 @@ def run_gpu(args):
         if world > 1:
             dist.barrier()
         h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.recording = True
         h0.record(stream)
         for _ in range(e2e_steps):
             host_step()
         h1.record(stream)
         stream.synchronize()
+        sampler.recording = False
         e2e_ms = h0.elapsed_time(h1)
-        sampler.stop()
 
     status = lordba.device_status()
     if status != 0:
@@ -365,26 +579,37 @@ def run_gpu(args):
 
     ms, e2e_ms, dep_ms = max_over_ranks([ms, e2e_ms, dep_ms], dev if world > 1 else None)
 
+    extra = None
+    if world == 1 and not args.no_workloads:
+        del xs, ys
+        torch.cuda.empty_cache()
+        extra = supplementary_workloads(lordba, dev, stream, sampler)
+    sampler.stop()
+
     if rank == 0:
         peak, peak_kind = measured_peak()
         alg_bytes = workloads.algorithmic_bytes(T, D_IN, D_OUT, R, ELEM)
         sec_per_step = ms * 1e-3 / args.steps
         achieved = alg_bytes / sec_per_step / 1e9
-        variant = {0: "auto", 1: "fma", 2: "tc", 3: "mma"}[lordba.get_variant()]
+        full, rem = split_steps(args.steps, n_sets)
         line = {
             "metric": METRIC, "value": aggregate_tokens_per_s(world, T, args.steps, ms), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "config1: LLaMA-2-7B attention projection adapter, d_in=d_out=4096, "
-                                   "r=16, T=2048 tokens per GPU per step, bf16 x/y, fp32 scales",
+            "config": {"workload": WORKLOAD,
                        "l2": "steps rotate through %d device buffer sets (%.0f MB > 8 x L2)"
                              % (n_sets, n_sets * set_bytes / 1e6),
-                       "launch": "CUDA graph of %d steps replayed" % n_sets,
+                       "launch": "every timed step is a CUDA-graph node: %d replay(s) of a %d-step graph + one "
+                                 "%d-step graph; no call is issued from Python inside a timed region"
+                                 % (full, n_sets, rem),
+                       "timing": "median over %d back-to-back repeats of (W warm-up steps, event, K steps, event)"
+                                 % repeats,
                        "step_dependency": "every step waits for the previous one" if args.no_overlap else
                                           "steps after the first of a graph are declared independent "
                                           "(LORDBA_PROJ_OVERLAP): they may overlap the previous step's tail",
-                       "kernel_variant": variant, "parallelism": "token shards, no collective",
+                       "kernel_variant": VARIANT_NAMES[lordba.get_variant()],
+                       "parallelism": "token shards, no collective",
                        "parity_max_err_over_rms": parity},
             "hbm_gbs": achieved,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -395,15 +620,20 @@ def run_gpu(args):
                     "h2d_bytes_per_step": (T * D_IN + T * D_OUT) * ELEM,
                     "d2h_bytes_per_step": T * D_OUT * ELEM, "steps": e2e_steps},
             "gpu_launches": int(round(launches_per_step * args.steps)),
+            "timed_steps_are": "graph replays",
             "clocks": sampler.summary(),
-            # per-step time over single graph replays (this rank): the timed region's figure is the mean
-            "step_us_spread": {"p10": float(np.percentile(spread_us, 10)), "median": float(np.median(spread_us)),
-                               "p90": float(np.percentile(spread_us, 90)), "replays": n_spread,
-                               "steps_per_replay": n_sets},
+            # the timed region repeated back to back (this rank): ms_per_step is the median
+            "repeat_spread": {"repeats": repeats, "p10_ms_per_step": float(np.percentile(region_ms, 10)) / args.steps,
+                              "median_ms_per_step": float(np.median(region_ms)) / args.steps,
+                              "p90_ms_per_step": float(np.percentile(region_ms, 90)) / args.steps},
             # the same workload with every step waiting for the one before it (not the headline)
             "dependent_steps": {"ms_per_step": dep_ms, "value": world * T / (dep_ms * 1e-3), "unit": UNIT,
-                                "roofline_frac": alg_bytes / (dep_ms * 1e-3) / 1e9 / peak, "steps": dep_steps},
+                                "roofline_frac": alg_bytes / (dep_ms * 1e-3) / 1e9 / peak,
+                                "steps": args.steps, "repeats": int(len(dep_region))},
+            "eager_calls": eager,
         }
+        if extra is not None:
+            line["workloads"] = extra
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(p)
         print(json.dumps(line))
@@ -412,12 +642,49 @@ def run_gpu(args):
     return 0
 
 
-# ----------------------------------------------------------------------------- other workloads
+def eager_loops(lordba, xs, ys, packed_A, packed_B, s_in, s_r, s_out, n_sets, stream, calls=1000):
+    """1000 independent config-1 calls issued from the host without a graph: microseconds per call
+    (device time between two events, host bound) for the plain entry point and for prepared calls,
+    whose tensor maps and launch parameters were built once by lordba_plan_init."""
+    import torch
+    out = {"calls": calls}
+    flags = lambda i: lordba.PROJ_OVERLAP if i % n_sets else 0
+    projs = [lordba.make_proj(xs[i], packed_A, packed_B, s_in, s_r, s_out, ys[i], R, flags(i)) for i in range(n_sets)]
+    plans = [lordba.plan_init([projs[i]], [T], lordba.BF16) for i in range(n_sets)]
+    lib = lordba.load()
+    s = int(stream.cuda_stream)
+    import ctypes
+
+    def plain(i):
+        rc = lib.lordba_adapter_forward_ex(ctypes.byref(projs[i % n_sets]), T, lordba.BF16, s)
+        if rc:
+            raise RuntimeError("lordba_adapter_forward_ex: %d" % rc)
+
+    def planned(i):
+        rc = lib.lordba_adapter_forward_planned(plans[i % n_sets].ptr, s)
+        if rc:
+            raise RuntimeError("lordba_adapter_forward_planned: %d" % rc)
+
+    for name, fn in (("plain_us_per_call", plain), ("planned_us_per_call", planned)):
+        for i in range(50):
+            fn(i)
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(calls):
+            fn(i)
+        e1.record(stream)
+        stream.synchronize()
+        out[name] = e0.elapsed_time(e1) * 1e3 / calls
+    return out
+
+
+# ----------------------------------------------------------------------------- one other workload (CLI)
 
 def run_workload(args):
-    """The other configurations (single GPU, device-generated inputs, no oracle leg): one step =
-    ONE library call, single or batched.  Prints the same kind of JSON line; parity of these shapes
-    is covered by the GPU tests, not here."""
+    """One of the other configurations (single GPU, device-generated inputs, no oracle leg): one
+    step = ONE library call, single or batched.  Prints the same kind of JSON line; parity of these
+    shapes is covered by the GPU tests, not here."""
     import torch
     from paper_2605_24058_b200 import lordba
 
@@ -431,101 +698,36 @@ def run_workload(args):
     H, F = workloads.HIDDEN, workloads.FFN
     layer = [(di, do) for _, di, do in workloads.LAYER_PROJECTIONS]
     n_seg = args.segments if args.workload == "multi" else 0
-    shapes = {"attn": [(H, H)], "multi": [(H, H)] * max(n_seg, 1), "gate": [(H, F)], "down": [(F, H)], "layer": layer, "decode": layer,
-              "full": layer * workloads.N_LAYERS}[args.workload]
-    gen = torch.Generator(device=dev)
-    gen.manual_seed(1234)
-
-    def rand_signs(rows, cols):
-        return (torch.randint(0, 2, (rows, cols), device=dev, generator=gen, dtype=torch.int8) * 2 - 1)
-
-    esh = (args.ell,) if args.ell > 1 else ()      # (ell, d) scales: a multi-envelope adapter (Eq. 4)
-    io_t, io_code = {"bf16": (torch.bfloat16, lordba.BF16), "f16": (torch.float16, lordba.F16)}[args.dtype]
-    # an adapter exported with half-precision scales: values rounded to float16, declared to the library
-    exported = (lambda s: s.to(torch.float16).to(torch.float32)) if args.scales_f16 else (lambda s: s)
-    base_flags = lordba.PROJ_SCALES_F16 if args.scales_f16 else 0
-    adapters = []
-    for di, do in shapes:
-        adapters.append(dict(
-            pa=lordba.pack_signs(rand_signs(r, di), 0), pb=lordba.pack_signs(rand_signs(do, r), 1),
-            s_in=exported(torch.exp(0.5 * torch.randn(*esh, di, device=dev, generator=gen))),
-            s_r=exported(64.0 * (0.02 * torch.randn(*esh, r, device=dev, generator=gen)).abs()),
-            s_out=exported(torch.exp(0.5 * torch.randn(*esh, do, device=dev, generator=gen)))))
-    set_bytes = sum(Tn * (di + do) * ELEM for di, do in shapes)
-    alg_bytes = sum(workloads.algorithmic_bytes(Tn, di, do, r, ELEM) + 4 * (args.ell - 1) * (di + r + do)
-                    for di, do in shapes)
-    n_sets = int(max(1, min(np.ceil(8 * L2_BYTES / set_bytes), 40e9 // set_bytes)))
-    if set_bytes > 2 * L2_BYTES:
-        n_sets = 1                       # one set already exceeds the L2: every step re-reads it from DRAM
-    sets = []
-    for _ in range(n_sets):
-        sets.append([(torch.randn(Tn, di, device=dev, generator=gen, dtype=torch.float32).to(io_t),
-                      torch.randn(Tn, do, device=dev, generator=gen, dtype=torch.float32).to(io_t))
-                     for di, do in shapes])
-    overlap_ok = n_sets > 1 and not args.no_overlap
-
-    def step(i):
-        flags = base_flags | (lordba.PROJ_OVERLAP if (overlap_ok and i % n_sets != 0) else 0)
-        bufs = sets[i % n_sets]
-        projs = [lordba.make_proj(x, a["pa"], a["pb"], a["s_in"], a["s_r"], a["s_out"], y, r, flags)
-                 for (x, y), a in zip(bufs, adapters)]
-        if n_seg:
-            # multi-adapter batch: n_seg segments of Tn tokens, one adapter each, one call
-            lordba.adapter_forward_segments(projs, [Tn] * n_seg, io_code)
-        elif len(projs) == 1:
-            lordba.adapter_forward_ex(projs[0], Tn, io_code)
-        else:
-            lordba.adapter_forward_batched(projs, Tn, io_code)
-
+    shapes = {"attn": [(H, H)], "multi": [(H, H)] * max(n_seg, 1), "gate": [(H, F)], "down": [(F, H)],
+              "layer": layer, "decode": layer, "full": layer * workloads.N_LAYERS}[args.workload]
+    w = DeviceWorkload(lordba, dev, shapes, r, Tn, ell=args.ell, dtype=args.dtype, scales_f16=args.scales_f16,
+                       segments=n_seg, overlap=not args.no_overlap)
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
-    with torch.cuda.stream(stream):
-        n_graph = max(n_sets, 4)
-        for i in range(n_graph):
-            step(i)
-        stream.synchronize()
-        n0 = lordba.launch_count()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
-            for i in range(n_graph):
-                step(i)
-        launches_per_step = (lordba.launch_count() - n0) / n_graph
-        reps_w, reps = max(1, args.warmup // n_graph), max(1, args.steps // n_graph)
-        sampler = ClockSampler(0)
-        sampler.start()
-        for _ in range(reps_w):
-            graph.replay()
-        stream.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        sampler.recording = True
-        e0.record(stream)
-        for _ in range(reps):
-            graph.replay()
-        e1.record(stream)
-        stream.synchronize()
-        sampler.recording = False
-        sampler.stop()
-    steps = reps * n_graph
-    ms = e0.elapsed_time(e1)
-    if lordba.device_status() != 0:
-        raise RuntimeError("device status word set")
+    sampler = ClockSampler(0)
+    sampler.start()
+    sampler.recording = True
+    res = time_workload(w, stream, args.steps, args.warmup)
+    sampler.recording = False
+    sampler.stop()
     peak, peak_kind = measured_peak()
-    achieved = alg_bytes / (ms * 1e-3 / steps) / 1e9
+    ms_per_step = res["us_per_call"] * 1e-3
     line = {
         "metric": "adapter-branch tokens/s, workload %s (r=%d, ell=%d, T=%d, %d projection(s) per call)"
                   % (args.workload, r, args.ell, Tn, len(shapes)),
-        "value": Tn * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
-        "warmup": reps_w * n_graph, "ms_per_step": ms / steps, "higher_is_better": True,
+        "value": Tn * (n_seg if n_seg else 1) / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
         "config": {"workload": args.workload, "projections": len(shapes), "rank": r, "tokens": Tn,
                    "scales": "float16 values, declared (LORDBA_PROJ_SCALES_F16)" if args.scales_f16 else "float32",
-                   "l2": "%d buffer set(s) of %.0f MB" % (n_sets, set_bytes / 1e6),
-                   "launch": "CUDA graph of %d steps replayed" % n_graph,
-                   "step_dependency": "declared independent" if overlap_ok else "each step waits for the previous one"},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None, "peak_kind": "of " + peak_kind,
-                     "algorithmic_bytes_per_launch": alg_bytes},
-        "e2e": None, "gpu_launches": int(round(launches_per_step * steps)), "clocks": sampler.summary(),
+                   "l2": "%d buffer set(s) of %.0f MB" % (w.n_sets, w.set_bytes / 1e6),
+                   "launch": "CUDA graphs of %d steps replayed; median over %d repeats" % (w.n_graph, res["repeats"]),
+                   "step_dependency": res["step_dependency"], "kernel_variant": res["variant"]},
+        "roofline": {"bound": "hbm", "achieved": res["gbs"], "peak": peak, "unit": "GB/s",
+                     "frac": res["frac"], "traffic": None, "peak_kind": "of " + peak_kind,
+                     "algorithmic_bytes_per_launch": w.alg_bytes},
+        "spread_us": {"p10": res["p10_us"], "median": res["us_per_call"], "p90": res["p90_us"]},
+        "e2e": None, "gpu_launches": int(round(res["launches_per_call"] * args.steps)), "clocks": sampler.summary(),
     }
     print(json.dumps(line))
     return 0
@@ -580,18 +782,21 @@ def run_dense_lora_context(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=8000)
-    ap.add_argument("--warmup", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps per region (default: 2000 for the headline, 20 for the other workloads)")
+    ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default=None, choices=["auto", "fma", "tc", "mma"],
                     help="pin the kernel family (default: the library's own choice)")
     ap.add_argument("--traffic", type=float, default=NCU_DRAM_BYTES_PER_LAUNCH,
                     help="ncu DRAM bytes per launch to report in roofline.traffic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true",
+                    help="headline only: skip the `workloads` key (configs 2 to 4 and the widened rows)")
     ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full", "multi", "lora-dense"],
-                    help="attn = the headline configuration (default); the others are supplementary: one "
-                         "MLP projection, a layer's seven projections in one batched call (prefill, or "
-                         "decode with --tokens 1..64), or all 224 projections in one call")
+                    help="attn = the headline configuration (default); the others time one supplementary "
+                         "workload alone: one MLP projection, a layer's seven projections in one batched call "
+                         "(prefill, or decode with --tokens 1..64), or all 224 projections in one call")
     ap.add_argument("--segments", type=int, default=8,
                     help="workload multi: segments (adapters) per call, --tokens rows each, attention shape")
     ap.add_argument("--rank", type=int, default=R)
@@ -604,13 +809,21 @@ def main():
     ap.add_argument("--no-overlap", action="store_true",
                     help="every step waits for the previous one to finish (no LORDBA_PROJ_OVERLAP)")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3)
+    headline = not (args.workload != "attn" or args.ell != 1 or args.rank != R or args.tokens != T or
+                    args.dtype != "bf16" or args.scales_f16)
+    if args.impl == "reference" or headline or args.workload == "lora-dense":
+        dflt_steps, dflt_warm = 2000, 100
+    elif args.workload == "full":
+        dflt_steps, dflt_warm = 4, 3
+    else:
+        dflt_steps, dflt_warm = 20, 5
+    args.steps = max(1, args.steps if args.steps is not None else dflt_steps)
+    args.warmup = max(3, args.warmup if args.warmup is not None else dflt_warm)
     if args.impl == "reference":
         return run_reference(args)
     if args.workload == "lora-dense":
         return run_dense_lora_context(args)
-    if (args.workload != "attn" or args.ell != 1 or args.rank != R or args.tokens != T or args.dtype != "bf16" or
-            args.scales_f16):
+    if not headline:
         return run_workload(args)
     return run_gpu(args)
 

@@ -30,7 +30,9 @@
  *   - Return value: a lordba_status.  Argument errors are detected on the host
  *     and nothing is launched.  There is no CPU fallback: without a usable CUDA
  *     device the calls return LORDBA_ECUDA.
- *   - Supported rank: 1 <= r <= 64.
+ *   - Supported rank: 1 <= r <= 64.  A call takes at most LORDBA_MAX_PROJS projections
+ *     (LORDBA_EUNSUPPORTED beyond that).
+ *   - No entry point allocates host or device memory.
  *
  * Bit-packed carriers (the paper says only "bit-packed"; this layout is the
  * library's own).  Bit 1 <=> +1, bit 0 <=> -1, 32-bit little-endian words,
@@ -52,6 +54,8 @@
 #ifdef __cplusplus
 extern "C" {
 #endif
+
+#define LORDBA_MAX_PROJS 4096
 
 typedef enum {
     LORDBA_F32 = 0,   /* x and y are float32                                   */
@@ -126,8 +130,8 @@ typedef struct lordba_proj {
 
 /*
  * lordba_proj.flags: the caller states that every entry of s_in is exactly representable as an
- * IEEE half, which is the case for an adapter exported with fp16 scales (the method trains the
- * scales in fp32 and casts them to fp16 at export) and widened by lordba_scales_from_f16.  With
+ * IEEE half, which is the case for an adapter exported with fp16 scales (Section 3.2: the scales
+ * are trained in float32 and leave training as halves) and widened by lordba_scales_from_f16.  With
  * LORDBA_F16 activations the streaming kernel then forms x * s_in in one tensor-core pass
  * instead of two; with a false statement the low bits of s_in beyond a half are ignored, nothing
  * else.  Other kernels and dtypes accept the flag and ignore it.
@@ -147,8 +151,8 @@ int lordba_scales_from_f16(const uint16_t *src, float *dst, int64_t n, void *str
 int64_t lordba_packed_words(int64_t rows, int64_t cols, int role);
 
 /*
- * Bit-pack a sign matrix ("bit-packed {B1,B2} stored once per adapter",
- * Section 3.3).  signs: [device] int8, rows x cols row-major; an entry < 0 packs
+ * Bit-pack a sign matrix: the two sign carriers are kept as one bit per entry and packed
+ * once per adapter (Section 3.3).  signs: [device] int8, rows x cols row-major; an entry < 0 packs
  * as -1, anything else (0 included: sign(0) = +1) as +1.  role 0: rows = r,
  * cols = d_in.  role 1: rows = d_out, cols = r.  packed: [device], at least
  * lordba_packed_words() words, fully overwritten (pad bits 0).
@@ -200,13 +204,13 @@ int lordba_adapter_forward_batched(const lordba_proj *projs, int n_proj, int64_t
                                    void *stream);
 
 /*
- * Multi-adapter batch (Section 3.1, condition A4: many task adapters served over one frozen
- * base): segment i is tokens[i] consecutive token rows that go through their own adapter.
+ * Multi-adapter batch (Section 2, adapter-mode deployment, condition A4: many task adapters
+ * served over one frozen base): segment i is tokens[i] consecutive token rows that go through their own adapter.
  * segs[i].x / .y point at the segment's first row (usually into one shared x / y matrix),
  * the other fields name the segment's adapter; several segments may share an adapter.
  * segs, tokens: [host] arrays of n_seg entries, read before the call returns.  Segments are
  * treated as simultaneous (same disjointness rules as the batched call); empty segments are
- * skipped.  One launch per 24 segments of equal padded rank.
+ * skipped.  One launch per 24 segments of equal padded rank (per 96 on the tcgen05 kernel).
  */
 int lordba_adapter_forward_segments(const lordba_proj *segs, const int64_t *tokens, int n_seg, int dtype,
                                     void *stream);
@@ -242,7 +246,10 @@ int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
  *     workspace.  If lordba_host_workspace_bytes(T, d_in, d_out, dtype) exceeds
  *     LORDBA_STATIC_SCRATCH_BYTES the call returns LORDBA_ETOOLARGE and does nothing.
  *   - The first call on a device looks up the buffer's device address (with that device current)
- *     and remembers it; make that first call outside any stream capture.
+ *     and remembers it.  If nothing of the library has run on that device yet, this lookup is
+ *     also the moment at which the CUDA runtime loads the library's device code there, which
+ *     reserves the buffer and may synchronise the device: make that first call at start-up,
+ *     outside any stream capture and outside latency-critical code.
  *   - All calls on a device share the one buffer.  It still holds the previous call's x and y;
  *     nothing in it has to start at zero, because every byte that is read was copied in by the
  *     same call first.  Two calls whose work overlaps on the GPU (different streams, no
@@ -253,6 +260,47 @@ int lordba_adapter_forward_host_static(const void *x_host, const uint32_t *packe
                                        const uint32_t *packed_B, const float *s_in, const float *s_r,
                                        const float *s_out, void *y_host, int64_t T, int64_t d_in,
                                        int64_t d_out, int r, int dtype, void *stream);
+
+/*
+ * Which kernel family a call would run each projection on, without launching anything: the
+ * answer of lordba_adapter_forward_batched (tokens == NULL: every projection has T rows) or of
+ * lordba_adapter_forward_segments (tokens[i] rows each) for the same arguments and the current
+ * lordba_set_variant setting.  variants: [host] n_proj entries, each set to LORDBA_VARIANT_FMA,
+ * _TC or _MMA (0 for a projection without rows).  The CUDA-core kernel (FMA) takes every shape but
+ * runs an order of magnitude below the tensor-core kernels, which want bf16 / float16 activations,
+ * d_in and d_out multiples of 64, row pitches multiples of 8 elements and 16-byte aligned x, y,
+ * scales and carriers: a caller can see that fallback coming here.  Returns the status the call
+ * itself would return for bad arguments.
+ */
+int lordba_query_variant(const lordba_proj *projs, int n_proj, int64_t T, const int64_t *tokens, int dtype,
+                         int *variants);
+
+/*
+ * Prepared calls.  Every forward call builds its launch parameters on the host first (tensor maps
+ * for the copy engine, six per projection in the streaming kernel).  A caller that repeats a call
+ * with the same pointers and sizes (a layer's adapters over fixed activation buffers, step after
+ * step) can have that done once:
+ *
+ *   lordba_plan_bytes   the storage a plan for these arguments needs (0 on bad arguments);
+ *   lordba_plan_init    validates the arguments exactly like lordba_adapter_forward_batched
+ *                       (tokens == NULL) or lordba_adapter_forward_segments (tokens given), chooses
+ *                       the kernels and writes the prepared launches into plan: [host], 64-byte
+ *                       aligned, caller-owned, plan_bytes long (LORDBA_ETOOLARGE if too short).
+ *                       Nothing is launched;
+ *   lordba_adapter_forward_planned   enqueues the prepared launches on stream: the same kernels
+ *                       with the same arguments as the unprepared call.
+ *
+ * A plan holds device addresses: it belongs to the device that was current at lordba_plan_init
+ * (LORDBA_EINVAL on another one), stays valid while the buffers it names are, and may be replayed
+ * any number of times, from any stream; it holds no resources and needs no release.
+ * LORDBA_PROJ_OVERLAP in the projections' flags is part of the plan.
+ */
+size_t lordba_plan_bytes(const lordba_proj *projs, int n_proj, int64_t T, const int64_t *tokens, int dtype);
+int lordba_plan_init(void *plan, size_t plan_bytes, const lordba_proj *projs, int n_proj, int64_t T,
+                     const int64_t *tokens, int dtype);
+int lordba_adapter_forward_planned(const void *plan, void *stream);
+/* Kernel launches a plan holds (-1 if plan is not a plan). */
+int lordba_plan_launches(const void *plan);
 
 /* Storage of one adapter in bits, Eq. 5: r(d_in+d_out) + 16 ell (d_in+r+d_out). */
 int64_t lordba_adapter_bits(int64_t d_in, int64_t d_out, int r, int ell);

@@ -17,6 +17,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 BUILD = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "liblordba.so")
+TESTHOOKS_LIB = os.path.join(PKG, "liblordba_testhooks.so")
 SOURCES = ("api.cu", "pack.cu", "forward_fma.cu", "forward_tc.cu", "forward_mma.cu")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Wno-deprecated-gpu-targets",
@@ -36,16 +37,23 @@ def _newest_header() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(BUILD, exist_ok=True)
+def build_library(force: bool = False, verbose: bool = False, test_hooks: bool = False) -> str:
+    """Build the library.  test_hooks=True builds a second library, liblordba_testhooks.so, from
+    the same sources with -DLORDBA_TEST_HOOKS (bounded device-side waits give up after about a
+    millisecond, and lordba_test_skip_item makes one copy request go missing): only the test of
+    the timeout path loads it; the product library never has the hooks."""
+    build_dir = BUILD + ("_testhooks" if test_hooks else "")
+    lib_path = TESTHOOKS_LIB if test_hooks else LIB
+    extra = ["-DLORDBA_TEST_HOOKS"] if test_hooks else []
+    os.makedirs(build_dir, exist_ok=True)
     nvcc = _nvcc()
     hdr = _newest_header()
     jobs = []
     for src in SOURCES:
         s = os.path.join(CSRC, src)
-        o = os.path.join(BUILD, src + ".o")
+        o = os.path.join(build_dir, src + ".o")
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 
     def run(cmd):
@@ -57,13 +65,14 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=4) as ex:
         list(ex.map(run, jobs))
-    objs = [os.path.join(BUILD, s + ".o") for s in SOURCES]
-    if jobs or not os.path.exists(LIB):
-        tmp = LIB + ".tmp.%d" % os.getpid()
+    objs = [os.path.join(build_dir, s + ".o") for s in SOURCES]
+    if jobs or not os.path.exists(lib_path):
+        tmp = lib_path + ".tmp.%d" % os.getpid()
         run([nvcc, "-shared", "-o", tmp] + objs + ["-Xlinker", "--exclude-libs=ALL"])
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib_path)
+    return lib_path
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv,
+                        test_hooks="--test-hooks" in sys.argv))

@@ -1,10 +1,10 @@
 // C ABI of liblordba: argument validation on the host, kernel-family choice,
 // launches.  See include/lordba.h for the contract of every entry point.
+#include <algorithm>
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
-#include <vector>
 
 #include "lordba_internal.h"
 
@@ -16,6 +16,9 @@ std::atomic<int> g_variant{LORDBA_VARIANT_AUTO};
 __device__ int g_device_status;   // written by bounded waits that gave up
 std::mutex g_status_mutex;
 int *g_status_ptr[64] = {nullptr};
+#ifdef LORDBA_TEST_HOOKS
+std::atomic<int> g_test_skip_item{-1};
+#endif
 }  // namespace
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
@@ -31,6 +34,72 @@ int *device_status_word()
         g_status_ptr[dev] = static_cast<int *>(p);
     }
     return g_status_ptr[dev];
+}
+
+int test_skip_item()
+{
+#ifdef LORDBA_TEST_HOOKS
+    return g_test_skip_item.load(std::memory_order_relaxed);
+#else
+    return -1;
+#endif
+}
+
+int FamilySelector::family(const lordba_proj &p, int64_t rows) const
+{
+    if (rows <= 0) return 0;
+    if (variant == LORDBA_VARIANT_FMA || dtype == LORDBA_F32) return LORDBA_VARIANT_FMA;
+    if (use_tc) return tc_supported(p, rows, dtype) ? LORDBA_VARIANT_TC : LORDBA_VARIANT_FMA;
+    return mma_supported(p, rows, dtype) ? LORDBA_VARIANT_MMA : LORDBA_VARIANT_FMA;
+}
+
+int launch_record(const LaunchRec &rec, const void *arg0, const void *arg1, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(rec.grid[0], rec.grid[1], rec.grid[2]);
+    cfg.blockDim = dim3(rec.block, 1, 1);
+    cfg.dynamicSmemBytes = rec.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    unsigned na = 0;
+    if (rec.cluster > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = rec.cluster; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (rec.pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
+    void *args[2] = {const_cast<void *>(arg0), const_cast<void *>(arg1)};
+    if (cudaLaunchKernelExC(&cfg, rec.func, args) != cudaSuccess) {
+        cudaGetLastError();
+        return LORDBA_ECUDA;
+    }
+    count_launch();
+    return LORDBA_OK;
+}
+
+int LaunchSink::emit(LaunchRec rec, const void *arg0, const void *arg1)
+{
+    if (immediate) return launch_record(rec, arg0, arg1, stream);
+    const size_t a0 = (sizeof(LaunchRec) + 63) / 64 * 64;
+    const size_t a1 = a0 + ((size_t)rec.arg_bytes[0] + 63) / 64 * 64;
+    const size_t total = a1 + (rec.n_args > 1 ? ((size_t)rec.arg_bytes[1] + 63) / 64 * 64 : 0);
+    rec.total_bytes = (uint32_t)total;
+    if (buf) {
+        if (used + total > cap) return LORDBA_ETOOLARGE;
+        std::memcpy(buf + used, &rec, sizeof(rec));
+        std::memcpy(buf + used + a0, arg0, rec.arg_bytes[0]);
+        if (rec.n_args > 1) std::memcpy(buf + used + a1, arg1, rec.arg_bytes[1]);
+    }
+    used += total;
+    ++count;
+    return LORDBA_OK;
 }
 
 namespace {
@@ -67,53 +136,107 @@ int validate_proj(const lordba_proj &p, int64_t T, int dtype)
     return LORDBA_OK;
 }
 
+// Left to itself the library takes the tcgen05 kernel where it was measured ahead of the
+// streaming one: ranks above 32 from 32 tiles of 128 tokens (one projection at T = 4096, a layer
+// at T = 2048), ranks 24 and 32 from eight waves of such tiles (below that the streaming kernel
+// is ahead).
+FamilySelector make_selector(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, int dtype)
+{
+    FamilySelector sel;
+    sel.dtype = dtype;
+    sel.variant = g_variant.load(std::memory_order_relaxed);
+    sel.use_tc = (sel.variant == LORDBA_VARIANT_TC);
+    if (sel.variant == LORDBA_VARIANT_AUTO && dtype != LORDBA_F32) {
+        int64_t tiles = 0;
+        bool all_ok = false, all_high = true;
+        for (int i = 0; i < n; ++i) {
+            const int64_t rows = rows_of(tokens, T, i);
+            if (rows == 0) continue;
+            if (tiles == 0) all_ok = true;
+            all_ok = all_ok && projs[i].r > 16 && tc_supported(projs[i], rows, dtype);
+            all_high = all_high && projs[i].r > 32;
+            tiles += (rows + 127) / 128;
+        }
+        sel.use_tc = all_ok && tiles >= (all_high ? 32 : 8 * 148);
+    }
+    return sel;
+}
+
 // batch_checked: the caller has verified that the projections of this call are independent of
 // one another (disjoint y buffers, no x inside a y), so its launches may overlap each other.
 // tokens: per-projection token rows, or nullptr when every projection has T rows.
-int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, int dtype, cudaStream_t stream,
+int dispatch(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, int dtype, LaunchSink &sink,
              bool batch_checked)
 {
-    const int variant = g_variant.load(std::memory_order_relaxed);
-    std::vector<int64_t> rows(n, T);
-    if (tokens) rows.assign(tokens, tokens + n);
-    if (variant == LORDBA_VARIANT_FMA || dtype == LORDBA_F32) {
-        if (variant == LORDBA_VARIANT_TC || variant == LORDBA_VARIANT_MMA) return LORDBA_EUNSUPPORTED;
-        return launch_forward_fma(projs, rows.data(), n, dtype, stream);
-    }
-    // Split the list: what the chosen tensor-core kernel can take, and the rest.  Left to itself
-    // the library takes the tcgen05 kernel where it was measured ahead of the streaming one: ranks
-    // above 32 from 32 tiles of 128 tokens (one projection at T = 4096, a layer at T = 2048), ranks
-    // 24 and 32 from eight waves of such tiles (below that the streaming kernel is ahead).  (That kernel wants one token count for all
-    // projections.)
-    bool use_tc = (variant == LORDBA_VARIANT_TC);
-    if (use_tc && tokens) return LORDBA_EUNSUPPORTED;
-    if (variant == LORDBA_VARIANT_AUTO && !tokens) {
-        int64_t tiles = 0;
-        bool all_ok = n > 0, all_high = true;
+    const FamilySelector sel = make_selector(projs, n, T, tokens, dtype);
+    if (sel.variant != LORDBA_VARIANT_AUTO) {
+        // a pinned family must be able to take every projection of the call
         for (int i = 0; i < n; ++i) {
-            all_ok = all_ok && projs[i].r > 16 && tc_supported(projs[i], T, dtype);
-            all_high = all_high && projs[i].r > 32;
-            tiles += T / 128;
+            const int64_t rows = rows_of(tokens, T, i);
+            if (rows > 0 && sel.family(projs[i], rows) != sel.variant) return LORDBA_EUNSUPPORTED;
         }
-        use_tc = all_ok && tiles >= (all_high ? 32 : 8 * 148);
     }
-    std::vector<lordba_proj> fast, fma;
-    std::vector<int64_t> fast_rows, fma_rows;
+    int launches = 0;
+    int rc = launch_forward_tc(projs, tokens, T, n, sel, sink, batch_checked, &launches);
+    if (rc != LORDBA_OK) return rc;
+    rc = launch_forward_mma(projs, tokens, T, n, sel, sink, batch_checked, &launches);
+    if (rc != LORDBA_OK) return rc;
+    return launch_forward_fma(projs, tokens, T, n, sel, sink);
+}
+
+int dispatch_now(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, int dtype, cudaStream_t stream,
+                 bool batch_checked)
+{
+    LaunchSink sink;
+    sink.stream = stream;
+    return dispatch(projs, n, T, tokens, dtype, sink, batch_checked);
+}
+
+size_t bytes_of(const lordba_proj &p, int64_t rows, int64_t ld, int64_t width, size_t e)
+{
+    (void)p;
+    return ((size_t)(rows - 1) * (size_t)ld + (size_t)width) * e;
+}
+
+// The projections of a call are simultaneous: outputs pairwise disjoint, no input inside an
+// output.  Sorted intervals: n log n.
+int check_independent(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, size_t e)
+{
+    struct Iv { uintptr_t lo, hi; };
+    Iv ys[kMaxCallProjs];
+    int m = 0;
     for (int i = 0; i < n; ++i) {
-        if (rows[i] == 0) continue;
-        const bool ok = use_tc ? tc_supported(projs[i], rows[i], dtype) : mma_supported(projs[i], rows[i], dtype);
-        (ok ? fast : fma).push_back(projs[i]);
-        (ok ? fast_rows : fma_rows).push_back(rows[i]);
+        const int64_t rows = rows_of(tokens, T, i);
+        if (rows <= 0) continue;
+        const uintptr_t lo = reinterpret_cast<uintptr_t>(projs[i].y);
+        ys[m++] = Iv{lo, lo + bytes_of(projs[i], rows, projs[i].ldy, projs[i].d_out, e)};
     }
-    if (variant != LORDBA_VARIANT_AUTO && !fma.empty()) return LORDBA_EUNSUPPORTED;
-    if (!fast.empty()) {
-        const int rc = use_tc ? launch_forward_tc(fast.data(), (int)fast.size(), T, dtype, stream, batch_checked)
-                              : launch_forward_mma(fast.data(), fast_rows.data(), (int)fast.size(), dtype, stream,
-                                                   batch_checked);
+    std::sort(ys, ys + m, [](const Iv &a, const Iv &b) { return a.lo < b.lo; });
+    for (int i = 0; i + 1 < m; ++i)
+        if (ys[i].hi > ys[i + 1].lo) return LORDBA_EINVAL;
+    for (int i = 0; i < n; ++i) {
+        const int64_t rows = rows_of(tokens, T, i);
+        if (rows <= 0) continue;
+        const uintptr_t lo = reinterpret_cast<uintptr_t>(projs[i].x);
+        const uintptr_t hi = lo + bytes_of(projs[i], rows, projs[i].ldx, projs[i].d_in, e);
+        // first output that ends after the input starts (the outputs are disjoint: their ends are sorted too)
+        const Iv *it = std::upper_bound(ys, ys + m, lo, [](uintptr_t v, const Iv &a) { return v < a.hi; });
+        if (it != ys + m && it->lo < hi) return LORDBA_EINVAL;
+    }
+    return LORDBA_OK;
+}
+
+// Validation shared by the batched, the segmented and the prepared calls.
+int validate_call(const lordba_proj *projs, int n, int64_t T, const int64_t *tokens, int dtype)
+{
+    if (n < 0 || (n > 0 && !projs)) return LORDBA_EINVAL;
+    if (n > kMaxCallProjs) return LORDBA_EUNSUPPORTED;
+    if (!tokens && T < 0) return LORDBA_EINVAL;
+    for (int i = 0; i < n; ++i) {
+        const int rc = validate_proj(projs[i], rows_of(tokens, T, i), dtype);
         if (rc != LORDBA_OK) return rc;
     }
-    if (!fma.empty()) return launch_forward_fma(fma.data(), fma_rows.data(), (int)fma.size(), dtype, stream);
-    return LORDBA_OK;
+    return check_independent(projs, n, T, tokens, (dtype == LORDBA_F32) ? 4 : 2);
 }
 
 lordba_proj dense_proj(const void *x, const uint32_t *pa, const uint32_t *pb, const float *s_in,
@@ -178,7 +301,7 @@ int lordba_adapter_forward_ex(const lordba_proj *p, int64_t T, int dtype, void *
     const int rc = validate_proj(*p, T, dtype);
     if (rc != LORDBA_OK) return rc;
     if (T == 0) return LORDBA_OK;
-    return dispatch(p, 1, T, nullptr, dtype, static_cast<cudaStream_t>(stream), false);
+    return dispatch_now(p, 1, T, nullptr, dtype, static_cast<cudaStream_t>(stream), false);
 }
 
 int lordba_adapter_forward(const void *x, const uint32_t *packed_A, const uint32_t *packed_B,
@@ -211,51 +334,138 @@ int lordba_adapter_forward_f32(const float *x, const uint32_t *packed_A, const u
 int lordba_adapter_forward_batched(const lordba_proj *projs, int n_proj, int64_t T, int dtype,
                                    void *stream)
 {
-    if (n_proj < 0 || (n_proj > 0 && !projs)) return LORDBA_EINVAL;
-    const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
-    for (int i = 0; i < n_proj; ++i) {
-        const int rc = validate_proj(projs[i], T, dtype);
-        if (rc != LORDBA_OK) return rc;
-    }
-    if (T > 0) {
-        // outputs must be pairwise disjoint and no input may lie in an output (n_proj is small:
-        // 7 per layer, 224 per model)
-        for (int i = 0; i < n_proj; ++i)
-            for (int j = 0; j < n_proj; ++j) {
-                if (i == j) continue;
-                const size_t ni = ((size_t)(T - 1) * projs[i].ldy + projs[i].d_out) * e;
-                const size_t nj = ((size_t)(T - 1) * projs[j].ldy + projs[j].d_out) * e;
-                const size_t nx = ((size_t)(T - 1) * projs[i].ldx + projs[i].d_in) * e;
-                if (j > i && overlaps(projs[i].y, ni, projs[j].y, nj)) return LORDBA_EINVAL;
-                if (overlaps(projs[i].x, nx, projs[j].y, nj)) return LORDBA_EINVAL;
-            }
-    }
+    const int rc = validate_call(projs, n_proj, T, nullptr, dtype);
+    if (rc != LORDBA_OK) return rc;
     if (T == 0 || n_proj == 0) return LORDBA_OK;
-    return dispatch(projs, n_proj, T, nullptr, dtype, static_cast<cudaStream_t>(stream), true);
+    return dispatch_now(projs, n_proj, T, nullptr, dtype, static_cast<cudaStream_t>(stream), true);
 }
 
 int lordba_adapter_forward_segments(const lordba_proj *segs, const int64_t *tokens, int n_seg, int dtype,
                                     void *stream)
 {
-    if (n_seg < 0 || (n_seg > 0 && (!segs || !tokens))) return LORDBA_EINVAL;
-    const size_t e = (dtype == LORDBA_F32) ? 4 : 2;
-    for (int i = 0; i < n_seg; ++i) {
-        const int rc = validate_proj(segs[i], tokens[i], dtype);
-        if (rc != LORDBA_OK) return rc;
-    }
-    // segments are simultaneous: outputs pairwise disjoint, no input inside an output
-    for (int i = 0; i < n_seg; ++i)
-        for (int j = 0; j < n_seg; ++j) {
-            if (i == j || tokens[i] == 0 || tokens[j] == 0) continue;
-            const size_t ni = ((size_t)(tokens[i] - 1) * segs[i].ldy + segs[i].d_out) * e;
-            const size_t nj = ((size_t)(tokens[j] - 1) * segs[j].ldy + segs[j].d_out) * e;
-            const size_t nx = ((size_t)(tokens[i] - 1) * segs[i].ldx + segs[i].d_in) * e;
-            if (j > i && overlaps(segs[i].y, ni, segs[j].y, nj)) return LORDBA_EINVAL;
-            if (overlaps(segs[i].x, nx, segs[j].y, nj)) return LORDBA_EINVAL;
-        }
+    if (n_seg > 0 && !tokens) return LORDBA_EINVAL;
+    const int rc = validate_call(segs, n_seg, 0, tokens, dtype);
+    if (rc != LORDBA_OK) return rc;
     if (n_seg == 0) return LORDBA_OK;
-    return dispatch(segs, n_seg, 0, tokens, dtype, static_cast<cudaStream_t>(stream), true);
+    return dispatch_now(segs, n_seg, 0, tokens, dtype, static_cast<cudaStream_t>(stream), true);
 }
+
+int lordba_query_variant(const lordba_proj *projs, int n_proj, int64_t T, const int64_t *tokens, int dtype,
+                         int *variants)
+{
+    if (!variants && n_proj > 0) return LORDBA_EINVAL;
+    const int rc = validate_call(projs, n_proj, T, tokens, dtype);
+    if (rc != LORDBA_OK) return rc;
+    const FamilySelector sel = make_selector(projs, n_proj, T, tokens, dtype);
+    for (int i = 0; i < n_proj; ++i) {
+        const int64_t rows = rows_of(tokens, T, i);
+        variants[i] = sel.family(projs[i], rows);
+        if (rows > 0 && sel.variant != LORDBA_VARIANT_AUTO && variants[i] != sel.variant) return LORDBA_EUNSUPPORTED;
+    }
+    return LORDBA_OK;
+}
+
+// ---- prepared calls -----------------------------------------------------------------------
+
+namespace {
+struct PlanHeader {
+    uint32_t magic, version;
+    int32_t device;
+    int32_t n_launches;
+    uint64_t bytes;        // header + records
+    uint64_t pad_[5];
+};
+static_assert(sizeof(PlanHeader) == 64, "plan header is one 64-byte block");
+constexpr uint32_t kPlanMagic = 0x4c44424du, kPlanVersion = 2;
+
+int build_plan(void *storage, size_t cap, const lordba_proj *projs, int n_proj, int64_t T, const int64_t *tokens,
+               int dtype, size_t *bytes_out)
+{
+    const int rc = validate_call(projs, n_proj, T, tokens, dtype);
+    if (rc != LORDBA_OK) return rc;
+    LaunchSink sink;
+    sink.immediate = false;
+    if (storage) {
+        if (!aligned(storage, 64)) return LORDBA_EALIGN;
+        if (cap < sizeof(PlanHeader)) return LORDBA_ETOOLARGE;
+        sink.buf = static_cast<uint8_t *>(storage) + sizeof(PlanHeader);
+        sink.cap = cap - sizeof(PlanHeader);
+    }
+    bool any = false;
+    for (int i = 0; i < n_proj; ++i) any = any || rows_of(tokens, T, i) > 0;
+    if (any) {
+        const int rc2 = dispatch(projs, n_proj, T, tokens, dtype, sink, true);
+        if (rc2 != LORDBA_OK) return rc2;
+    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LORDBA_ECUDA;
+    if (storage) {
+        PlanHeader h;
+        std::memset(&h, 0, sizeof(h));
+        h.magic = kPlanMagic; h.version = kPlanVersion; h.device = dev; h.n_launches = sink.count;
+        h.bytes = sizeof(PlanHeader) + sink.used;
+        std::memcpy(storage, &h, sizeof(h));
+    }
+    if (bytes_out) *bytes_out = sizeof(PlanHeader) + sink.used;
+    return LORDBA_OK;
+}
+}  // namespace
+
+size_t lordba_plan_bytes(const lordba_proj *projs, int n_proj, int64_t T, const int64_t *tokens, int dtype)
+{
+    size_t bytes = 0;
+    if (build_plan(nullptr, 0, projs, n_proj, T, tokens, dtype, &bytes) != LORDBA_OK) return 0;
+    return bytes;
+}
+
+int lordba_plan_init(void *plan, size_t plan_bytes, const lordba_proj *projs, int n_proj, int64_t T,
+                     const int64_t *tokens, int dtype)
+{
+    if (!plan) return LORDBA_EINVAL;
+    return build_plan(plan, plan_bytes, projs, n_proj, T, tokens, dtype, nullptr);
+}
+
+int lordba_plan_launches(const void *plan)
+{
+    if (!plan || !aligned(plan, 64)) return -1;
+    const PlanHeader *h = static_cast<const PlanHeader *>(plan);
+    if (h->magic != kPlanMagic || h->version != kPlanVersion) return -1;
+    return h->n_launches;
+}
+
+int lordba_adapter_forward_planned(const void *plan, void *stream)
+{
+    if (!plan) return LORDBA_EINVAL;
+    if (!aligned(plan, 64)) return LORDBA_EALIGN;
+    const PlanHeader *h = static_cast<const PlanHeader *>(plan);
+    if (h->magic != kPlanMagic || h->version != kPlanVersion) return LORDBA_EINVAL;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LORDBA_ECUDA;
+    if (dev != h->device) return LORDBA_EINVAL;      // a plan holds addresses of the device it was made on
+    const uint8_t *p = static_cast<const uint8_t *>(plan) + sizeof(PlanHeader);
+    const uint8_t *end = static_cast<const uint8_t *>(plan) + h->bytes;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < h->n_launches; ++i) {
+        const LaunchRec *rec = reinterpret_cast<const LaunchRec *>(p);
+        if (p + sizeof(LaunchRec) > end || p + rec->total_bytes > end) return LORDBA_EINVAL;
+        const size_t a0 = (sizeof(LaunchRec) + 63) / 64 * 64;
+        const size_t a1 = a0 + ((size_t)rec->arg_bytes[0] + 63) / 64 * 64;
+        const int rc = launch_record(*rec, p + a0, rec->n_args > 1 ? p + a1 : nullptr, s);
+        if (rc != LORDBA_OK) return rc;
+        p += rec->total_bytes;
+    }
+    return LORDBA_OK;
+}
+
+#ifdef LORDBA_TEST_HOOKS
+// Test-hooks build only: the producers of the tensor-core kernels leave out the copy request of
+// pipeline item `item` (counted from 0 within every CTA's first tile); -1 switches the hook off.
+int lordba_test_skip_item(int item)
+{
+    g_test_skip_item.store(item, std::memory_order_relaxed);
+    return LORDBA_OK;
+}
+#endif
 
 size_t lordba_host_workspace_bytes(int64_t T, int64_t d_in, int64_t d_out, int dtype)
 {
@@ -288,7 +498,7 @@ int lordba_adapter_forward_host(const void *x_host, const uint32_t *packed_A,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(xd, x_host, bx, cudaMemcpyHostToDevice, s) != cudaSuccess) return LORDBA_ECUDA;
     if (cudaMemcpyAsync(yd, y_host, by, cudaMemcpyHostToDevice, s) != cudaSuccess) return LORDBA_ECUDA;
-    const int rc2 = dispatch(&p, 1, T, nullptr, dtype, s, false);
+    const int rc2 = dispatch_now(&p, 1, T, nullptr, dtype, s, false);
     if (rc2 != LORDBA_OK) return rc2;
     if (cudaMemcpyAsync(y_host, yd, by, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LORDBA_ECUDA;
     return LORDBA_OK;

@@ -14,6 +14,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <cstring>
+
 #include "lordba_internal.h"
 
 namespace lordba {
@@ -321,42 +323,53 @@ fma_forward_kernel(const __grid_constant__ FmaBatch batch)
 }
 
 template <typename T>
-cudaError_t launch_rank(const FmaBatch &b, int n, int rp, cudaStream_t stream)
+const void *kernel_for(int rp)
+{
+    switch (rp) {
+        case 8:  return reinterpret_cast<const void *>(&fma_forward_kernel<T, 8>);
+        case 16: return reinterpret_cast<const void *>(&fma_forward_kernel<T, 16>);
+        case 32: return reinterpret_cast<const void *>(&fma_forward_kernel<T, 32>);
+        default: return reinterpret_cast<const void *>(&fma_forward_kernel<T, 64>);
+    }
+}
+
+int emit_rank(const FmaBatch &b, int n, int rp, int dtype, LaunchSink &sink)
 {
     const int tt = kAccPerThread / rp;
     int64_t T_tokens = 0;                          // the longest projection sets grid.x
     for (int i = 0; i < n; ++i) if (b.tokens[i] > T_tokens) T_tokens = b.tokens[i];
     const int64_t tiles = (T_tokens + tt - 1) / tt;
-    dim3 grid((unsigned)tiles, (unsigned)n, 1);
-    switch (rp) {
-        case 8:  fma_forward_kernel<T, 8><<<grid, kThreads, 0, stream>>>(b); break;
-        case 16: fma_forward_kernel<T, 16><<<grid, kThreads, 0, stream>>>(b); break;
-        case 32: fma_forward_kernel<T, 32><<<grid, kThreads, 0, stream>>>(b); break;
-        default: fma_forward_kernel<T, 64><<<grid, kThreads, 0, stream>>>(b); break;
-    }
-    count_launch();
-    return cudaGetLastError();
+    LaunchRec rec;
+    std::memset(&rec, 0, sizeof(rec));
+    rec.func = (dtype == LORDBA_F32)    ? kernel_for<float>(rp)
+               : (dtype == LORDBA_F16) ? kernel_for<__half>(rp)
+                                       : kernel_for<__nv_bfloat16>(rp);
+    rec.grid[0] = (unsigned)tiles; rec.grid[1] = (unsigned)n; rec.grid[2] = 1;
+    rec.block = kThreads;
+    rec.n_args = 1;
+    rec.arg_bytes[0] = sizeof(FmaBatch);
+    return sink.emit(rec, &b, nullptr);
 }
 
 int padded_rank(int r) { return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64; }
 
 }  // namespace
 
-int launch_forward_fma(const lordba_proj *projs, const int64_t *tokens, int n, int dtype, cudaStream_t stream)
+int launch_forward_fma(const lordba_proj *projs, const int64_t *tokens, int64_t T, int n, const FamilySelector &sel,
+                       LaunchSink &sink)
 {
-    if (n == 0) return LORDBA_OK;
     // Group projections of equal padded rank into launches of at most kMaxBatch.
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
         FmaBatch b;
         int m = 0;
         for (int i = 0; i <= n; ++i) {
-            const bool take = (i < n) && tokens[i] > 0 && padded_rank(projs[i].r) == rp;
-            if (take) { b.tokens[m] = tokens[i]; b.p[m++] = projs[i]; }
+            const int64_t rows = (i < n) ? rows_of(tokens, T, i) : 0;
+            const bool take = (i < n) && rows > 0 && padded_rank(projs[i].r) == rp &&
+                              sel.family(projs[i], rows) == LORDBA_VARIANT_FMA;
+            if (take) { b.tokens[m] = rows; b.p[m++] = projs[i]; }
             if (m == kMaxBatch || (i == n && m > 0)) {
-                const cudaError_t e = (dtype == LORDBA_F32)    ? launch_rank<float>(b, m, rp, stream)
-                                      : (dtype == LORDBA_F16) ? launch_rank<__half>(b, m, rp, stream)
-                                                              : launch_rank<__nv_bfloat16>(b, m, rp, stream);
-                if (e != cudaSuccess) return LORDBA_ECUDA;
+                const int rc = emit_rank(b, m, rp, sel.dtype, sink);
+                if (rc != LORDBA_OK) return rc;
                 m = 0;
             }
         }

@@ -57,7 +57,6 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <type_traits>
@@ -78,7 +77,6 @@ constexpr int kMaxBatch = 24;        // projections per launch (six tensor maps 
 constexpr int kMaxSlots = 8;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr int kSmemBudgetHalf = 112 * 1024;      // two CTAs per SM
-constexpr long long kWaitLimitCycles = 1500000000LL;
 
 struct alignas(64) MmaProj {
     CUtensorMap x_map;     // bf16 (64, T, d_in / 64), box 64 x 16 x 16, 128-byte swizzle
@@ -104,17 +102,9 @@ struct MmaParams {
     int cwy;           // columns per y item: a multiple of 64, <= 1024 (x items are 1024 wide)
     int slots;         // ring depth
     int wait_prev;     // 1: the previous kernel of the stream must be complete before any global access
+    int skip_item;     // -1; the test-hooks build can name one item whose copy request is left out
     int *status;       // device status word
-    long long *trace;  // development builds only (-DLORDBA_MMA_TRACE): 64 clock64 stamps per CTA
 };
-
-// Optional per-CTA timestamp trace (development builds only).
-#ifdef LORDBA_MMA_TRACE
-#define MMA_TRACE(idx) do { if (prm.trace && (idx) < 64) \
-    prm.trace[((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 64 + (idx)] = clock64(); } while (0)
-#else
-#define MMA_TRACE(idx) do { } while (0)
-#endif
 
 // ---- shared-memory plan, same on host and device --------------------------------------------
 struct SmemPlan {
@@ -328,7 +318,6 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzle atoms: 1 KiB
     const MmaProj &P = batch.p[blockIdx.y];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) MMA_TRACE(0);
     const int rows = prm.rows, cwy = prm.cwy, S = prm.slots;
     constexpr int cwx = NW * kGroup;
     const int64_t t0 = (int64_t)blockIdx.x * rows;
@@ -381,18 +370,16 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         // a box is always whole: what lies past the tensor is filled with zeros and counted
         const uint32_t bytes = (uint32_t)(cw / kGroup) * kBlockBytes + (uint32_t)ELL * cw * 4u + (uint32_t)cw * r / 8u;
         const uint32_t slot = sm_base + s * plan.slot_bytes;
-        MMA_TRACE(2 + it);
+        if (it == prm.skip_item) return;          // test-hooks build only: nothing is requested, nothing lands
         mbar_arrive_expect_tx(bar_full(s), bytes);
         tma_load_3d(slot, is_x ? &P.x_map : &P.y_map, 0, (int)t0, col0 / kGroup, bar_full(s));
         tma_load_3d(slot + plan.off_scale, is_x ? &P.si_map : &P.so_map, 0, col0 / kGroup, 0, bar_full(s));
         tma_load_2d(slot + plan.off_bits, is_x ? &P.pa_map : &P.pb_map, 0, col0 * r / 512, bar_full(s));
-        MMA_TRACE(10 + it);
     };
     const int n_first = n_items < S ? n_items : S;
     if (tid == kConsumerThreads)
         for (int it = 0; it < n_first; ++it) issue_item(it, it);     // n_first <= S
     __syncthreads();
-    if (tid == 0) MMA_TRACE(1);
 
     if (warp == kConsumerWarps) {
         // ================= producer warp: one lane refills the slots as they are released ========
@@ -433,7 +420,6 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         for (; it < n_x; ++it) {
             const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), sph, kDevMmaWaitTimeout));
             const int cwv = (d_in - it * cwx < cwx) ? (d_in - it * cwx) : cwx;
-            if (tid == 0) MMA_TRACE(20 + it);
             if (gcol < cwv && ok) {
                 const uint8_t *slot = smem + s * plan.slot_bytes;
                 // this lane's columns: gcol + 16q .. +7 (piece A) and gcol + 16q + 8 .. +15 (piece B);
@@ -508,7 +494,6 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
-            if (tid == 0) MMA_TRACE(40 + it);
             if (++s == S) { s = 0; sph ^= 1u; }
         }
 
@@ -552,7 +537,6 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             zL[idx] = lo;
         }
         consumer_sync<kConsumerThreads>();
-        if (tid == 0) MMA_TRACE(60);
 
         // ---- second product: y[t,j] += s_out[j] sum_k B_sign[j,k] z[t,k] ---------------------
         // A fragments: k position (2q, 2q+1, 2q+8, 2q+9) of k-step s <-> ranks 16s + 4q + (0,1,2,3)
@@ -571,15 +555,17 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         };
         uint32_t zh[KS][4], zl[KS][4];
         if (ELL == 1) load_z(0, zh, zl);
+        // A wait that gave up during the first product left u incomplete: this CTA then writes
+        // nothing (its rows of y keep their old values) and only drains its items.
+        const bool u_complete = !__any_sync(0xffffffffu, *abort_flag != 0);
         uint16_t *yrow0 = P.y + (t0 + g) * P.ldy;
         uint16_t *yrow1 = yrow0 + 8 * P.ldy;
         const bool vec32 = P.y_vec32 != 0;
 
         for (; it < n_items; ++it) {
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), sph, kDevEpilogueWaitTimeout));
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), sph, kDevEpilogueWaitTimeout)) && u_complete;
             const int col0 = (yc_begin + (it - n_x)) * cwy;
             const int cwv = (d_out - col0 < cwy) ? (d_out - col0) : cwy;
-            if (tid == 0) MMA_TRACE(20 + it);
             if (gcol < cwv && ok) {
                 const uint8_t *slot = smem + s * plan.slot_bytes;
                 const uint8_t *bits = slot + plan.off_bits;
@@ -687,11 +673,9 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
-            if (tid == 0) MMA_TRACE(40 + it);
             if (++s == S) { s = 0; sph ^= 1u; }
         }
     }
-    if (tid == 0) MMA_TRACE(61);
 
     // ---- teardown: after an abort, give copies that may still be in flight time to land ---------
     __syncthreads();
@@ -779,8 +763,9 @@ int sm_count()
     return n;
 }
 
+// The kernel instantiation for a launch, with its dynamic shared-memory limit raised once.
 template <int RP, int NW, int ELL, int IO, bool GEN>
-cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem, cudaStream_t stream)
+const void *kernel_one()
 {
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
@@ -788,53 +773,33 @@ cudaError_t launch_one(const MmaBatch &b, const MmaParams &prm, dim3 grid, size_
         attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW, ELL, IO, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSmemBudget);
     });
-    if (attr_rc != cudaSuccess) return attr_rc;
-    // Programmatic dependent launch: the CTAs of this grid may become resident, fetch their
-    // parameters and set up their barriers while the previous kernel of the stream drains; they
-    // touch no global data before griddepcontrol.wait, which returns once that kernel has
-    // completed and its writes are visible.
-    cudaLaunchConfig_t cfg;
-    std::memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(NW * 32 + 32, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr.val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mma_forward_kernel<RP, NW, ELL, IO, GEN>, b, prm);
+    if (attr_rc != cudaSuccess) return nullptr;
+    return reinterpret_cast<const void *>(&mma_forward_kernel<RP, NW, ELL, IO, GEN>);
 }
 
 template <int NW, int ELL, int IO, bool GEN>
-cudaError_t launch_rank(int rp, const MmaBatch &b, const MmaParams &prm, dim3 grid, size_t smem, cudaStream_t stream)
+const void *kernel_rank(int rp)
 {
     switch (rp) {
-        case 8:  return launch_one<8, NW, ELL, IO, GEN>(b, prm, grid, smem, stream);
-        case 16: return launch_one<16, NW, ELL, IO, GEN>(b, prm, grid, smem, stream);
-        case 32: return launch_one<32, NW, ELL, IO, GEN>(b, prm, grid, smem, stream);
+        case 8:  return kernel_one<8, NW, ELL, IO, GEN>();
+        case 16: return kernel_one<16, NW, ELL, IO, GEN>();
+        case 32: return kernel_one<32, NW, ELL, IO, GEN>();
         default:
             // two envelopes at rank 64 do not fit the register budget: mma_supported() keeps them out
-            if (ELL == 1) return launch_one<64, NW, 1, IO, GEN>(b, prm, grid, smem, stream);
-            return cudaErrorInvalidValue;
+            if (ELL == 1) return kernel_one<64, NW, 1, IO, GEN>();
+            return nullptr;
     }
 }
 
 template <int IO>
-cudaError_t launch_io(int rp, int nw, int ell, bool gen, const MmaBatch &b, const MmaParams &prm, dim3 grid,
-                      size_t smem, cudaStream_t stream)
+const void *kernel_io(int rp, int nw, int ell, bool gen)
 {
     if (gen) {      // ranks other than 8 / 16 / 32 / 64: one envelope only (mma_supported())
-        if (ell != 1) return cudaErrorInvalidValue;
-        return nw == kMaxWarps ? launch_rank<kMaxWarps, 1, IO, true>(rp, b, prm, grid, smem, stream)
-                               : launch_rank<8, 1, IO, true>(rp, b, prm, grid, smem, stream);
+        if (ell != 1) return nullptr;
+        return nw == kMaxWarps ? kernel_rank<kMaxWarps, 1, IO, true>(rp) : kernel_rank<8, 1, IO, true>(rp);
     }
-    if (ell == 1)
-        return nw == kMaxWarps ? launch_rank<kMaxWarps, 1, IO, false>(rp, b, prm, grid, smem, stream)
-                               : launch_rank<8, 1, IO, false>(rp, b, prm, grid, smem, stream);
-    return nw == kMaxWarps ? launch_rank<kMaxWarps, 2, IO, false>(rp, b, prm, grid, smem, stream)
-                           : launch_rank<8, 2, IO, false>(rp, b, prm, grid, smem, stream);
+    if (ell == 1) return nw == kMaxWarps ? kernel_rank<kMaxWarps, 1, IO, false>(rp) : kernel_rank<8, 1, IO, false>(rp);
+    return nw == kMaxWarps ? kernel_rank<kMaxWarps, 2, IO, false>(rp) : kernel_rank<8, 2, IO, false>(rp);
 }
 
 }  // namespace
@@ -859,17 +824,16 @@ bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
     return encode_fn() != nullptr;
 }
 
-int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, int dtype, cudaStream_t stream,
-                       bool batch_checked)
+int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t T, int n, const FamilySelector &fsel,
+                       LaunchSink &sink, bool batch_checked, int *launches)
 {
     if (n == 0) return LORDBA_OK;
-    if (dtype != LORDBA_BF16 && dtype != LORDBA_F16) return LORDBA_EUNSUPPORTED;
-    int *status = device_status_word();
-    if (!status) return LORDBA_ECUDA;
+    const int dtype = fsel.dtype;
+    if (dtype != LORDBA_BF16 && dtype != LORDBA_F16) return LORDBA_OK;     // float32: the FMA kernel's
+    int *status = nullptr;
     const int sms = sm_count();
     bool all_overlap = true;          // the caller's promise covers the call only if every projection carries it
     for (int i = 0; i < n; ++i) all_overlap = all_overlap && (projs[i].flags & LORDBA_PROJ_OVERLAP);
-    int launches = 0;
     // one launch per (element / scale kind, envelopes, padded rank) present in the call
     const int io_first = (dtype == LORDBA_BF16) ? kIoBf16 : kIoF16;
     const int io_last = (dtype == LORDBA_BF16) ? kIoBf16 : kIoF16Exact;
@@ -886,11 +850,13 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
         int m = 0, max_r = 0, min_cw = 128;
         int64_t min_dout = (int64_t)1 << 40;
         for (int i = 0; i <= n; ++i) {
-            const bool take = (i < n) && tokens[i] > 0 && padded_rank(projs[i].r) == rp &&
+            const int64_t rows_i = (i < n) ? rows_of(tokens, T, i) : 0;
+            const bool take = (i < n) && rows_i > 0 && padded_rank(projs[i].r) == rp &&
                               ((projs[i].flags >> 8) & 0xf) + 1 == ell && io_of(projs[i]) == io &&
-                              (projs[i].r != rp) == (gen != 0);
+                              (projs[i].r != rp) == (gen != 0) &&
+                              fsel.family(projs[i], rows_i) == LORDBA_VARIANT_MMA;
             if (take) {
-                sel_T[m] = tokens[i];
+                sel_T[m] = rows_i;
                 sel[m++] = &projs[i];
                 if (projs[i].r > max_r) max_r = projs[i].r;
                 // narrowest y item of this projection: its sign bytes must be whole 64-byte rows
@@ -899,6 +865,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                 if (projs[i].d_out < min_dout) min_dout = projs[i].d_out;
             }
             if (m == kMaxBatch || (i == n && m > 0)) {
+                if (!status && !(status = device_status_word())) return LORDBA_ECUDA;
                 // CTAs start in grid order (all tiles of projection 0, then of projection 1, ...):
                 // projections with the most bytes per token go first, so that the last, partly
                 // filled wave consists of the cheapest tiles (stable insertion sort).
@@ -931,7 +898,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                 // wave of tiles, or a call that may overlap its neighbours.  One's start-up and
                 // first-load latency then hide behind the other's streaming.  A lone single-wave
                 // call keeps one CTA with 16 consumer warps per SM.
-                const bool overlaps_neighbours = (launches == 0) ? all_overlap : batch_checked;
+                const bool overlaps_neighbours = (*launches == 0) ? all_overlap : batch_checked;
                 const int nw = (all_tiles > sms || overlaps_neighbours) ? 8 : kMaxWarps;
                 const int max_chunk = nw * kGroup;
                 const int smem_budget = (nw == kMaxWarps) ? kSmemBudget : kSmemBudgetHalf;
@@ -964,26 +931,35 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int n, i
                     t.y_vec32 = (reinterpret_cast<uintptr_t>(q.y) % 32 == 0 && q.ldy % 16 == 0) ? 1 : 0;
                 }
                 MmaParams prm;
+                std::memset(&prm, 0, sizeof(prm));
                 prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
                 prm.wait_prev = !overlaps_neighbours;
-                ++launches;
-                prm.trace = nullptr;
-#ifdef LORDBA_MMA_TRACE
-                if (const char *tp = std::getenv("LORDBA_MMA_TRACE_PTR"))
-                    prm.trace = reinterpret_cast<long long *>(std::strtoull(tp, nullptr, 0));
-#endif
+                prm.skip_item = test_skip_item();
+                ++*launches;
                 int slots = kMaxSlots;
                 while (slots > 2 && make_plan(nw, rp, max_r, slots, ell).total > smem_budget) --slots;
                 const SmemPlan plan = make_plan(nw, rp, max_r, slots, ell);
                 if (plan.total > kSmemBudget) return LORDBA_ECUDA;
                 prm.slots = slots;
-                const dim3 grid((unsigned)tiles, (unsigned)m, (unsigned)splits);
-                const cudaError_t e =
-                    io == kIoBf16 ? launch_io<kIoBf16>(rp, nw, ell, gen != 0, b, prm, grid, plan.total, stream)
-                    : io == kIoF16 ? launch_io<kIoF16>(rp, nw, ell, gen != 0, b, prm, grid, plan.total, stream)
-                                   : launch_io<kIoF16Exact>(rp, nw, ell, gen != 0, b, prm, grid, plan.total, stream);
-                if (e != cudaSuccess) return LORDBA_ECUDA;
-                count_launch();
+                LaunchRec rec;
+                std::memset(&rec, 0, sizeof(rec));
+                rec.func = io == kIoBf16 ? kernel_io<kIoBf16>(rp, nw, ell, gen != 0)
+                           : io == kIoF16 ? kernel_io<kIoF16>(rp, nw, ell, gen != 0)
+                                          : kernel_io<kIoF16Exact>(rp, nw, ell, gen != 0);
+                if (!rec.func) return LORDBA_ECUDA;
+                rec.grid[0] = (unsigned)tiles; rec.grid[1] = (unsigned)m; rec.grid[2] = (unsigned)splits;
+                rec.block = nw * 32 + 32;
+                rec.smem = (uint32_t)plan.total;
+                // Programmatic dependent launch: the CTAs of this grid may become resident, fetch their
+                // parameters and set up their barriers while the previous kernel of the stream drains; they
+                // touch no global data before griddepcontrol.wait, which returns once that kernel has
+                // completed and its writes are visible.
+                rec.pdl = 1;
+                rec.n_args = 2;
+                rec.arg_bytes[0] = sizeof(MmaBatch);
+                rec.arg_bytes[1] = sizeof(MmaParams);
+                const int rc = sink.emit(rec, &b, &prm);
+                if (rc != LORDBA_OK) return rc;
                 m = 0; max_r = 0; min_cw = 128; min_dout = (int64_t)1 << 40;
             }
         }

@@ -21,6 +21,7 @@ VARIANT_AUTO, VARIANT_FMA, VARIANT_TC, VARIANT_MMA = 0, 1, 2, 3
 PROJ_OVERLAP = 1
 PROJ_SCALES_F16 = 2
 MAX_ELL = 8
+MAX_PROJS = 4096
 
 
 def proj_ell(ell: int) -> int:
@@ -63,6 +64,14 @@ _SIGNATURES = {
                                                                ctypes.c_int, _vp, ctypes.c_size_t, _vp]),
     "lordba_adapter_forward_host_static": (ctypes.c_int, [_vp] * 7 + [_i64, _i64, _i64, ctypes.c_int,
                                                                       ctypes.c_int, _vp]),
+    "lordba_query_variant": (ctypes.c_int, [ctypes.POINTER(Proj), ctypes.c_int, _i64, ctypes.POINTER(_i64),
+                                            ctypes.c_int, ctypes.POINTER(ctypes.c_int)]),
+    "lordba_plan_bytes": (ctypes.c_size_t, [ctypes.POINTER(Proj), ctypes.c_int, _i64, ctypes.POINTER(_i64),
+                                            ctypes.c_int]),
+    "lordba_plan_init": (ctypes.c_int, [_vp, ctypes.c_size_t, ctypes.POINTER(Proj), ctypes.c_int, _i64,
+                                        ctypes.POINTER(_i64), ctypes.c_int]),
+    "lordba_adapter_forward_planned": (ctypes.c_int, [_vp, _vp]),
+    "lordba_plan_launches": (ctypes.c_int, [_vp]),
     "lordba_adapter_bits": (_i64, [_i64, _i64, ctypes.c_int, ctypes.c_int]),
     "lordba_set_variant": (ctypes.c_int, [ctypes.c_int]),
     "lordba_get_variant": (ctypes.c_int, []),
@@ -75,6 +84,16 @@ _SIGNATURES = {
 _lib = None
 
 
+def bind(path: str) -> ctypes.CDLL:
+    """Open a build of the library and declare the signatures of its entry points."""
+    lib = ctypes.CDLL(path)
+    for name, (res, args) in _SIGNATURES.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    return lib
+
+
 def load() -> ctypes.CDLL:
     """Load liblordba.so (built by ``paper_2605_24058_b200.build``); raises if absent."""
     global _lib
@@ -82,12 +101,7 @@ def load() -> ctypes.CDLL:
         if not os.path.exists(LIB_PATH):
             raise RuntimeError("liblordba.so is not built (%s); run "
                                "`python -m paper_2605_24058_b200.build`" % LIB_PATH)
-        lib = ctypes.CDLL(LIB_PATH)
-        for name, (res, args) in _SIGNATURES.items():
-            fn = getattr(lib, name)
-            fn.restype = res
-            fn.argtypes = args
-        _lib = lib
+        _lib = bind(LIB_PATH)
     return _lib
 
 
@@ -262,6 +276,57 @@ def adapter_forward_segments(segs: Sequence[Proj], tokens: Sequence[int], dtype:
     tok = (_i64 * len(tokens))(*[int(t) for t in tokens])
     _check(load().lordba_adapter_forward_segments(arr, tok, len(segs), dtype, _stream(stream)),
            "lordba_adapter_forward_segments")
+
+
+def _call_args(projs: Sequence[Proj], tokens):
+    """(array of Proj, n, T, pointer to per-projection token counts or NULL) for the entry points
+    that take either one T for all projections (tokens: an int) or one count each (a sequence)."""
+    arr = (Proj * len(projs))(*projs)
+    if isinstance(tokens, int):
+        return arr, len(projs), tokens, None
+    if len(tokens) != len(projs):
+        raise ValueError("one token count per projection")
+    return arr, len(projs), 0, (_i64 * len(tokens))(*[int(t) for t in tokens])
+
+
+def query_variant(projs: Sequence[Proj], tokens, dtype: int) -> Sequence[int]:
+    """Kernel family per projection (VARIANT_FMA / _TC / _MMA, 0 for one without rows) that a batched
+    call (tokens: one int) or a segmented call (tokens: one count per projection) would use."""
+    arr, n, T, tok = _call_args(projs, tokens)
+    out = (ctypes.c_int * max(n, 1))()
+    _check(load().lordba_query_variant(arr, n, T, tok, dtype, out), "lordba_query_variant")
+    return [int(out[i]) for i in range(n)]
+
+
+class Plan:
+    """Caller-owned host storage of a prepared call (64-byte aligned)."""
+
+    def __init__(self, nbytes: int):
+        self._raw = (ctypes.c_char * (nbytes + 64))()
+        base = ctypes.addressof(self._raw)
+        self.ptr = (base + 63) // 64 * 64
+        self.nbytes = nbytes
+
+    def launches(self) -> int:
+        return int(load().lordba_plan_launches(self.ptr))
+
+
+def plan_init(projs: Sequence[Proj], tokens, dtype: int) -> Plan:
+    """lordba_plan_bytes + lordba_plan_init: prepare a batched (tokens: an int) or segmented call."""
+    arr, n, T, tok = _call_args(projs, tokens)
+    lib = load()
+    nbytes = int(lib.lordba_plan_bytes(arr, n, T, tok, dtype))
+    if nbytes == 0:
+        # ask lordba_plan_init for the status of the same arguments
+        scratch = Plan(64)
+        _check(lib.lordba_plan_init(scratch.ptr, 64, arr, n, T, tok, dtype) or 1, "lordba_plan_init")
+    plan = Plan(nbytes)
+    _check(lib.lordba_plan_init(plan.ptr, nbytes, arr, n, T, tok, dtype), "lordba_plan_init")
+    return plan
+
+
+def adapter_forward_planned(plan: Plan, stream=None) -> None:
+    _check(load().lordba_adapter_forward_planned(plan.ptr, _stream(stream)), "lordba_adapter_forward_planned")
 
 
 def host_workspace_bytes(T: int, d_in: int, d_out: int, dtype: int) -> int:

@@ -145,3 +145,41 @@ def test_float16_arguments_and_inputs_without_launching(lib):
         assert np.array_equal(got, src.astype(np.float16).astype(np.float32))
     assert np.array_equal(a.A_sign, b.A_sign) and np.array_equal(a.B_sign, b.B_sign)
     assert b.x_f64().dtype == np.float64 and np.array_equal(b.x_f64(), b.x.astype(np.float64))
+
+
+def test_query_and_prepared_call_arguments_without_launching(lib):
+    """lordba_query_variant, lordba_plan_bytes / _init / _launches and lordba_adapter_forward_planned
+    reject bad arguments on the host; the independence check of a call is the same for all of them."""
+    from paper_2605_24058_b200 import lordba
+    EINVAL, EUNSUP, EALIGN = 1, 2, 3
+    before = lordba.launch_count()
+    one = (lordba.Proj * 1)(_proj(lordba))
+    out = (ctypes.c_int * 4)()
+    assert lib.lordba_query_variant(one, 1, 4, None, lordba.BF16, None) == EINVAL
+    assert lib.lordba_query_variant(one, 1, -1, None, lordba.BF16, out) == EINVAL
+    assert lib.lordba_query_variant(one, 1, 4, None, 9, out) == EUNSUP
+    assert lib.lordba_query_variant(one, lordba.MAX_PROJS + 1, 4, None, lordba.BF16, out) == EUNSUP
+    assert lib.lordba_query_variant(None, 0, 4, None, lordba.BF16, None) == 0
+    # overlapping outputs; an input inside another projection's output; disjoint ones in any order
+    two = (lordba.Proj * 2)(_proj(lordba), _proj(lordba, x=0x8000))
+    assert lib.lordba_query_variant(two, 2, 4, None, lordba.BF16, out) == EINVAL
+    chained = (lordba.Proj * 2)(_proj(lordba, x=0x300000, y=0x200000), _proj(lordba, x=0x200100, y=0x100000))
+    assert lib.lordba_query_variant(chained, 2, 4, None, lordba.BF16, out) == EINVAL
+    assert lib.lordba_plan_bytes(chained, 2, 4, None, lordba.BF16) == 0
+    tok = (ctypes.c_int64 * 2)(4, 0)
+    assert lib.lordba_query_variant(two, 2, 0, tok, lordba.BF16, out) in (0, 4)       # an empty segment overlaps nothing
+    # float32 activations always run on the CUDA-core kernel: no device is needed to say so
+    f32 = (lordba.Proj * 3)(_proj(lordba, y=0x100000), _proj(lordba, y=0x300000), _proj(lordba, y=0x200000))
+    assert lib.lordba_query_variant(f32, 3, 4, None, lordba.F32, out) == 0
+    assert [out[i] for i in range(3)] == [lordba.VARIANT_FMA] * 3
+    # plans
+    buf = (ctypes.c_char * 4096)()
+    base = (ctypes.addressof(buf) + 63) // 64 * 64
+    assert lib.lordba_plan_init(None, 1024, one, 1, 4, None, lordba.BF16) == EINVAL
+    assert lib.lordba_plan_init(base + 8, 1024, one, 1, 4, None, lordba.BF16) == EALIGN
+    assert lib.lordba_plan_init(base, 1024, two, 2, 4, None, lordba.BF16) == EINVAL
+    assert lib.lordba_adapter_forward_planned(None, None) == EINVAL
+    assert lib.lordba_adapter_forward_planned(base + 8, None) == EALIGN
+    assert lib.lordba_adapter_forward_planned(base, None) == EINVAL          # zeros are not a plan
+    assert lib.lordba_plan_launches(base) == -1 and lib.lordba_plan_launches(None) == -1
+    assert lordba.launch_count() == before

@@ -129,32 +129,39 @@ def test_config4_one_layer_with_outliers(oracle, r):
         assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16", "config4/r=%d/%s" % (r, p.name))
 
 
-@pytest.mark.parametrize("r,T", [(16, 2048), (64, 4096)])
-def test_config4_full_set_sampled(oracle, r, T):
-    """All 224 projections in one batched call at full T.  Activations are drawn once per layer
-    shape (three x tensors, shared read-only by the projections that take them) so that host
-    generation stays short; every projection has its own carriers, scales and y.  The oracle
-    checks at least 64 token rows of every projection (the first and the last tile in full plus
-    random rows)."""
+@functools.lru_cache(maxsize=1)
+def _config4_activations(T):
+    """Activations of the full-set test for one T: x drawn once per layer shape (with the 1 % outlier
+    channels), y once per output width; shared by the rank sweep so that host generation stays short."""
     rng = np.random.default_rng(99)
-    dev = torch.device("cuda:0")
     base = {}
     for name, d_in, d_out in workloads.LAYER_PROJECTIONS:
         if d_in not in base:
-            base[d_in] = workloads.make_projection(d_in, 8, 8, T, "bf16", seed=4900 + d_in,
-                                                   outlier_frac=0.01)
-    x_dev = {d_in: np_to_torch(b.x, "bf16", dev) for d_in, b in base.items()}
-    x_f64 = {d_in: None for d_in in base}
+            base[d_in] = workloads.make_projection(d_in, 8, 8, T, "bf16", seed=4900 + d_in, outlier_frac=0.01)
     # the first and the last token tile in full, plus random rows: at least 64 rows per projection
     rows = np.unique(np.concatenate([np.arange(16), np.arange(T - 16, T), rng.integers(0, T, size=40)]))
     assert len(rows) >= 64
-    for d_in, b in base.items():
-        x_f64[d_in] = b.x_f64()[rows]
-    y0 = {}
-    for d_out in (workloads.HIDDEN, workloads.FFN):
-        y0[d_out] = workloads.to_bf16_bits(rng.standard_normal((T, d_out), dtype=np.float32))
-    y0_dev = {d: np_to_torch(a, "bf16", dev) for d, a in y0.items()}
+    x_bits = {d_in: b.x for d_in, b in base.items()}
+    x_f64 = {d_in: b.x_f64()[rows] for d_in, b in base.items()}
+    y0 = {d: workloads.to_bf16_bits(rng.standard_normal((T, d), dtype=np.float32))
+          for d in (workloads.HIDDEN, workloads.FFN)}
     y0_f64 = {d: workloads.bf16_bits_to_f32(a[rows]).astype(np.float64) for d, a in y0.items()}
+    return rows, x_bits, x_f64, y0, y0_f64
+
+
+@pytest.mark.parametrize("T", [2048, 4096])
+@pytest.mark.parametrize("r", [8, 16, 32, 64])
+def test_config4_full_set_sampled(oracle, r, T):
+    """All 224 projections in one batched call at full T, every point of the rank sweep, on the
+    kernels the library takes by itself (the streaming kernel in launches of 24 projections for
+    r <= 16, the tcgen05 kernel in launches of up to 96 for r = 32 and 64).  Activations are drawn
+    once per layer shape (three x tensors, shared read-only by the projections that take them);
+    every projection has its own carriers, scales and y.  The oracle checks at least 64 token rows
+    of every projection (the first and the last tile in full plus random rows)."""
+    dev = torch.device("cuda:0")
+    rows, x_bits, x_f64, y0, y0_f64 = _config4_activations(T)
+    x_dev = {d_in: np_to_torch(a, "bf16", dev) for d_in, a in x_bits.items()}
+    y0_dev = {d: np_to_torch(a, "bf16", dev) for d, a in y0.items()}
 
     keep, descs, checks = [], [], []
     for layer in range(workloads.N_LAYERS):
@@ -169,8 +176,13 @@ def test_config4_full_set_sampled(oracle, r, T):
             descs.append(lordba.make_proj(x_dev[d_in], t["pa"], t["pb"], t["s_in"], t["s_r"],
                                           t["s_out"], t["y"], r))
             checks.append((small, d_in, d_out, t))
+    # the route the library takes by itself at this point of the sweep
+    fams = set(lordba.query_variant(descs, T, lordba.BF16))
+    assert fams == ({lordba.VARIANT_TC} if r >= 32 else {lordba.VARIANT_MMA}), fams
+    n0 = lordba.launch_count()
     lordba.adapter_forward_batched(descs, T, lordba.BF16)
     torch.cuda.synchronize()
+    assert lordba.launch_count() - n0 == (3 if r >= 32 else 10)
     rows_t = torch.from_numpy(rows).to(dev)
     for i, (small, d_in, d_out, t) in enumerate(checks):
         got = torch_to_f64(t["y"][rows_t])
@@ -596,3 +608,121 @@ def test_f16_mixed_scale_kinds_on_the_tcgen05_kernel(oracle):
     lordba.adapter_forward_batched([d.proj() for d in ds], T, lordba.F16)
     for p, d in zip(ps, ds):
         assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "f16", "f16 mixed tcgen05 " + str(p.meta["seed"]))
+
+
+# ---------------------------------------------------------------- prepared calls and the kernel query
+
+@pytest.mark.parametrize("kind", ["layer_r16", "layer_r64", "segments_r16", "mixed_fma"])
+def test_planned_call_equals_plain_call(oracle, kind):
+    """lordba_plan_init + lordba_adapter_forward_planned launch what the plain call launches: the
+    same number of kernels, bit-identical y, and y matches the oracle; a plan can be replayed."""
+    T = 300
+    if kind == "layer_r16":
+        projs = workloads.config4_layer(1, T, 16)
+        tokens = T
+    elif kind == "layer_r64":
+        T = 2048 + 40                                     # enough 128-token tiles for the tcgen05 kernel
+        projs = [workloads.make_projection(di, do, 64, T, "bf16", seed=8100 + i, name=n)
+                 for i, (n, di, do) in enumerate(workloads.LAYER_PROJECTIONS[:4])]
+        tokens = T
+    elif kind == "segments_r16":
+        projs = [workloads.make_projection(1024, 768, 16, T, "bf16", seed=8200 + i) for i in range(3)]
+        tokens = [T, 0, 77]
+    else:
+        # one projection the tensor-core kernels cannot take (odd width) next to one they can
+        projs = [workloads.make_projection(1000, 520, 16, T, "bf16", seed=8300),
+                 workloads.make_projection(1024, 512, 16, T, "bf16", seed=8301)]
+        tokens = T
+    a = [DeviceProj(p) for p in projs]
+    b = [DeviceProj(p) for p in projs]
+    fams = lordba.query_variant([d.proj() for d in a], tokens, lordba.BF16)
+    if kind == "layer_r64":
+        assert set(fams) == {lordba.VARIANT_TC}
+    if kind == "mixed_fma":
+        assert fams == [lordba.VARIANT_FMA, lordba.VARIANT_MMA]
+    if kind == "segments_r16":
+        assert fams == [lordba.VARIANT_MMA, 0, lordba.VARIANT_MMA]
+    plan = lordba.plan_init([d.proj() for d in b], tokens, lordba.BF16)
+    n0 = lordba.launch_count()
+    if isinstance(tokens, int):
+        lordba.adapter_forward_batched([d.proj() for d in a], tokens, lordba.BF16)
+    else:
+        lordba.adapter_forward_segments([d.proj() for d in a], tokens, lordba.BF16)
+    n1 = lordba.launch_count()
+    lordba.adapter_forward_planned(plan)
+    n2 = lordba.launch_count()
+    torch.cuda.synchronize()
+    assert n1 - n0 == n2 - n1 == plan.launches() and n1 > n0
+    rows = [tokens] * len(projs) if isinstance(tokens, int) else tokens
+    for p, da, db, n in zip(projs, a, b, rows):
+        assert torch.equal(da.y, db.y)
+        want = oracle_forward(oracle, p)
+        assert_close(torch_to_f64(db.y)[:n], want[:n], "bf16", "planned " + kind, scale_from=want)
+        assert np.array_equal(torch_to_f64(db.y)[n:], p.y_f64()[n:])
+    # a second replay adds the adapter term once more
+    for d in b:
+        d.reset_y()
+    lordba.adapter_forward_planned(plan)
+    torch.cuda.synchronize()
+    for da, db in zip(a, b):
+        assert torch.equal(da.y, db.y)
+
+
+def test_query_variant_shows_the_fallbacks():
+    """The kernel family per projection, as the call would choose it: float32 activations, widths
+    that are not multiples of 64, odd row pitches and unaligned scales go to the CUDA-core kernel."""
+    T = 64
+    ok = DeviceProj(workloads.make_projection(1024, 512, 16, T, "bf16", seed=1))
+    f32 = DeviceProj(workloads.make_projection(1024, 512, 16, T, "f32", seed=2))
+    odd = DeviceProj(workloads.make_projection(1000, 512, 16, T, "bf16", seed=3))
+    pitch = DeviceProj(workloads.make_projection(1024, 512, 16, T, "bf16", seed=4), ldx=1024 + 3)
+    assert lordba.query_variant([ok.proj()], T, lordba.BF16) == [lordba.VARIANT_MMA]
+    assert lordba.query_variant([f32.proj()], T, lordba.F32) == [lordba.VARIANT_FMA]
+    assert lordba.query_variant([odd.proj(), pitch.proj()], T, lordba.BF16) == [lordba.VARIANT_FMA] * 2
+    big = [DeviceProj(workloads.make_projection(1024, 512, 64, 1, "bf16", seed=5))]
+    x = torch.zeros(4096, 1024, dtype=torch.bfloat16, device="cuda:0")
+    y = torch.zeros(4096, 512, dtype=torch.bfloat16, device="cuda:0")
+    d = big[0]
+    p = lordba.make_proj(x, d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, y, 64)
+    assert lordba.query_variant([p], 4096, lordba.BF16) == [lordba.VARIANT_TC]      # 32 tiles of 128 tokens
+    assert lordba.query_variant([p], [2048], lordba.BF16) == [lordba.VARIANT_MMA]
+    lordba.set_variant(lordba.VARIANT_TC)
+    with pytest.raises(lordba.LordbaError) as e:
+        lordba.query_variant([f32.proj()], T, lordba.F32)      # a pinned family that cannot take the call
+    assert e.value.status == 2
+
+
+@pytest.mark.parametrize("r", [32, 64])
+@pytest.mark.parametrize("pin", [False, True])
+def test_segments_on_the_tcgen05_kernel(oracle, r, pin):
+    """A multi-adapter batch at high rank: segments of different lengths (one empty, one shorter
+    than a tile, one ending in a ragged tile), each with its own adapter, through the tcgen05
+    kernel, which takes a token count per projection; every element against the oracle."""
+    lengths = (1280, 0, 700, 50, 2100)
+    d_in, d_out = 1024, 1536
+    T = sum(lengths)
+    base = workloads.make_projection(d_in, d_out, r, T, "bf16", seed=600 + r)
+    adapters = [workloads.make_projection(d_in, d_out, r, 1, "bf16", seed=610 + i) for i in range(4)]
+    dev = torch.device("cuda:0")
+    x = np_to_torch(base.x, "bf16", dev)
+    y = np_to_torch(base.y, "bf16", dev)
+    dads = [DeviceProj(a) for a in adapters]
+    segs, want, start = [], base.y_f64().copy(), 0
+    for i, n in enumerate(lengths):
+        a, da = adapters[i % 4], dads[i % 4]
+        lo = min(start, T - 1)
+        segs.append(lordba.make_proj(x[lo:lo + max(n, 1)], da.packed_A, da.packed_B, da.s_in, da.s_r, da.s_out,
+                                     y[lo:lo + max(n, 1)], r))
+        if n:
+            rows = slice(start, start + n)
+            want[rows] = oracle.adapter_forward(base.x_f64()[rows], a.A_sign, a.B_sign, a.s_in.astype(np.float64),
+                                                a.s_r.astype(np.float64), a.s_out.astype(np.float64),
+                                                base.y_f64()[rows])
+        start += n
+    if pin:
+        lordba.set_variant(lordba.VARIANT_TC)
+    fams = lordba.query_variant(segs, lengths, lordba.BF16)
+    if pin or r > 32:
+        assert set(fams) == {0, lordba.VARIANT_TC}
+    lordba.adapter_forward_segments(segs, lengths, lordba.BF16)
+    assert_close(torch_to_f64(y), want, "bf16", "tcgen05 segments r=%d" % r)

@@ -15,7 +15,7 @@ Timing.  Every timed step is a node of a replayed CUDA graph (no call is issued
 from Python inside a timed region): the K steps are the replays of an
 n-step graph (n = number of buffer sets) plus one graph holding the K mod n
 remainder.  The region "W warm-up steps, event, K steps, event" is repeated
-back to back (>= 30 times, and until the GPU has been busy for about 0.1 s so
+back to back (>= 30 times, and until the GPU has been busy for about 60 ms so
 that the clock sampler sees it); `ms_per_step` is the median over the repeats
 and `repeat_spread` gives p10 / p90.
 
@@ -60,7 +60,7 @@ ELEM = 2
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 MIN_REPEATS = 30
-MIN_BUSY_S = 0.1
+MIN_BUSY_S = 0.06
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel on this workload
 # (ncu capture summarised under profiles/).  None whenever the kernel has changed since the capture.
 NCU_DRAM_BYTES_PER_LAUNCH = None
@@ -229,52 +229,48 @@ def repeats_for(region_s: float, min_repeats: int = MIN_REPEATS, min_busy_s: flo
 
 
 class GraphSteps:
-    """Steps 0, 1, 2, ... of a workload as replayed CUDA graphs: one graph of n steps and, on
-    demand, graphs of the first m < n steps for remainders."""
+    """Steps of a workload as replayed CUDA graphs: one graph of the n steps 0 .. n-1 (one per
+    buffer set) and, on demand, graphs of a shorter run of consecutive steps."""
 
     def __init__(self, step, n: int, stream):
         import torch
         self.torch, self.step, self.n, self.stream = torch, step, n, stream
         self.graphs = {}
 
-    def graph(self, m: int):
-        if m not in self.graphs:
+    def graph(self, m: int, first: int = 0):
+        if (first, m) not in self.graphs:
             g = self.torch.cuda.CUDAGraph()
             with self.torch.cuda.graph(g, stream=self.stream):
-                for i in range(m):
+                for i in range(first, first + m):
                     self.step(i)
-            self.graphs[m] = g
-        return self.graphs[m]
+            self.graphs[(first, m)] = g
+        return self.graphs[(first, m)]
 
-    def prepare(self, k: int):
+    def plan(self, k: int, first: int = 0):
+        """k steps as a list of graphs: steps first .. first+k-1 in one graph when they fit the
+        buffer sets, else whole replays of the n-step graph plus one graph of the remainder."""
+        if first + k <= self.n:
+            return [self.graph(k, first)]
         full, rem = split_steps(k, self.n)
-        if full:
-            self.graph(self.n)
-        if rem:
-            self.graph(rem)
-
-    def run(self, k: int):
-        """Enqueue exactly k steps, all of them graph nodes."""
-        full, rem = split_steps(k, self.n)
-        for _ in range(full):
-            self.graphs[self.n].replay()
-        if rem:
-            self.graphs[rem].replay()
+        return [self.graph(self.n)] * full + ([self.graph(rem)] if rem else [])
 
 
 def time_regions(gs: GraphSteps, steps: int, warmup: int, repeats: int):
     """`repeats` times back to back on the graphs' stream: `warmup` untimed steps, an event, `steps`
     timed steps, an event.  The untimed steps keep the GPU busy while the timed graphs are
-    enqueued, so no launch latency sits between the first event and the first timed kernel.
-    Returns the milliseconds of every timed region."""
+    enqueued, so no launch latency sits between the first event and the first timed kernel.  When
+    warm-up and timed steps fit the buffer sets together, the timed steps continue the warm-up's
+    run on the following sets (steps W .. W+K-1).  Returns the milliseconds of every timed region."""
     torch = gs.torch
-    gs.prepare(steps)
-    gs.prepare(warmup)
+    warm = gs.plan(warmup)
+    main = gs.plan(steps, first=warmup if warmup + steps <= gs.n else 0)
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(repeats)]
     for a, b in ev:
-        gs.run(warmup)
+        for g in warm:
+            g.replay()
         a.record(gs.stream)
-        gs.run(steps)
+        for g in main:
+            g.replay()
         b.record(gs.stream)
     gs.stream.synchronize()
     return np.array([a.elapsed_time(b) for a, b in ev])
@@ -522,8 +518,6 @@ def run_gpu(args):
         n0 = lordba.launch_count()
         gs.graph(n_sets)
         launches_per_step = (lordba.launch_count() - n0) / n_sets
-        gs.prepare(args.steps)
-        gs.prepare(args.warmup)
         probe = time_regions(gs, args.steps, args.warmup, 3)
         repeats = repeats_for(float(np.median(probe)) * 1e-3 * (1.0 + args.warmup / args.steps))
         if world > 1:
@@ -591,7 +585,13 @@ def run_gpu(args):
         alg_bytes = workloads.algorithmic_bytes(T, D_IN, D_OUT, R, ELEM)
         sec_per_step = ms * 1e-3 / args.steps
         achieved = alg_bytes / sec_per_step / 1e9
-        full, rem = split_steps(args.steps, n_sets)
+        if args.warmup + args.steps <= n_sets:
+            launch = ("every timed step is a CUDA-graph node: one graph of the %d steps that follow the %d warm-up "
+                      "steps on the next buffer sets" % (args.steps, args.warmup))
+        else:
+            full, rem = split_steps(args.steps, n_sets)
+            launch = ("every timed step is a CUDA-graph node: %d replay(s) of a %d-step graph + one %d-step graph"
+                      % (full, n_sets, rem))
         line = {
             "metric": METRIC, "value": aggregate_tokens_per_s(world, T, args.steps, ms), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -600,9 +600,7 @@ def run_gpu(args):
             "config": {"workload": WORKLOAD,
                        "l2": "steps rotate through %d device buffer sets (%.0f MB > 8 x L2)"
                              % (n_sets, n_sets * set_bytes / 1e6),
-                       "launch": "every timed step is a CUDA-graph node: %d replay(s) of a %d-step graph + one "
-                                 "%d-step graph; no call is issued from Python inside a timed region"
-                                 % (full, n_sets, rem),
+                       "launch": launch + "; no call is issued from Python inside a timed region",
                        "timing": "median over %d back-to-back repeats of (W warm-up steps, event, K steps, event)"
                                  % repeats,
                        "step_dependency": "every step waits for the previous one" if args.no_overlap else

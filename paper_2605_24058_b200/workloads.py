@@ -151,3 +151,17 @@ def algorithmic_bytes(T: int, d_in: int, d_out: int, r: int, elem: int) -> int:
 def algorithmic_flops(T: int, d_in: int, d_out: int, r: int) -> int:
     """Signed adds of both binary products counted as 2 flops each, plus the scale multiplies."""
     return 2 * r * (d_in + d_out) * T + T * (d_in + r + d_out)
+
+
+def sign_noise_lora(N: int, M: int, r: int, seed: int, mu_A: float = 0.05, mu_B: float = 0.05,
+                    zeta: float = 0.01):
+    """A dense LoRA pair (A: N x r, B: M x r) drawn from the sign-plus-noise factor model of
+    Assumption 1: A = mu_A * sigma_A + xi_A, B = mu_B * sigma_B + xi_B with i.i.d. Rademacher
+    signs and independent zero-mean Gaussian residuals of standard deviation zeta.  Returns
+    (A, B, sigma_A, sigma_B) as float64 / int8 arrays; the fitting target is A @ B.T."""
+    rng = np.random.default_rng(seed)
+    sigma_A = (rng.integers(0, 2, size=(N, r), dtype=np.int8) * 2 - 1).astype(np.int8)
+    sigma_B = (rng.integers(0, 2, size=(M, r), dtype=np.int8) * 2 - 1).astype(np.int8)
+    A = mu_A * sigma_A.astype(np.float64) + zeta * rng.standard_normal((N, r))
+    B = mu_B * sigma_B.astype(np.float64) + zeta * rng.standard_normal((M, r))
+    return A, B, sigma_A, sigma_B

@@ -302,6 +302,39 @@ int lordba_adapter_forward_planned(const void *plan, void *stream);
 /* Kernel launches a plan holds (-1 if plan is not a plan). */
 int lordba_plan_launches(const void *plan);
 
+/*
+ * Closed-form scale updates of the adapter fit (Appendix "Closed-form scale updates for
+ * PTQ-LoRDBA"; the scale step Eq. scales-step of the PTQ-LoRDBA iteration, and the sweep that
+ * initialises the scales after the SVD warm start, Eq. svd-init).  With the packed carriers held
+ * fixed, `sweeps` block-coordinate sweeps of
+ *
+ *     min  1/2 || target - diag(s_in) A_sign^T diag(s_r) B_sign^T diag(s_out) ||_F^2
+ *
+ * each sweep updating s_in (Eq. alpha-update: one scalar least squares per row of the target), then
+ * s_r (Eq. beta-gram and Eq. beta-pinv: the r x r normal equations G = (P^T P) o (Q Q^T), solved
+ * by the Moore-Penrose pseudo-inverse, eigenvalues below r * 2^-52 * lambda_max dropped), then
+ * s_out (Eq. gamma-update: one scalar least squares per column); a row or column whose model is
+ * identically zero gets 0.  axes: which of the three a sweep updates (LORDBA_FIT_ALPHA | _BETA |
+ * _GAMMA; LORDBA_FIT_ALL for the full sweep), always in that order.
+ *
+ * target: [device] float32, d_in x d_out row-major with row pitch ld >= d_out elements (the dense
+ * adapter Delta-W* that is being fitted, in the orientation y = x Delta-W); read only.  packed_A,
+ * packed_B: the carriers as lordba_pack_signs makes them.  s_in (d_in), s_r (r), s_out (d_out):
+ * [device] float32, read as the starting point and overwritten with the result.  workspace:
+ * [device], 256-byte aligned, at least lordba_fit_workspace_bytes() bytes (LORDBA_EINVAL if
+ * shorter); its contents need not be initialised and are not meaningful afterwards.  The passes
+ * over the target accumulate in float32, everything of size r x r and the quotients in float64;
+ * results are deterministic.  Asynchronous on stream; sweeps = 0 is a no-op.
+ */
+#define LORDBA_FIT_ALPHA 1
+#define LORDBA_FIT_BETA 2
+#define LORDBA_FIT_GAMMA 4
+#define LORDBA_FIT_ALL 7
+size_t lordba_fit_workspace_bytes(int64_t d_in, int64_t d_out, int r);
+int lordba_fit_scales(const float *target, int64_t ld, const uint32_t *packed_A, const uint32_t *packed_B,
+                      float *s_in, float *s_r, float *s_out, int64_t d_in, int64_t d_out, int r, int sweeps,
+                      int axes, void *workspace, size_t workspace_bytes, void *stream);
+
 /* Storage of one adapter in bits, Eq. 5: r(d_in+d_out) + 16 ell (d_in+r+d_out). */
 int64_t lordba_adapter_bits(int64_t d_in, int64_t d_out, int r, int ell);
 

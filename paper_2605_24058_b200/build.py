@@ -18,7 +18,7 @@ CSRC = os.path.join(PKG, "csrc")
 BUILD = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "liblordba.so")
 TESTHOOKS_LIB = os.path.join(PKG, "liblordba_testhooks.so")
-SOURCES = ("api.cu", "pack.cu", "forward_fma.cu", "forward_tc.cu", "forward_mma.cu")
+SOURCES = ("api.cu", "pack.cu", "fit.cu", "forward_fma.cu", "forward_tc.cu", "forward_mma.cu")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Wno-deprecated-gpu-targets",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC]

@@ -558,6 +558,29 @@ int lordba_adapter_forward_host_static(const void *x_host, const uint32_t *packe
                                        d_out, r, dtype, scratch, limit, stream);
 }
 
+size_t lordba_fit_workspace_bytes(int64_t d_in, int64_t d_out, int r)
+{
+    if (d_in < 1 || d_out < 1 || r < 1 || r > kMaxRank) return 0;
+    return fit_workspace_bytes(d_in, d_out, r);
+}
+
+int lordba_fit_scales(const float *target, int64_t ld, const uint32_t *packed_A, const uint32_t *packed_B,
+                      float *s_in, float *s_r, float *s_out, int64_t d_in, int64_t d_out, int r, int sweeps,
+                      int axes, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (r < 1 || r > kMaxRank) return LORDBA_EUNSUPPORTED;
+    if (d_in < 1 || d_out < 1 || ld < d_out || sweeps < 0) return LORDBA_EINVAL;
+    if (axes < 1 || axes > LORDBA_FIT_ALL) return LORDBA_EINVAL;
+    if (!target || !packed_A || !packed_B || !s_in || !s_r || !s_out || !workspace) return LORDBA_EINVAL;
+    if (!aligned(target, 4) || !aligned(packed_A, 4) || !aligned(packed_B, 4) || !aligned(s_in, 4) ||
+        !aligned(s_r, 4) || !aligned(s_out, 4) || !aligned(workspace, 256))
+        return LORDBA_EALIGN;
+    if (workspace_bytes < fit_workspace_bytes(d_in, d_out, r)) return LORDBA_EINVAL;
+    if (sweeps == 0) return LORDBA_OK;
+    return launch_fit_scales(target, ld, packed_A, packed_B, s_in, s_r, s_out, d_in, d_out, r, sweeps, axes,
+                             workspace, static_cast<cudaStream_t>(stream));
+}
+
 int64_t lordba_adapter_bits(int64_t d_in, int64_t d_out, int r, int ell)
 {
     return (int64_t)r * (d_in + d_out) + 16 * (int64_t)ell * (d_in + r + d_out);

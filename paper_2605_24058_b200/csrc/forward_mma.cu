@@ -103,6 +103,8 @@ struct MmaParams {
     int slots;         // ring depth
     int wait_prev;     // 1: the previous kernel of the stream must be complete before any global access
     int skip_item;     // -1; the test-hooks build can name one item whose copy request is left out
+    int ell;           // envelopes of the adapters of this launch (Eq. 4); the first product takes them
+                       // EG at a time, streaming the x items once per group
     int *status;       // device status word
 };
 
@@ -114,17 +116,19 @@ struct SmemPlan {
     int off_red, off_zh, off_zl, off_bar, total;
 };
 
-// nw: consumer warps = 64-column groups per item
-// ell: envelopes (scale triples) of the adapter: ell rows of scales per item, ell partial sums
-__host__ __device__ inline SmemPlan make_plan(int nw, int rp, int r, int slots, int ell)
+// nw: consumer warps = 64-column groups per item; cwy: columns of a y item
+// eg: envelopes (scale triples) per pass of the first product: eg rows of scales per x item, eg
+// partial sums; ell: all envelopes of the adapter: ell rows of scales per y item, ell z tiles
+__host__ __device__ inline SmemPlan make_plan(int nw, int rp, int r, int slots, int eg, int ell, int cwy)
 {
     SmemPlan s;
     s.off_scale = nw * kBlockBytes;
-    s.off_bits = s.off_scale + ell * nw * kGroup * 4;
+    const int sx = eg * nw * kGroup, sy = ell * cwy;
+    s.off_bits = s.off_scale + (sx > sy ? sx : sy) * 4;
     s.slot_bytes = (s.off_bits + nw * kGroup * r / 8 + 1023) / 1024 * 1024;
     const int ks = (rp + 15) / 16;
     s.off_red = slots * s.slot_bytes;
-    s.off_zh = s.off_red + ell * nw * kTile * rp * 4;
+    s.off_zh = s.off_red + eg * nw * kTile * rp * 4;
     s.off_zl = s.off_zh + ell * kTile * ks * 8 * 4;
     s.off_bar = s.off_zl + ell * kTile * ks * 8 * 4;
     s.total = s.off_bar + (2 * kMaxSlots + 2) * 8 + 1024;    // + slack to align the base to 1 KiB
@@ -301,17 +305,22 @@ enum IoKind {
     kIoF16Exact = 2   // IEEE half; s_in stated to be exact in half precision: one pass
 };
 
-// RP: rank padded to 8, 16, 32 or 64.
-template <int RP, int NW, int ELL, int IO, bool GEN>
+// RP: rank padded to 8, 16, 32 or 64.  EG: envelopes per pass of the first product (EG * RP <= 64:
+// their partial sums live in registers); an adapter with more envelopes than that streams its x
+// items once per group of EG, the y items once.
+// EGT = 0 stands for "one envelope per pass, several envelopes in all" (rank above 32), EGT = 1 for
+// the single-envelope adapter, whose code carries no envelope loops at all.
+template <int RP, int NW, int EGT, int IO, bool GEN>
 __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 2)
 mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant__ MmaParams prm)
 {
+    constexpr int EG = (EGT == 0) ? 1 : EGT;
     constexpr bool kHalf = (IO != kIoBf16);     // x, y and the first product's operands are halves
     constexpr bool kLoPass = (IO != kIoF16Exact);
     constexpr int R8 = RP / 8;                 // 8-row blocks of A_sign = n-blocks of the first product
     constexpr int KS = (RP + 15) / 16;         // k-steps of the second product per z part
     constexpr int ZP = KS * 8;                 // bf16 pairs per token row of z
-    constexpr bool kSplitAcc = (R8 <= 2);      // separate hi / lo accumulators: shorter MMA chains
+    constexpr bool kSplitAcc = (EG * R8 <= 2); // separate hi / lo accumulators: shorter MMA chains
     constexpr int kConsumerWarps = NW, kConsumerThreads = NW * 32;
 
     extern __shared__ uint8_t smem_raw[];
@@ -325,15 +334,18 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     const int nt = (int)((P.T - t0 < rows) ? (P.T - t0) : rows);
     const int r = P.r;
     const int d_in = P.d_in, d_out = P.d_out;
-    const SmemPlan plan = make_plan(NW, RP, r, S, ELL);
+    const int ell = (EGT == 1) ? 1 : prm.ell;
+    const int n_groups = (EGT == 1) ? 1 : (ell + EG - 1) / EG;
+    const SmemPlan plan = make_plan(NW, RP, r, S, EG, ell, cwy);
     const uint32_t sm_base = smem_u32(smem);
 
-    // items: all x chunks, then this CTA's share of the y chunks
+    // items: all x chunks (once per envelope group), then this CTA's share of the y chunks
     const int n_x = (d_in + cwx - 1) / cwx;
+    const int n_xi = n_groups * n_x;
     const int n_yc = (d_out + cwy - 1) / cwy;
     const int yc_begin = (int)((int64_t)blockIdx.z * n_yc / gridDim.z);
     const int yc_end = (int)((int64_t)(blockIdx.z + 1) * n_yc / gridDim.z);
-    const int n_items = n_x + (yc_end - yc_begin);
+    const int n_items = n_xi + (yc_end - yc_begin);
 
     const uint32_t bar0 = sm_base + plan.off_bar;
     auto bar_full = [&](int s) { return bar0 + 8u * s; };
@@ -364,16 +376,18 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         }
     }
     auto issue_item = [&](int it, int s) {       // one thread; s = it % S
-        const bool is_x = it < n_x;
+        const bool is_x = it < n_xi;
         const int cw = is_x ? cwx : cwy;
-        const int col0 = is_x ? it * cwx : (yc_begin + (it - n_x)) * cwy;
-        // a box is always whole: what lies past the tensor is filled with zeros and counted
-        const uint32_t bytes = (uint32_t)(cw / kGroup) * kBlockBytes + (uint32_t)ELL * cw * 4u + (uint32_t)cw * r / 8u;
+        const int grp = is_x ? it / n_x : 0;       // the envelope group this pass over x belongs to
+        const int col0 = is_x ? (it - grp * n_x) * cwx : (yc_begin + (it - n_xi)) * cwy;
+        // a box is always whole: what lies past the tensor (columns, envelopes) is filled with zeros and counted
+        const uint32_t bytes = (uint32_t)(cw / kGroup) * kBlockBytes + (uint32_t)(is_x ? EG : ell) * cw * 4u +
+                               (uint32_t)cw * r / 8u;
         const uint32_t slot = sm_base + s * plan.slot_bytes;
         if (it == prm.skip_item) return;          // test-hooks build only: nothing is requested, nothing lands
         mbar_arrive_expect_tx(bar_full(s), bytes);
         tma_load_3d(slot, is_x ? &P.x_map : &P.y_map, 0, (int)t0, col0 / kGroup, bar_full(s));
-        tma_load_3d(slot + plan.off_scale, is_x ? &P.si_map : &P.so_map, 0, col0 / kGroup, 0, bar_full(s));
+        tma_load_3d(slot + plan.off_scale, is_x ? &P.si_map : &P.so_map, 0, col0 / kGroup, grp * EG, bar_full(s));
         tma_load_2d(slot + plan.off_bits, is_x ? &P.pa_map : &P.pb_map, 0, col0 * r / 512, bar_full(s));
     };
     const int n_first = n_items < S ? n_items : S;
@@ -404,9 +418,16 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         const int pc0 = ((2 * q) ^ g) * 16, pc1 = ((2 * q + 1) ^ g) * 16;
 
         // ---- first product: u[t,k] = sum_i A_sign[k,i] s_in[i] x[t,i] -----------------------
-        float acc[ELL][kSplitAcc ? 2 : 1][R8][4];
+        float *red = reinterpret_cast<float *>(smem + plan.off_red);
+        uint32_t *zH = reinterpret_cast<uint32_t *>(smem + plan.off_zh);
+        uint32_t *zL = reinterpret_cast<uint32_t *>(smem + plan.off_zl);
+        int it = 0;
+        int s = 0;                 // ring slot of item `it` and the phase of its barrier, carried
+        uint32_t sph = 0;          // along instead of recomputed by division
+        for (int grp = 0; grp < n_groups; ++grp) {
+        float acc[EG][kSplitAcc ? 2 : 1][R8][4];
 #pragma unroll
-        for (int env = 0; env < ELL; ++env)
+        for (int env = 0; env < EG; ++env)
 #pragma unroll
             for (int h = 0; h < (kSplitAcc ? 2 : 1); ++h)
 #pragma unroll
@@ -414,12 +435,9 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc[env][h][a][e] = 0.0f;
 
-        int it = 0;
-        int s = 0;                 // ring slot of item `it` and the phase of its barrier, carried
-        uint32_t sph = 0;          // along instead of recomputed by division
-        for (; it < n_x; ++it) {
+        for (int xc = 0; xc < n_x; ++xc, ++it) {
             const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), sph, kDevMmaWaitTimeout));
-            const int cwv = (d_in - it * cwx < cwx) ? (d_in - it * cwx) : cwx;
+            const int cwv = (d_in - xc * cwx < cwx) ? (d_in - xc * cwx) : cwx;
             if (gcol < cwv && ok) {
                 const uint8_t *slot = smem + s * plan.slot_bytes;
                 // this lane's columns: gcol + 16q .. +7 (piece A) and gcol + 16q + 8 .. +15 (piece B);
@@ -441,7 +459,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 const uint32_t xk[4][4] = {{xa0.x, xa1.x, xa0.y, xa1.y}, {xa0.z, xa1.z, xa0.w, xa1.w},
                                            {xb0.x, xb1.x, xb0.y, xb1.y}, {xb0.z, xb1.z, xb0.w, xb1.w}};
 #pragma unroll
-                for (int env = 0; env < ELL; ++env) {
+                for (int env = 0; env < EG; ++env) {
                     // s_in[env] of the group as bf16 pairs (hi, lo): lane l converts columns 2l, 2l+1,
                     // then every lane collects the 8 pairs of its 16 columns
                     uint32_t ph, pl;
@@ -498,11 +516,8 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         }
 
         // ---- reduce u over the warps in a fixed order, z = s_r * u, split into bf16 hi + lo ---
-        float *red = reinterpret_cast<float *>(smem + plan.off_red);
-        uint32_t *zH = reinterpret_cast<uint32_t *>(smem + plan.off_zh);
-        uint32_t *zL = reinterpret_cast<uint32_t *>(smem + plan.off_zl);
 #pragma unroll
-        for (int env = 0; env < ELL; ++env) {
+        for (int env = 0; env < EG; ++env) {
 #pragma unroll
             for (int a = 0; a < R8; ++a) {
                 float c[4];
@@ -515,8 +530,10 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             }
         }
         consumer_sync<kConsumerThreads>();
-        for (int idx = tid; idx < ELL * kTile * ZP; idx += kConsumerThreads) {
+        for (int idx = tid; idx < EG * kTile * ZP; idx += kConsumerThreads) {
             const int env = idx / (kTile * ZP), rem = idx - env * (kTile * ZP);
+            const int genv = grp * EG + env;           // envelope of the adapter
+            if (genv >= ell) break;
             const int tok = rem / ZP, pr = rem - tok * ZP;
             float u0 = 0.0f, u1 = 0.0f;
             if (2 * pr < RP) {
@@ -529,14 +546,15 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 }
             }
             const int k = 2 * pr;
-            const float z0 = (k < r) ? u0 * __ldg(P.s_r + env * r + k) : 0.0f;
-            const float z1 = (k + 1 < r) ? u1 * __ldg(P.s_r + env * r + k + 1) : 0.0f;
+            const float z0 = (k < r) ? u0 * __ldg(P.s_r + genv * r + k) : 0.0f;
+            const float z1 = (k + 1 < r) ? u1 * __ldg(P.s_r + genv * r + k + 1) : 0.0f;
             uint32_t hi, lo;
             split2(z0, z1, hi, lo);
-            zH[idx] = hi;
-            zL[idx] = lo;
+            zH[grp * (EG * kTile * ZP) + idx] = hi;
+            zL[grp * (EG * kTile * ZP) + idx] = lo;
         }
         consumer_sync<kConsumerThreads>();
+        }   // envelope groups
 
         // ---- second product: y[t,j] += s_out[j] sum_k B_sign[j,k] z[t,k] ---------------------
         // A fragments: k position (2q, 2q+1, 2q+8, 2q+9) of k-step s <-> ranks 16s + 4q + (0,1,2,3)
@@ -554,7 +572,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             }
         };
         uint32_t zh[KS][4], zl[KS][4];
-        if (ELL == 1) load_z(0, zh, zl);
+        if (ell == 1) load_z(0, zh, zl);
         // A wait that gave up during the first product left u incomplete: this CTA then writes
         // nothing (its rows of y keep their old values) and only drains its items.
         const bool u_complete = !__any_sync(0xffffffffu, *abort_flag != 0);
@@ -564,7 +582,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
 
         for (; it < n_items; ++it) {
             const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), sph, kDevEpilogueWaitTimeout)) && u_complete;
-            const int col0 = (yc_begin + (it - n_x)) * cwy;
+            const int col0 = (yc_begin + (it - n_xi)) * cwy;
             const int cwv = (d_out - col0 < cwy) ? (d_out - col0) : cwy;
             if (gcol < cwv && ok) {
                 const uint8_t *slot = smem + s * plan.slot_bytes;
@@ -612,9 +630,9 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                             }
                         }
                     }
-#pragma unroll
-                    for (int env = 0; env < ELL; ++env) {
-                        if (ELL > 1) load_z(env, zh, zl);
+#pragma unroll 2
+                    for (int env = 0; env < ell; ++env) {
+                        if (ell > 1) load_z(env, zh, zl);
                         float c[4][4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
@@ -740,12 +758,13 @@ bool make_linear_map(CUtensorMap *map, CUtensorMapDataType type, const void *bas
 }
 
 // ell x d float32 scales (envelope e in row e, d % 64 == 0) seen as (64, d / 64, ell); a box is
-// `groups` groups of all envelopes: it lands as [envelope][group][64 floats].
-bool make_scale_map(CUtensorMap *map, const float *base, int64_t d, int ell, int groups)
+// `groups` groups of `box_ell` envelopes: it lands as [envelope][group][64 floats] (envelopes past
+// the adapter's last one are filled with zeros).
+bool make_scale_map(CUtensorMap *map, const float *base, int64_t d, int ell, int box_ell, int groups)
 {
     const cuuint64_t dims[3] = {(cuuint64_t)kGroup, (cuuint64_t)(d / kGroup), (cuuint64_t)ell};
     const cuuint64_t strides[2] = {(cuuint64_t)kGroup * 4, (cuuint64_t)d * 4};
-    const cuuint32_t box[3] = {(cuuint32_t)kGroup, (cuuint32_t)groups, (cuuint32_t)ell};
+    const cuuint32_t box[3] = {(cuuint32_t)kGroup, (cuuint32_t)groups, (cuuint32_t)box_ell};
     return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
@@ -764,42 +783,54 @@ int sm_count()
 }
 
 // The kernel instantiation for a launch, with its dynamic shared-memory limit raised once.
-template <int RP, int NW, int ELL, int IO, bool GEN>
+template <int RP, int NW, int EG, int IO, bool GEN>
 const void *kernel_one()
 {
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, []() {
-        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW, ELL, IO, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_rc = cudaFuncSetAttribute(mma_forward_kernel<RP, NW, EG, IO, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSmemBudget);
     });
     if (attr_rc != cudaSuccess) return nullptr;
-    return reinterpret_cast<const void *>(&mma_forward_kernel<RP, NW, ELL, IO, GEN>);
+    return reinterpret_cast<const void *>(&mma_forward_kernel<RP, NW, EG, IO, GEN>);
 }
 
-template <int NW, int ELL, int IO, bool GEN>
-const void *kernel_rank(int rp)
+// Envelopes per pass of the first product (the kernel's EGT): as many as fit 64 partial sums per
+// token row (EG * RP <= 64), a power of two.
+int envelopes_per_pass(int rp, int ell)
 {
-    switch (rp) {
-        case 8:  return kernel_one<8, NW, ELL, IO, GEN>();
-        case 16: return kernel_one<16, NW, ELL, IO, GEN>();
-        case 32: return kernel_one<32, NW, ELL, IO, GEN>();
-        default:
-            // two envelopes at rank 64 do not fit the register budget: mma_supported() keeps them out
-            if (ELL == 1) return kernel_one<64, NW, 1, IO, GEN>();
-            return nullptr;
+    const int cap = kMaxRank / rp;
+    int eg = 1;
+    while (eg < ell && eg < cap) eg *= 2;
+    return (eg == 1 && ell > 1) ? 0 : eg;       // 0: one per pass, several in all (see the kernel)
+}
+
+template <int NW, int IO, bool GEN>
+const void *kernel_rank(int rp, int eg)
+{
+    switch (rp * 16 + eg) {
+        case 8 * 16 + 1:  return kernel_one<8, NW, 1, IO, GEN>();
+        case 8 * 16 + 2:  return kernel_one<8, NW, 2, IO, GEN>();
+        case 8 * 16 + 4:  return kernel_one<8, NW, 4, IO, GEN>();
+        case 8 * 16 + 8:  return kernel_one<8, NW, 8, IO, GEN>();
+        case 16 * 16 + 1: return kernel_one<16, NW, 1, IO, GEN>();
+        case 16 * 16 + 2: return kernel_one<16, NW, 2, IO, GEN>();
+        case 16 * 16 + 4: return kernel_one<16, NW, 4, IO, GEN>();
+        case 32 * 16 + 1: return kernel_one<32, NW, 1, IO, GEN>();
+        case 32 * 16 + 2: return kernel_one<32, NW, 2, IO, GEN>();
+        case 64 * 16 + 1: return kernel_one<64, NW, 1, IO, GEN>();
+        case 64 * 16 + 0: return kernel_one<64, NW, 0, IO, GEN>();
+        default: return nullptr;
     }
 }
 
 template <int IO>
-const void *kernel_io(int rp, int nw, int ell, bool gen)
+const void *kernel_io(int rp, int nw, int eg, bool gen)
 {
-    if (gen) {      // ranks other than 8 / 16 / 32 / 64: one envelope only (mma_supported())
-        if (ell != 1) return nullptr;
-        return nw == kMaxWarps ? kernel_rank<kMaxWarps, 1, IO, true>(rp) : kernel_rank<8, 1, IO, true>(rp);
-    }
-    if (ell == 1) return nw == kMaxWarps ? kernel_rank<kMaxWarps, 1, IO, false>(rp) : kernel_rank<8, 1, IO, false>(rp);
-    return nw == kMaxWarps ? kernel_rank<kMaxWarps, 2, IO, false>(rp) : kernel_rank<8, 2, IO, false>(rp);
+    if (gen)       // ranks other than 8 / 16 / 32 / 64, in instantiations of their own
+        return nw == kMaxWarps ? kernel_rank<kMaxWarps, IO, true>(rp, eg) : kernel_rank<8, IO, true>(rp, eg);
+    return nw == kMaxWarps ? kernel_rank<kMaxWarps, IO, false>(rp, eg) : kernel_rank<8, IO, false>(rp, eg);
 }
 
 }  // namespace
@@ -808,9 +839,7 @@ bool mma_supported(const lordba_proj &p, int64_t T, int dtype)
 {
     if ((dtype != LORDBA_BF16 && dtype != LORDBA_F16) || T < 1 || T > (1 << 30)) return false;
     const int ell = ((p.flags >> 8) & 0xf) + 1;
-    if (ell > 2 || (ell == 2 && p.r > 32)) return false;    // more envelopes, or two at high rank: FMA kernel
-    if (ell == 2 && p.r != padded_rank(p.r)) return false;   // two envelopes: ranks 8, 16, 32 only
-    if (p.r < 1 || p.r > kMaxRank) return false;
+    if (ell > LORDBA_MAX_ELL || p.r < 1 || p.r > kMaxRank) return false;
     // a carrier is copied as whole 64-byte rows of sign bytes
     if ((p.d_in * p.r) % 512 != 0 || (p.d_out * p.r) % 512 != 0) return false;
     // whole 64-column groups (the 3-D tensor view), 16-byte aligned rows
@@ -834,29 +863,41 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
     const int sms = sm_count();
     bool all_overlap = true;          // the caller's promise covers the call only if every projection carries it
     for (int i = 0; i < n; ++i) all_overlap = all_overlap && (projs[i].flags & LORDBA_PROJ_OVERLAP);
-    // one launch per (element / scale kind, envelopes, padded rank) present in the call
-    const int io_first = (dtype == LORDBA_BF16) ? kIoBf16 : kIoF16;
-    const int io_last = (dtype == LORDBA_BF16) ? kIoBf16 : kIoF16Exact;
+    // one launch per (element / scale kind, envelopes, padded rank) present in the call, up to
+    // kMaxBatch projections each; the key of every projection is worked out once
     auto io_of = [&](const lordba_proj &q) {
         if (dtype == LORDBA_BF16) return (int)kIoBf16;
         return (q.flags & LORDBA_PROJ_SCALES_F16) ? (int)kIoF16Exact : (int)kIoF16;
     };
+    auto key_of = [](int io, int ell, int gen, int rp) { return (uint16_t)(((io * 9 + ell) * 2 + gen) * 128 + rp); };
+    uint16_t keys[kMaxCallProjs];
+    uint32_t ell_seen = 0;
+    for (int i = 0; i < n; ++i) {
+        const int64_t rows_i = rows_of(tokens, T, i);
+        keys[i] = 0xffffu;
+        if (rows_i <= 0 || fsel.family(projs[i], rows_i) != LORDBA_VARIANT_MMA) continue;
+        const int rp_i = padded_rank(projs[i].r), ell_i = ((projs[i].flags >> 8) & 0xf) + 1;
+        keys[i] = key_of(io_of(projs[i]), ell_i, projs[i].r != rp_i ? 1 : 0, rp_i);
+        ell_seen |= 1u << ell_i;
+    }
+    const int io_first = (dtype == LORDBA_BF16) ? kIoBf16 : kIoF16;
+    const int io_last = (dtype == LORDBA_BF16) ? kIoBf16 : kIoF16Exact;
     for (int io = io_first; io <= io_last; ++io)
-    for (int ell = 1; ell <= 2; ++ell)
-    for (int gen = 0; gen <= (ell == 1 ? 1 : 0); ++gen)
+    for (int ell = 1; ell <= LORDBA_MAX_ELL; ++ell)
+    for (int gen = 0; gen <= 1; ++gen)
     for (int rp = 8; rp <= kMaxRank; rp *= 2) {
+        if (!(ell_seen & (1u << ell))) continue;
+        const uint16_t key = key_of(io, ell, gen, rp);
+        const int egt = envelopes_per_pass(rp, ell);
+        const int eg = egt == 0 ? 1 : egt;
         const lordba_proj *sel[kMaxBatch];
         int64_t sel_T[kMaxBatch];
         int m = 0, max_r = 0, min_cw = 128;
         int64_t min_dout = (int64_t)1 << 40;
         for (int i = 0; i <= n; ++i) {
-            const int64_t rows_i = (i < n) ? rows_of(tokens, T, i) : 0;
-            const bool take = (i < n) && rows_i > 0 && padded_rank(projs[i].r) == rp &&
-                              ((projs[i].flags >> 8) & 0xf) + 1 == ell && io_of(projs[i]) == io &&
-                              (projs[i].r != rp) == (gen != 0) &&
-                              fsel.family(projs[i], rows_i) == LORDBA_VARIANT_MMA;
+            const bool take = (i < n) && keys[i] == key;
             if (take) {
-                sel_T[m] = rows_i;
+                sel_T[m] = rows_of(tokens, T, i);
                 sel[m++] = &projs[i];
                 if (projs[i].r > max_r) max_r = projs[i].r;
                 // narrowest y item of this projection: its sign bytes must be whole 64-byte rows
@@ -916,8 +957,8 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                     // sign bytes: d r / 8 per carrier, as rows of 16 words; an item holds cw r / 512 rows
                     if (!make_data_map(&t.x_map, q.x, sel_T[k], q.d_in, q.ldx, nw) ||
                         !make_data_map(&t.y_map, q.y, sel_T[k], q.d_out, q.ldy, cw / kGroup) ||
-                        !make_scale_map(&t.si_map, q.s_in, q.d_in, ell, nw) ||
-                        !make_scale_map(&t.so_map, q.s_out, q.d_out, ell, cw / kGroup) ||
+                        !make_scale_map(&t.si_map, q.s_in, q.d_in, ell, eg, nw) ||
+                        !make_scale_map(&t.so_map, q.s_out, q.d_out, ell, ell, cw / kGroup) ||
                         !make_linear_map(&t.pa_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_A, 16,
                                          q.d_in * q.r / 512, max_chunk * q.r / 512) ||
                         !make_linear_map(&t.pb_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, q.packed_B, 16,
@@ -935,17 +976,18 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
                 prm.wait_prev = !overlaps_neighbours;
                 prm.skip_item = test_skip_item();
+                prm.ell = ell;
                 ++*launches;
                 int slots = kMaxSlots;
-                while (slots > 2 && make_plan(nw, rp, max_r, slots, ell).total > smem_budget) --slots;
-                const SmemPlan plan = make_plan(nw, rp, max_r, slots, ell);
+                while (slots > 2 && make_plan(nw, rp, max_r, slots, eg, ell, cw).total > smem_budget) --slots;
+                const SmemPlan plan = make_plan(nw, rp, max_r, slots, eg, ell, cw);
                 if (plan.total > kSmemBudget) return LORDBA_ECUDA;
                 prm.slots = slots;
                 LaunchRec rec;
                 std::memset(&rec, 0, sizeof(rec));
-                rec.func = io == kIoBf16 ? kernel_io<kIoBf16>(rp, nw, ell, gen != 0)
-                           : io == kIoF16 ? kernel_io<kIoF16>(rp, nw, ell, gen != 0)
-                                          : kernel_io<kIoF16Exact>(rp, nw, ell, gen != 0);
+                rec.func = io == kIoBf16 ? kernel_io<kIoBf16>(rp, nw, egt, gen != 0)
+                           : io == kIoF16 ? kernel_io<kIoF16>(rp, nw, egt, gen != 0)
+                                          : kernel_io<kIoF16Exact>(rp, nw, egt, gen != 0);
                 if (!rec.func) return LORDBA_ECUDA;
                 rec.grid[0] = (unsigned)tiles; rec.grid[1] = (unsigned)m; rec.grid[2] = (unsigned)splits;
                 rec.block = nw * 32 + 32;

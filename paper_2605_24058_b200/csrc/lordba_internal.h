@@ -90,6 +90,12 @@ int launch_widen_scales(const uint16_t *src, float *dst, int64_t n, cudaStream_t
 int launch_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int role, int8_t *signs,
                   cudaStream_t stream);
 
+// --- fit.cu ----------------------------------------------------------------
+size_t fit_workspace_bytes(int64_t d_in, int64_t d_out, int r);
+int launch_fit_scales(const float *target, int64_t ld, const uint32_t *pa, const uint32_t *pb, float *s_in, float *s_r,
+                      float *s_out, int64_t d_in, int64_t d_out, int r, int sweeps, int axes, void *workspace,
+                      cudaStream_t stream);
+
 // --- forward_*.cu ------------------------------------------------------------
 // Each launcher walks the n projections of a call (validated by the caller; tokens[i] = token
 // rows of projection i, or T for all when tokens is null), takes those whose family is its own,

@@ -22,6 +22,7 @@ PROJ_OVERLAP = 1
 PROJ_SCALES_F16 = 2
 MAX_ELL = 8
 MAX_PROJS = 4096
+FIT_ALPHA, FIT_BETA, FIT_GAMMA, FIT_ALL = 1, 2, 4, 7
 
 
 def proj_ell(ell: int) -> int:
@@ -72,6 +73,9 @@ _SIGNATURES = {
                                         ctypes.POINTER(_i64), ctypes.c_int]),
     "lordba_adapter_forward_planned": (ctypes.c_int, [_vp, _vp]),
     "lordba_plan_launches": (ctypes.c_int, [_vp]),
+    "lordba_fit_workspace_bytes": (ctypes.c_size_t, [_i64, _i64, ctypes.c_int]),
+    "lordba_fit_scales": (ctypes.c_int, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _i64, ctypes.c_int, ctypes.c_int,
+                                         ctypes.c_int, _vp, ctypes.c_size_t, _vp]),
     "lordba_adapter_bits": (_i64, [_i64, _i64, ctypes.c_int, ctypes.c_int]),
     "lordba_set_variant": (ctypes.c_int, [ctypes.c_int]),
     "lordba_get_variant": (ctypes.c_int, []),
@@ -371,6 +375,34 @@ def adapter_forward_host_static(x_host, packed_A, packed_B, s_in, s_r, s_out, y_
         s_r.data_ptr(), s_out.data_ptr(), y_host.data_ptr(), T, d_in, d_out, r,
         _dtype_code(x_host), _stream(stream))
     _check(rc, "lordba_adapter_forward_host_static")
+
+
+def fit_workspace_bytes(d_in: int, d_out: int, r: int) -> int:
+    return int(load().lordba_fit_workspace_bytes(d_in, d_out, r))
+
+
+def fit_scales(target, packed_A, packed_B, s_in, s_r, s_out, r: int, sweeps: int = 1, axes: int = FIT_ALL,
+               workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Closed-form scale sweeps (s_in, then s_r, then s_out) against the dense float32 target
+    (d_in x d_out, rows contiguous) with the packed carriers fixed; the three scale tensors are
+    updated in place.  workspace: a uint8 CUDA tensor of fit_workspace_bytes(), made here if absent."""
+    _need_cuda(target, packed_A, packed_B, s_in, s_r, s_out)
+    if target.dtype != torch.float32 or target.dim() != 2 or (target.shape[1] > 1 and target.stride(1) != 1):
+        raise ValueError("target must be a 2-D float32 tensor with contiguous rows")
+    d_in, d_out = target.shape
+    for s, n in ((s_in, d_in), (s_r, r), (s_out, d_out)):
+        if s.dtype != torch.float32 or not s.is_contiguous() or s.numel() != n:
+            raise ValueError("scales must be contiguous float32 vectors of d_in, r and d_out entries")
+    if packed_A.numel() != packed_words(r, d_in, 0) or packed_B.numel() != packed_words(d_out, r, 1):
+        raise ValueError("packed carrier sizes do not match (r, d_in, d_out)")
+    need = fit_workspace_bytes(d_in, d_out, r)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=target.device)
+    ld = target.stride(0) if d_in > 1 else max(d_out, target.stride(0))
+    rc = load().lordba_fit_scales(target.data_ptr(), ld, packed_A.data_ptr(), packed_B.data_ptr(), s_in.data_ptr(),
+                                  s_r.data_ptr(), s_out.data_ptr(), d_in, d_out, r, sweeps, axes,
+                                  workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(rc, "lordba_fit_scales")
 
 
 def adapter_bits(d_in: int, d_out: int, r: int, ell: int = 1) -> int:

@@ -925,6 +925,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 // every size from 8 to 4096 tokens: an MMA costs the same with 14 or 16 live rows,
                 // and fewer, fuller CTAs leave room for the neighbouring calls' CTAs.
                 const int64_t rows = kTile;
+                const bool overlaps_neighbours = (*launches == 0) ? all_overlap : batch_checked;
                 int64_t tiles = 0, all_tiles = 0;      // widest projection (grid.x), and the sum
                 for (int k = 0; k < m; ++k) {
                     const int64_t tk = (sel_T[k] + rows - 1) / rows;
@@ -939,7 +940,6 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 // wave of tiles, or a call that may overlap its neighbours.  One's start-up and
                 // first-load latency then hide behind the other's streaming.  A lone single-wave
                 // call keeps one CTA with 16 consumer warps per SM.
-                const bool overlaps_neighbours = (*launches == 0) ? all_overlap : batch_checked;
                 const int nw = (all_tiles > sms || overlaps_neighbours) ? 8 : kMaxWarps;
                 const int max_chunk = nw * kGroup;
                 const int smem_budget = (nw == kMaxWarps) ? kSmemBudget : kSmemBudgetHalf;

@@ -399,20 +399,65 @@ def _ell_inputs(d_in, d_out, r, T, dtype, ell, seed):
     return base, s_in, s_r, s_out
 
 
+ELL_SHAPES = [
+    # T, d_in, d_out, r, ell
+    (70, 256, 192, 8, 2), (300, 1024, 768, 16, 2), (33, 200, 136, 24, 3), (150, 4096, 1024, 16, 4),
+    (2048, 4096, 4096, 16, 2),
+    # every envelope count the streaming kernel takes in one pass (ell * padded rank <= 64) ...
+    (200, 1024, 768, 4, 2), (130, 512, 1024, 8, 8), (90, 1024, 512, 16, 3), (300, 768, 1024, 8, 5),
+    (100, 1024, 768, 12, 3), (2048, 4096, 4096, 4, 2), (2048, 4096, 4096, 16, 4),
+    # ... and in several passes over x (ell * padded rank > 64)
+    (300, 1024, 1024, 32, 4), (64, 512, 512, 64, 2), (200, 1024, 1024, 32, 8), (100, 512, 512, 64, 8),
+    (150, 1024, 512, 20, 5), (77, 512, 1024, 40, 3),
+]
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
-@pytest.mark.parametrize("T,d_in,d_out,r,ell", [(70, 256, 192, 8, 2), (300, 1024, 768, 16, 2), (33, 200, 136, 24, 3),
-                                                (150, 4096, 1024, 16, 4), (2048, 4096, 4096, 16, 2)])
+@pytest.mark.parametrize("T,d_in,d_out,r,ell", ELL_SHAPES)
 def test_multi_envelope_forward(oracle, dtype, T, d_in, d_out, r, ell):
     if dtype != "bf16" and T > 1000:
         pytest.skip("full-size case is checked in bf16 only")
     base, s_in, s_r, s_out = _ell_inputs(d_in, d_out, r, T, dtype, ell, seed=90 + ell + r)
     d = DeviceProj(base)
     dev = d.x.device
-    lordba.adapter_forward_ell(d.x, d.packed_A, d.packed_B, torch.from_numpy(s_in).to(dev),
-                               torch.from_numpy(s_r).to(dev), torch.from_numpy(s_out).to(dev), d.y, r)
+    t_in, t_r, t_out = (torch.from_numpy(v).to(dev) for v in (s_in, s_r, s_out))
+    if dtype != "f32" and d_in % 64 == 0 and d_out % 64 == 0:
+        # every envelope count and rank runs on the tensor cores
+        p = lordba.make_proj(d.x, d.packed_A, d.packed_B, t_in, t_r, t_out, d.y, r)
+        assert lordba.query_variant([p], T, lordba.BF16 if dtype == "bf16" else lordba.F16) == [lordba.VARIANT_MMA]
+    lordba.adapter_forward_ell(d.x, d.packed_A, d.packed_B, t_in, t_r, t_out, d.y, r)
     want = oracle.adapter_forward_ell(base.x_f64(), base.A_sign, base.B_sign, s_in.astype(np.float64),
                                       s_r.astype(np.float64), s_out.astype(np.float64), base.y_f64())
-    assert_close(torch_to_f64(d.y), want, dtype, "ell=%d %s" % (ell, dtype))
+    assert_close(torch_to_f64(d.y), want, dtype, "ell=%d r=%d %s" % (ell, r, dtype))
+
+
+def test_multi_envelope_batched_with_mixed_envelope_counts(oracle):
+    """One batched call whose projections differ in envelope count and rank: one launch per kind,
+    every element against the oracle; and the zero-envelope embedding (an extra envelope with
+    zero rank scales changes nothing, Eq. iota-embed)."""
+    T = 150
+    specs = [(1024, 512, 16, 1), (1024, 512, 16, 3), (512, 768, 8, 8), (768, 1024, 32, 2), (512, 512, 64, 3)]
+    devs, wants, keep = [], [], []
+    for i, (d_in, d_out, r, ell) in enumerate(specs):
+        base, s_in, s_r, s_out = _ell_inputs(d_in, d_out, r, T, "bf16", ell, seed=700 + i)
+        d = DeviceProj(base)
+        ts = [torch.from_numpy(v if ell > 1 else v[0]).to(d.x.device) for v in (s_in, s_r, s_out)]
+        keep.append(ts)
+        devs.append((d, lordba.make_proj(d.x, d.packed_A, d.packed_B, ts[0], ts[1], ts[2], d.y, r)))
+        wants.append(oracle.adapter_forward_ell(base.x_f64(), base.A_sign, base.B_sign, s_in.astype(np.float64),
+                                                s_r.astype(np.float64), s_out.astype(np.float64), base.y_f64()))
+    n0 = lordba.launch_count()
+    lordba.adapter_forward_batched([p for _, p in devs], T, lordba.BF16)
+    assert lordba.launch_count() - n0 == len(specs)
+    for (d, _), want, spec in zip(devs, wants, specs):
+        assert_close(torch_to_f64(d.y), want, "bf16", "mixed envelope counts %s" % (spec,))
+    base, s_in, s_r, s_out = _ell_inputs(1024, 768, 16, 200, "bf16", 2, seed=720)
+    a, b = DeviceProj(base), DeviceProj(base)
+    t = lambda v: torch.from_numpy(np.ascontiguousarray(v)).to(a.x.device)
+    pad = lambda v: np.concatenate([v, np.zeros_like(v[:1])]) if v.shape[1] == 16 else np.concatenate([v, np.ones_like(v[:1])])
+    lordba.adapter_forward_ell(a.x, a.packed_A, a.packed_B, t(s_in), t(s_r), t(s_out), a.y, 16)
+    lordba.adapter_forward_ell(b.x, b.packed_A, b.packed_B, t(pad(s_in)), t(pad(s_r)), t(pad(s_out)), b.y, 16)
+    assert torch.equal(a.y, b.y)
 
 
 def test_multi_envelope_with_one_envelope_equals_plain_call(oracle):

@@ -276,8 +276,13 @@ def time_regions(gs: GraphSteps, steps: int, warmup: int, repeats: int):
     return np.array([a.elapsed_time(b) for a, b in ev])
 
 
+FIXED_REPEATS = None      # --repeats: a fixed repeat count (short runs under a profiler)
+
+
 def timed(gs: GraphSteps, steps: int, warmup: int, min_repeats: int = MIN_REPEATS, min_busy_s: float = MIN_BUSY_S):
     """Probe the region once to size the repeat count, then time it.  Returns the per-region ms."""
+    if FIXED_REPEATS:
+        return time_regions(gs, steps, warmup, FIXED_REPEATS)
     probe = time_regions(gs, steps, warmup, 3)
     region_s = float(np.median(probe)) * 1e-3 * (1.0 + warmup / max(1, steps))
     return time_regions(gs, steps, warmup, repeats_for(region_s, min_repeats, min_busy_s))
@@ -518,8 +523,11 @@ def run_gpu(args):
         n0 = lordba.launch_count()
         gs.graph(n_sets)
         launches_per_step = (lordba.launch_count() - n0) / n_sets
-        probe = time_regions(gs, args.steps, args.warmup, 3)
-        repeats = repeats_for(float(np.median(probe)) * 1e-3 * (1.0 + args.warmup / args.steps))
+        if FIXED_REPEATS:
+            repeats = FIXED_REPEATS
+        else:
+            probe = time_regions(gs, args.steps, args.warmup, 3)
+            repeats = repeats_for(float(np.median(probe)) * 1e-3 * (1.0 + args.warmup / args.steps))
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
@@ -789,6 +797,9 @@ def main():
     ap.add_argument("--traffic", type=float, default=NCU_DRAM_BYTES_PER_LAUNCH,
                     help="ncu DRAM bytes per launch to report in roofline.traffic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--repeats", type=int, default=None,
+                    help="repeat every timed region exactly this often (default: at least 30 and until the GPU "
+                         "has been busy for about 60 ms); a small number keeps a run under a profiler short")
     ap.add_argument("--no-workloads", action="store_true",
                     help="headline only: skip the `workloads` key (configs 2 to 4 and the widened rows)")
     ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full", "multi", "lora-dense"],
@@ -807,6 +818,8 @@ def main():
     ap.add_argument("--no-overlap", action="store_true",
                     help="every step waits for the previous one to finish (no LORDBA_PROJ_OVERLAP)")
     args = ap.parse_args()
+    global FIXED_REPEATS
+    FIXED_REPEATS = args.repeats if args.repeats and args.repeats > 0 else None
     headline = not (args.workload != "attn" or args.ell != 1 or args.rank != R or args.tokens != T or
                     args.dtype != "bf16" or args.scales_f16)
     if args.impl == "reference" or headline or args.workload == "lora-dense":

@@ -50,7 +50,12 @@ int FamilySelector::family(const lordba_proj &p, int64_t rows) const
     if (rows <= 0) return 0;
     if (variant == LORDBA_VARIANT_FMA || dtype == LORDBA_F32) return LORDBA_VARIANT_FMA;
     if (use_tc) return tc_supported(p, rows, dtype) ? LORDBA_VARIANT_TC : LORDBA_VARIANT_FMA;
-    return mma_supported(p, rows, dtype) ? LORDBA_VARIANT_MMA : LORDBA_VARIANT_FMA;
+    if (mma_supported(p, rows, dtype)) return LORDBA_VARIANT_MMA;
+    // Left to itself the library also gives the tcgen05 kernel what the streaming kernel cannot take
+    // but it can (widths that are not multiples of 64), from one 128-token tile up: a fifth to a
+    // half of the roofline there instead of the CUDA-core kernel's tenth.
+    if (variant == LORDBA_VARIANT_AUTO && rows >= 128 && tc_supported(p, rows, dtype)) return LORDBA_VARIANT_TC;
+    return LORDBA_VARIANT_FMA;
 }
 
 int launch_record(const LaunchRec &rec, const void *arg0, const void *arg1, cudaStream_t stream)

@@ -630,9 +630,14 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                             }
                         }
                     }
-#pragma unroll 2
-                    for (int env = 0; env < ell; ++env) {
-                        if (ell > 1) load_z(env, zh, zl);
+                    // the envelopes in runs of EG whose bodies are unrolled (a single run when all of
+                    // them fit one pass of the first product)
+                    for (int eb = 0; eb < ell; eb += EG)
+#pragma unroll
+                    for (int ei = 0; ei < EG; ++ei) {
+                        const int env = eb + ei;
+                        if (EGT != 1 && env >= ell) break;
+                        if (EGT != 1) load_z(env, zh, zl);
                         float c[4][4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)

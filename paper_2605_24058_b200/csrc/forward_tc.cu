@@ -1045,7 +1045,7 @@ bool tc_supported(const lordba_proj &p, int64_t T, int dtype)
 int launch_forward_tc(const lordba_proj *projs, const int64_t *tokens, int64_t T, int n, const FamilySelector &fsel,
                       LaunchSink &sink, bool batch_checked, int *launches)
 {
-    if (n == 0 || !fsel.use_tc) return LORDBA_OK;
+    if (n == 0) return LORDBA_OK;
     const int dtype = fsel.dtype;
     if (dtype != LORDBA_BF16 && dtype != LORDBA_F16) return LORDBA_OK;
     int *status = nullptr;

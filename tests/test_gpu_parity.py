@@ -657,7 +657,7 @@ def test_f16_mixed_scale_kinds_on_the_tcgen05_kernel(oracle):
 
 # ---------------------------------------------------------------- prepared calls and the kernel query
 
-@pytest.mark.parametrize("kind", ["layer_r16", "layer_r64", "segments_r16", "mixed_fma"])
+@pytest.mark.parametrize("kind", ["layer_r16", "layer_r64", "segments_r16", "mixed_families"])
 def test_planned_call_equals_plain_call(oracle, kind):
     """lordba_plan_init + lordba_adapter_forward_planned launch what the plain call launches: the
     same number of kernels, bit-identical y, and y matches the oracle; a plan can be replayed."""
@@ -674,8 +674,11 @@ def test_planned_call_equals_plain_call(oracle, kind):
         projs = [workloads.make_projection(1024, 768, 16, T, "bf16", seed=8200 + i) for i in range(3)]
         tokens = [T, 0, 77]
     else:
-        # one projection the tensor-core kernels cannot take (odd width) next to one they can
+        # three kernel families in one call: widths that are not multiples of 64 (the tcgen05 kernel
+        # takes them from 128 tokens up), a row pitch of 1001 elements (only the CUDA-core kernel),
+        # and a shape for the streaming kernel
         projs = [workloads.make_projection(1000, 520, 16, T, "bf16", seed=8300),
+                 workloads.make_projection(1001, 520, 16, T, "bf16", seed=8302),
                  workloads.make_projection(1024, 512, 16, T, "bf16", seed=8301)]
         tokens = T
     a = [DeviceProj(p) for p in projs]
@@ -683,8 +686,8 @@ def test_planned_call_equals_plain_call(oracle, kind):
     fams = lordba.query_variant([d.proj() for d in a], tokens, lordba.BF16)
     if kind == "layer_r64":
         assert set(fams) == {lordba.VARIANT_TC}
-    if kind == "mixed_fma":
-        assert fams == [lordba.VARIANT_FMA, lordba.VARIANT_MMA]
+    if kind == "mixed_families":
+        assert fams == [lordba.VARIANT_TC, lordba.VARIANT_FMA, lordba.VARIANT_MMA]
     if kind == "segments_r16":
         assert fams == [lordba.VARIANT_MMA, 0, lordba.VARIANT_MMA]
     plan = lordba.plan_init([d.proj() for d in b], tokens, lordba.BF16)
@@ -724,6 +727,10 @@ def test_query_variant_shows_the_fallbacks():
     assert lordba.query_variant([ok.proj()], T, lordba.BF16) == [lordba.VARIANT_MMA]
     assert lordba.query_variant([f32.proj()], T, lordba.F32) == [lordba.VARIANT_FMA]
     assert lordba.query_variant([odd.proj(), pitch.proj()], T, lordba.BF16) == [lordba.VARIANT_FMA] * 2
+    # from one 128-token tile up the tcgen05 kernel takes the odd width; the odd pitch stays where it is
+    odd2 = DeviceProj(workloads.make_projection(1000, 512, 16, 256, "bf16", seed=3))
+    pitch2 = DeviceProj(workloads.make_projection(1024, 512, 16, 256, "bf16", seed=4), ldx=1024 + 3)
+    assert lordba.query_variant([odd2.proj(), pitch2.proj()], 256, lordba.BF16) == [lordba.VARIANT_TC, lordba.VARIANT_FMA]
     big = [DeviceProj(workloads.make_projection(1024, 512, 64, 1, "bf16", seed=5))]
     x = torch.zeros(4096, 1024, dtype=torch.bfloat16, device="cuda:0")
     y = torch.zeros(4096, 512, dtype=torch.bfloat16, device="cuda:0")

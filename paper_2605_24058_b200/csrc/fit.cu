@@ -19,8 +19,9 @@
 //     beta    = ((Gp o Gq))^+ h,   h_k = sum_i alpha_i B1[i,k] W[i,k]      (Eq. beta-gram, beta-pinv)
 //     gamma_j = <d_j, V[:,j]> / (d_j^T Gp d_j),   d_j = beta * B2[:,j]      (Eq. gamma-update)
 //
-// (a zero denominator gives 0, the minimum-norm solution).  The passes over T accumulate in
-// float32 (short per-lane runs, then a tree); everything of size r x r, the quotients and the
+// (a zero denominator gives 0, the minimum-norm solution).  The passes over T are float32 FMAs
+// against signed scales expanded once per chunk into shared memory (per-lane or per-thread runs,
+// then a tree or a fixed-order sum); everything of size r x r, the quotients and the
 // pseudo-inverse (cyclic Jacobi eigendecomposition, eigenvalues below r eps lambda_max dropped)
 // are float64.  All reductions run in a fixed order: results are deterministic.
 #include <cstring>
@@ -55,58 +56,95 @@ __device__ __forceinline__ uint64_t a_bits(const uint32_t *__restrict__ pa, int6
 {
     const uint32_t *blk = pa + (i >> 6) * (int64_t)r * 2 + ((i & 63) >> 5);
     const int b = (int)(i & 31);
+    // eight independent loads at a time: the r words are far apart in time only if they wait for
+    // one another
     uint64_t v = 0;
-    for (int k = 0; k < r; ++k) v |= (uint64_t)((__ldg(blk + 2 * k) >> b) & 1u) << k;
+    for (int k0 = 0; k0 < r; k0 += 8) {
+        uint32_t w[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = (k0 + i < r) ? __ldg(blk + 2 * (k0 + i)) : 0u;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v |= (uint64_t)((w[i] >> b) & 1u) << (k0 + i);
+    }
     return v;
 }
 
-__device__ __forceinline__ float signed_f(float v, uint64_t bits, int k)
-{
-    // +v when bit k is set, -v otherwise
-    return __uint_as_float(__float_as_uint(v) ^ ((uint32_t)(~(bits >> k) & 1ull) << 31));
-}
+// ---- W[i,k] = sum_j T[i,j] gamma_j B_sign[j,k] ----------------------------------------------
+// A CTA owns 8 * RB rows of T (a warp RB of them) and walks the columns 128 at a time: the chunk's
+// signed scales gamma_j B_sign[j,k] are expanded once into shared memory and serve every row, a lane
+// takes the columns lane, lane + 32, ... and keeps RB x RP partial sums, joined by a shuffle tree at
+// the end (fixed order).
+constexpr int kRowCols = 128;
 
-// ---- W[i,k] = sum_j T[i,j] gamma_j B_sign[j,k]: one warp per row of T ------------------------
-template <int RP>
+template <int RP, int RB>
 __global__ void __launch_bounds__(kFitThreads)
 fit_row_pass_kernel(const float *__restrict__ T, int64_t ld, const uint32_t *__restrict__ pb,
                     const float *__restrict__ gamma, int64_t d_in, int64_t d_out, int r, float *__restrict__ W)
 {
-    const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * (kFitThreads / 32) + (threadIdx.x >> 5);
-    if (row >= d_in) return;
+    constexpr int kStride = RP + 4;                    // floats per column: 16-byte reads without bank conflicts
+    __shared__ __align__(16) float S[kRowCols * kStride];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row0 = ((int64_t)blockIdx.x * (kFitThreads / 32) + warp) * RB;
     const int64_t n_words = (d_out * r + 31) / 32;
-    float acc[RP];
+    float acc[RB][RP];
 #pragma unroll
-    for (int k = 0; k < RP; ++k) acc[k] = 0.0f;
-    const float *trow = T + row * ld;
-    for (int64_t j = lane; j < d_out; j += 32) {
-        const float t = trow[j] * __ldg(gamma + j);
-        const uint64_t bits = b_bits(pb, n_words, j, r);
+    for (int b = 0; b < RB; ++b)
 #pragma unroll
-        for (int k = 0; k < RP; ++k) acc[k] += signed_f(t, bits, k);      // ranks >= r: unused
+        for (int k = 0; k < RP; ++k) acc[b][k] = 0.0f;
+    for (int64_t j0 = 0; j0 < d_out; j0 += kRowCols) {
+        __syncthreads();
+        if (threadIdx.x < kRowCols) {
+            const int64_t j = j0 + threadIdx.x;
+            const bool in = j < d_out;
+            const uint64_t bits = in ? b_bits(pb, n_words, j, r) : 0ull;
+            const float g = in ? __ldg(gamma + j) : 0.0f;
+#pragma unroll
+            for (int k = 0; k < RP; ++k)
+                S[threadIdx.x * kStride + k] = (k < r) ? (((bits >> k) & 1ull) ? g : -g) : 0.0f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int cc = 0; cc < kRowCols / 32; ++cc) {
+            const int c = cc * 32 + lane;
+            const int64_t j = j0 + c;
+            float t[RB];
+#pragma unroll
+            for (int b = 0; b < RB; ++b) t[b] = (row0 + b < d_in && j < d_out) ? T[(row0 + b) * ld + j] : 0.0f;
+#pragma unroll
+            for (int k4 = 0; k4 < RP / 4; ++k4) {
+                const float4 sv = *reinterpret_cast<const float4 *>(&S[c * kStride + 4 * k4]);
+#pragma unroll
+                for (int b = 0; b < RB; ++b) {
+                    acc[b][4 * k4] = fmaf(t[b], sv.x, acc[b][4 * k4]);
+                    acc[b][4 * k4 + 1] = fmaf(t[b], sv.y, acc[b][4 * k4 + 1]);
+                    acc[b][4 * k4 + 2] = fmaf(t[b], sv.z, acc[b][4 * k4 + 2]);
+                    acc[b][4 * k4 + 3] = fmaf(t[b], sv.w, acc[b][4 * k4 + 3]);
+                }
+            }
+        }
     }
 #pragma unroll
-    for (int k = 0; k < RP; ++k) {
+    for (int b = 0; b < RB; ++b)
 #pragma unroll
-        for (int s = 16; s >= 1; s >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], s);
-    }
-    if (lane == 0) {
+        for (int k = 0; k < RP; ++k) {
+            float v = acc[b][k];
 #pragma unroll
-        for (int k = 0; k < RP; ++k)
-            if (k < r) W[row * r + k] = acc[k];
-    }
+            for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+            if (lane == 0 && k < r && row0 + b < d_in) W[(row0 + b) * r + k] = v;
+        }
 }
 
 // ---- V[c][k][j] = sum over the rows i of chunk c of alpha_i A_sign[k,i] T[i,j] ---------------
+// A thread owns one column of T; the signed scales alpha_i A_sign[k,i] of 64 rows at a time (one
+// block of the A carrier) are expanded once into shared memory and read by every thread at the
+// same address (a broadcast).
 template <int RP>
 __global__ void __launch_bounds__(kColsPerBlock)
 fit_col_pass_kernel(const float *__restrict__ T, int64_t ld, const uint32_t *__restrict__ pa,
                     const float *__restrict__ alpha, int64_t d_in, int64_t d_out, int r, int64_t rows_per_chunk,
                     float *__restrict__ Vpart)
 {
-    __shared__ uint64_t rowbits[64];
-    __shared__ float arow[64];
+    __shared__ __align__(16) float S[64 * RP];
     const int64_t j = (int64_t)blockIdx.x * kColsPerBlock + threadIdx.x;
     const int64_t i_begin = (int64_t)blockIdx.y * rows_per_chunk;
     const int64_t i_end = (i_begin + rows_per_chunk < d_in) ? i_begin + rows_per_chunk : d_in;
@@ -117,17 +155,26 @@ fit_col_pass_kernel(const float *__restrict__ T, int64_t ld, const uint32_t *__r
         __syncthreads();
         if (threadIdx.x < 64) {
             const int64_t i = i0 + threadIdx.x;
-            rowbits[threadIdx.x] = (i < i_end) ? a_bits(pa, i, r) : 0ull;
-            arow[threadIdx.x] = (i < i_end) ? __ldg(alpha + i) : 0.0f;
+            const bool in = i < i_end;
+            const uint64_t bits = in ? a_bits(pa, i, r) : 0ull;
+            const float a = in ? __ldg(alpha + i) : 0.0f;
+#pragma unroll
+            for (int k = 0; k < RP; ++k) S[threadIdx.x * RP + k] = (k < r) ? (((bits >> k) & 1ull) ? a : -a) : 0.0f;
         }
         __syncthreads();
         const int n = (int)((i_end - i0 < 64) ? (i_end - i0) : 64);
         if (j < d_out) {
+#pragma unroll 4
             for (int il = 0; il < n; ++il) {
-                const float t = T[(i0 + il) * ld + j] * arow[il];
-                const uint64_t bits = rowbits[il];
+                const float t = T[(i0 + il) * ld + j];
 #pragma unroll
-                for (int k = 0; k < RP; ++k) acc[k] += signed_f(t, bits, k);
+                for (int k4 = 0; k4 < RP / 4; ++k4) {
+                    const float4 sv = *reinterpret_cast<const float4 *>(&S[il * RP + 4 * k4]);
+                    acc[4 * k4] = fmaf(t, sv.x, acc[4 * k4]);
+                    acc[4 * k4 + 1] = fmaf(t, sv.y, acc[4 * k4 + 1]);
+                    acc[4 * k4 + 2] = fmaf(t, sv.z, acc[4 * k4 + 2]);
+                    acc[4 * k4 + 3] = fmaf(t, sv.w, acc[4 * k4 + 3]);
+                }
             }
         }
     }
@@ -225,21 +272,13 @@ fit_gamma_kernel(const uint32_t *__restrict__ pb, const float *__restrict__ Vpar
     gamma[j] = den > 0.0 ? (float)(num / den) : 0.0f;
 }
 
-// ---- beta = (Gp o Gq)^+ h, h_k = sum_i alpha_i B1[i,k] W[i,k] (Eq. beta-gram, Eq. beta-pinv): one CTA
-// Shared memory (dynamic): A and E, n x n doubles each (n = r rounded up to even), then
-// cs (n doubles), h (64), partial sums (threads / 32 x 64), eigen-coefficients (64).
+// ---- h_k = sum_i alpha_i B1[i,k] W[i,k] (Eq. beta-gram): one CTA, fixed-order tree --------------
 __global__ void __launch_bounds__(kFitThreads)
-fit_beta_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, const float *__restrict__ alpha,
-                const double *__restrict__ Gp, const double *__restrict__ Gq, int64_t d_in, int r,
-                float *__restrict__ beta)
+fit_h_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, const float *__restrict__ alpha,
+             int64_t d_in, int r, double *__restrict__ h)
 {
-    extern __shared__ double sh[];
-    const int n = (r + 1) & ~1;
-    double *A = sh, *E = A + n * n, *cs = E + n * n, *h = cs + 2 * 64, *red = h + 64, *coef = red + (kFitThreads / 32) * 64;
-    __shared__ double off_norm, all_norm;
+    __shared__ double red[(kFitThreads / 32) * 64];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    // h: rows strided over the threads, fixed-order tree
     double acc[64];
 #pragma unroll
     for (int k = 0; k < 64; ++k) acc[k] = 0.0;
@@ -257,31 +296,59 @@ fit_beta_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, co
         for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
         if (lane == 0) red[warp * 64 + k] = v;
     }
-    for (int e = tid; e < n * n; e += kFitThreads) {
-        const int p = e / n, q = e - p * n;
-        A[e] = (p < r && q < r) ? Gp[p * r + q] * Gq[p * r + q] : 0.0;     // Eq. beta-Schur
-        E[e] = (p == q) ? 1.0 : 0.0;
-    }
     __syncthreads();
-    if (tid < 64) {
+    if (tid < r) {
         double v = 0.0;
         for (int w = 0; w < kFitThreads / 32; ++w) v += red[w * 64 + tid];
-        h[tid] = (tid < r) ? v : 0.0;
+        h[tid] = v;
     }
+}
+
+// ---- beta = (Gp o Gq)^+ h (Eq. beta-Schur, Eq. beta-pinv): one CTA of 1024 threads ----------------
+// Shared memory (dynamic): A and E, n rows of n + 1 doubles each (n = r rounded up to even), then the
+// rotations of a round (2 x 64), h (64), the eigen-coefficients (64) and 2 x 32 partial norms.
+constexpr int kBetaThreads = 1024;
+
+__global__ void __launch_bounds__(kBetaThreads)
+fit_beta_kernel(const double *__restrict__ Gp, const double *__restrict__ Gq, const double *__restrict__ hvec, int r,
+                float *__restrict__ beta)
+{
+    extern __shared__ double sh[];
+    const int n = (r + 1) & ~1;
+    const int ns = n + 1;        // padded row length: column walks without bank conflicts
+    double *A = sh, *E = A + n * ns, *cs = E + n * ns, *h = cs + 2 * 64, *coef = h + 64, *part = coef + 64;
+    __shared__ double off_norm, all_norm;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    for (int e = tid; e < n * n; e += kBetaThreads) {
+        const int p = e / n, q = e - p * n;
+        A[p * ns + q] = (p < r && q < r) ? Gp[p * r + q] * Gq[p * r + q] : 0.0;     // Eq. beta-Schur
+        E[p * ns + q] = (p == q) ? 1.0 : 0.0;
+    }
+    if (tid < 64) h[tid] = (tid < r) ? hvec[tid] : 0.0;
     __syncthreads();
 
     // cyclic Jacobi, n / 2 disjoint rotations per round (round-robin pairing), at most 40 sweeps
     for (int sweep = 0; sweep < 40; ++sweep) {
+        double off = 0.0, all = 0.0;
+        for (int e = tid; e < n * n; e += kBetaThreads) {
+            const int p = e / n, q = e - p * n;
+            const double v = A[p * ns + q] * A[p * ns + q];
+            all += v;
+            if (p != q) off += v;
+        }
+#pragma unroll
+        for (int s = 16; s >= 1; s >>= 1) {
+            off += __shfl_xor_sync(0xffffffffu, off, s);
+            all += __shfl_xor_sync(0xffffffffu, all, s);
+        }
+        if (lane == 0) { part[warp] = off; part[32 + warp] = all; }
+        __syncthreads();
         if (tid == 0) {
-            double off = 0.0, all = 0.0;
-            for (int p = 0; p < n; ++p)
-                for (int q = 0; q < n; ++q) {
-                    const double v = A[p * n + q] * A[p * n + q];
-                    all += v;
-                    if (p != q) off += v;
-                }
-            off_norm = off;
-            all_norm = all;
+            double o = 0.0, a = 0.0;
+            for (int w = 0; w < kBetaThreads / 32; ++w) { o += part[w]; a += part[32 + w]; }
+            off_norm = o;
+            all_norm = a;
         }
         __syncthreads();
         if (off_norm <= 1e-30 * all_norm) break;
@@ -289,12 +356,12 @@ fit_beta_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, co
             // pair m of this round: (n-1, round) for m = 0, else ((round+m) % (n-1), (round-m) mod (n-1))
             if (tid < n / 2) {
                 const int m = tid;
-                int p = (m == 0) ? n - 1 : (round + m) % (n - 1);
-                int q = (m == 0) ? round : (round - m + (n - 1)) % (n - 1);
-                const double apq = A[p * n + q];
+                const int p = (m == 0) ? n - 1 : (round + m) % (n - 1);
+                const int q = (m == 0) ? round : (round - m + (n - 1)) % (n - 1);
+                const double apq = A[p * ns + q];
                 double c = 1.0, s = 0.0;
                 if (apq != 0.0) {
-                    const double theta = (A[q * n + q] - A[p * n + p]) / (2.0 * apq);
+                    const double theta = (A[q * ns + q] - A[p * ns + p]) / (2.0 * apq);
                     const double t = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
                     c = 1.0 / sqrt(t * t + 1.0);
                     s = t * c;
@@ -304,28 +371,28 @@ fit_beta_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, co
             }
             __syncthreads();
             // columns: A <- A J, E <- E J (task = row t, pair m)
-            for (int task = tid; task < n * (n / 2); task += kFitThreads) {
+            for (int task = tid; task < n * (n / 2); task += kBetaThreads) {
                 const int t = task / (n / 2), m = task - t * (n / 2);
                 const int p = (m == 0) ? n - 1 : (round + m) % (n - 1);
                 const int q = (m == 0) ? round : (round - m + (n - 1)) % (n - 1);
                 const double c = cs[2 * m], s = cs[2 * m + 1];
-                const double ap = A[t * n + p], aq = A[t * n + q];
-                A[t * n + p] = c * ap - s * aq;
-                A[t * n + q] = s * ap + c * aq;
-                const double ep = E[t * n + p], eq = E[t * n + q];
-                E[t * n + p] = c * ep - s * eq;
-                E[t * n + q] = s * ep + c * eq;
+                const double ap = A[t * ns + p], aq = A[t * ns + q];
+                A[t * ns + p] = c * ap - s * aq;
+                A[t * ns + q] = s * ap + c * aq;
+                const double ep = E[t * ns + p], eq = E[t * ns + q];
+                E[t * ns + p] = c * ep - s * eq;
+                E[t * ns + q] = s * ep + c * eq;
             }
             __syncthreads();
             // rows: A <- J^T A (task = column t, pair m)
-            for (int task = tid; task < n * (n / 2); task += kFitThreads) {
+            for (int task = tid; task < n * (n / 2); task += kBetaThreads) {
                 const int t = task / (n / 2), m = task - t * (n / 2);
                 const int p = (m == 0) ? n - 1 : (round + m) % (n - 1);
                 const int q = (m == 0) ? round : (round - m + (n - 1)) % (n - 1);
                 const double c = cs[2 * m], s = cs[2 * m + 1];
-                const double ap = A[p * n + t], aq = A[q * n + t];
-                A[p * n + t] = c * ap - s * aq;
-                A[q * n + t] = s * ap + c * aq;
+                const double ap = A[p * ns + t], aq = A[q * ns + t];
+                A[p * ns + t] = c * ap - s * aq;
+                A[q * ns + t] = s * ap + c * aq;
             }
             __syncthreads();
         }
@@ -334,20 +401,20 @@ fit_beta_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, co
     // beta = sum over eigenpairs with lambda > r eps lambda_max of (v^T h / lambda) v
     if (tid == 0) {
         double lmax = 0.0;
-        for (int k = 0; k < n; ++k) lmax = fmax(lmax, A[k * n + k]);
+        for (int k = 0; k < n; ++k) lmax = fmax(lmax, A[k * ns + k]);
         off_norm = (double)r * 2.220446049250313e-16 * lmax;
     }
     __syncthreads();
     if (tid < n) {
-        const double lam = A[tid * n + tid];
+        const double lam = A[tid * ns + tid];
         double dot = 0.0;
-        for (int p = 0; p < r; ++p) dot += E[p * n + tid] * h[p];
+        for (int p = 0; p < r; ++p) dot += E[p * ns + tid] * h[p];
         coef[tid] = (lam > off_norm) ? dot / lam : 0.0;
     }
     __syncthreads();
     if (tid < r) {
         double v = 0.0;
-        for (int k = 0; k < n; ++k) v += E[tid * n + k] * coef[k];
+        for (int k = 0; k < n; ++k) v += E[tid * ns + k] * coef[k];
         beta[tid] = (float)v;
     }
 }
@@ -358,6 +425,7 @@ struct FitWorkspace {
     float *W;          // d_in x r
     float *Vpart;      // chunks x r x d_out
     double *Gq, *Gp;   // r x r each
+    double *h;         // r
     int chunks;
     int64_t rows_per_chunk;
     size_t bytes;
@@ -377,6 +445,7 @@ FitWorkspace carve(void *base, int64_t d_in, int64_t d_out, int r)
     w.Vpart = reinterpret_cast<float *>(p + off); off += up((size_t)w.chunks * r * d_out * 4);
     w.Gq = reinterpret_cast<double *>(p + off); off += up((size_t)r * r * 8);
     w.Gp = reinterpret_cast<double *>(p + off); off += up((size_t)r * r * 8);
+    w.h = reinterpret_cast<double *>(p + off); off += up((size_t)r * 8);
     w.bytes = off;
     return w;
 }
@@ -384,15 +453,15 @@ FitWorkspace carve(void *base, int64_t d_in, int64_t d_out, int r)
 size_t beta_smem(int r)
 {
     const int n = (r + 1) & ~1;
-    return sizeof(double) * (size_t)(2 * n * n + 2 * 64 + 64 + (kFitThreads / 32) * 64 + 64);
+    return sizeof(double) * (size_t)(2 * n * (n + 1) + 2 * 64 + 64 + 64 + 64);
 }
 
-template <int RP>
+template <int RP, int RB>
 void launch_row(const float *T, int64_t ld, const uint32_t *pb, const float *gamma, int64_t d_in, int64_t d_out, int r,
                 float *W, cudaStream_t s)
 {
-    const int rows_per_block = kFitThreads / 32;
-    fit_row_pass_kernel<RP><<<(unsigned)((d_in + rows_per_block - 1) / rows_per_block), kFitThreads, 0, s>>>(
+    const int rows_per_block = (kFitThreads / 32) * RB;
+    fit_row_pass_kernel<RP, RB><<<(unsigned)((d_in + rows_per_block - 1) / rows_per_block), kFitThreads, 0, s>>>(
         T, ld, pb, gamma, d_in, d_out, r, W);
 }
 
@@ -422,10 +491,10 @@ int launch_fit_scales(const float *target, int64_t ld, const uint32_t *pa, const
         // rows of T through B2^T diag(gamma), and Q Q^T
         if (axes & (LORDBA_FIT_ALPHA | LORDBA_FIT_BETA)) {
             switch (rp) {
-                case 8:  launch_row<8>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
-                case 16: launch_row<16>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
-                case 32: launch_row<32>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
-                default: launch_row<64>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
+                case 8:  launch_row<8, 4>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
+                case 16: launch_row<16, 4>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
+                case 32: launch_row<32, 2>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
+                default: launch_row<64, 1>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
             }
             fit_gram_kernel<1><<<r, kFitThreads, 0, stream>>>(pb, s_out, d_out, r, b_words, w.Gq);
             count_launch(2);
@@ -440,8 +509,9 @@ int launch_fit_scales(const float *target, int64_t ld, const uint32_t *pa, const
             count_launch();
         }
         if (axes & LORDBA_FIT_BETA) {
-            fit_beta_kernel<<<1, kFitThreads, beta_smem(r), stream>>>(pa, w.W, s_in, w.Gp, w.Gq, d_in, r, s_r);
-            count_launch();
+            fit_h_kernel<<<1, kFitThreads, 0, stream>>>(pa, w.W, s_in, d_in, r, w.h);
+            fit_beta_kernel<<<1, kBetaThreads, beta_smem(r), stream>>>(w.Gp, w.Gq, w.h, r, s_r);
+            count_launch(2);
         }
         if (axes & LORDBA_FIT_GAMMA) {
             switch (rp) {

@@ -571,8 +571,16 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 zl[s][0] = l0.x; zl[s][1] = l1.x; zl[s][2] = l0.y; zl[s][3] = l1.y;
             }
         };
+        // z stays in registers across the items when all of it fits 16 of them: one envelope, or two
+        // at rank <= 16 (then EG = 2 means exactly two envelopes)
+        constexpr bool kZRes = (EGT == 2 && KS == 1);
         uint32_t zh[KS][4], zl[KS][4];
+        uint32_t zh2[KS][4], zl2[KS][4];           // (second envelope; unused unless kZRes)
         if (ell == 1) load_z(0, zh, zl);
+        if (kZRes) {
+            load_z(0, zh, zl);
+            load_z(1, zh2, zl2);
+        }
         // A wait that gave up during the first product left u incomplete: this CTA then writes
         // nothing (its rows of y keep their old values) and only drains its items.
         const bool u_complete = !__any_sync(0xffffffffu, *abort_flag != 0);
@@ -637,7 +645,10 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     for (int ei = 0; ei < EG; ++ei) {
                         const int env = eb + ei;
                         if (EGT != 1 && env >= ell) break;
-                        if (EGT != 1) load_z(env, zh, zl);
+                        if (EGT != 1 && !kZRes) load_z(env, zh, zl);
+                        // (resident z: envelope 0 in zh / zl, envelope 1 in zh2 / zl2)
+                        const uint32_t (*azh)[4] = (kZRes && ei == 1) ? zh2 : zh;
+                        const uint32_t (*azl)[4] = (kZRes && ei == 1) ? zl2 : zl;
                         float c[4][4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
@@ -655,10 +666,10 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                             }
 #pragma unroll
                             for (int i = 0; i < 4; ++i)
-                                mma_bf16(c[i], zh[ks][0], zh[ks][1], zh[ks][2], zh[ks][3], b0[i], b1[i]);
+                                mma_bf16(c[i], azh[ks][0], azh[ks][1], azh[ks][2], azh[ks][3], b0[i], b1[i]);
 #pragma unroll
                             for (int i = 0; i < 4; ++i)
-                                mma_bf16(c[i], zl[ks][0], zl[ks][1], zl[ks][2], zl[ks][3], b0[i], b1[i]);
+                                mma_bf16(c[i], azl[ks][0], azl[ks][1], azl[ks][2], azl[ks][3], b0[i], b1[i]);
                         }
                         const float4 *so4 = reinterpret_cast<const float4 *>(
                             slot + plan.off_scale + 4 * (env * cwy + gcol + 16 * q + 8 * cc));

@@ -231,6 +231,14 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1,
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// (d0, d1) += (a0, a1) * (b0, b1): one packed fp32 FMA, each half rounded like fmaf
+__device__ __forceinline__ void fma2(float &d0, float &d1, float a0, float a1, float b0, float b1)
+{
+    asm("{\n.reg .b64 ra, rb, rc;\nmov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %5};\nmov.b64 rc, {%0, %1};\n"
+        "fma.rn.f32x2 rc, ra, rb, rc;\nmov.b64 {%0, %1}, rc;\n}"
+        : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
@@ -679,8 +687,13 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                         for (int half = 0; half < 2; ++half)
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
-                                vs[half][2 * i] = fmaf(so[2 * i], c[i][2 * half], vs[half][2 * i]);
-                                vs[half][2 * i + 1] = fmaf(so[2 * i + 1], c[i][2 * half + 1], vs[half][2 * i + 1]);
+                                if (EGT != 1) {
+                                    // several envelopes: the packed form was measured ahead (7 % at two envelopes)
+                                    fma2(vs[half][2 * i], vs[half][2 * i + 1], so[2 * i], so[2 * i + 1], c[i][2 * half], c[i][2 * half + 1]);
+                                } else {
+                                    vs[half][2 * i] = fmaf(so[2 * i], c[i][2 * half], vs[half][2 * i]);
+                                    vs[half][2 * i + 1] = fmaf(so[2 * i + 1], c[i][2 * half + 1], vs[half][2 * i + 1]);
+                                }
                             }
                     }
 #pragma unroll

@@ -394,6 +394,42 @@ def time_workload(w: DeviceWorkload, stream, steps: int, warmup: int, min_repeat
             "step_dependency": "declared independent" if w.overlap_ok else "each call waits for the previous one"}
 
 
+def time_fit_sweep(lordba, dev, N, M, r, sweeps=10):
+    """One closed-form scale sweep of the adapter fit (lordba_fit_scales) on a dense N x M float32
+    target drawn on the device from the sign-plus-noise factor model, carriers at the latent signs:
+    microseconds per sweep (CUDA events around `sweeps` calls) against the time of reading the target
+    twice, which is what a sweep has to move."""
+    import torch
+    g = torch.Generator(device=dev)
+    g.manual_seed(77)
+    sA = torch.randint(0, 2, (N, r), device=dev, generator=g, dtype=torch.int8) * 2 - 1
+    sB = torch.randint(0, 2, (M, r), device=dev, generator=g, dtype=torch.int8) * 2 - 1
+    A = 0.05 * sA.float() + 0.01 * torch.randn(N, r, device=dev, generator=g)
+    B = 0.05 * sB.float() + 0.01 * torch.randn(M, r, device=dev, generator=g)
+    target = (A @ B.t()).contiguous()
+    pa = lordba.pack_signs(sA.t().contiguous(), 0)
+    pb = lordba.pack_signs(sB.contiguous(), 1)
+    s_in, s_r, s_out = torch.ones(N, device=dev), torch.ones(r, device=dev), torch.ones(M, device=dev)
+    ws = torch.empty(lordba.fit_workspace_bytes(N, M, r), dtype=torch.uint8, device=dev)
+    n0 = lordba.launch_count()
+    lordba.fit_scales(target, pa, pb, s_in, s_r, s_out, r, 1, lordba.FIT_ALL, ws)
+    launches = lordba.launch_count() - n0
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    lordba.fit_scales(target, pa, pb, s_in, s_r, s_out, r, sweeps, lordba.FIT_ALL, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    err = float(torch.linalg.norm(target - (s_in[:, None] * sA.float()) @ (s_r[:, None] * sB.float().t() * s_out[None, :])) /
+                torch.linalg.norm(target))
+    us = e0.elapsed_time(e1) * 1e3 / sweeps
+    peak, peak_kind = measured_peak()
+    alg = 2 * 4 * N * M
+    return {"us_per_sweep": us, "gbs": alg / (us * 1e-6) / 1e9, "frac": alg / (us * 1e-6) / 1e9 / peak,
+            "peak_kind": "of " + peak_kind, "alg_bytes": alg, "launches_per_sweep": launches,
+            "relative_residual_after": err, "note": "offline step; latency bound, not on the roofline"}
+
+
 def supplementary_workloads(lordba, dev, stream, sampler):
     """Configs 2 to 4 and the widened rows, each as {us_per_call, gbs, frac, variant, ...}."""
     import torch
@@ -437,6 +473,9 @@ def supplementary_workloads(lordba, dev, stream, sampler):
     for r in (8, 16, 32, 64):
         run("full_T2048_r%d" % r, 4, 2, shared=shared, min_repeats=8, min_busy_s=0.02, shapes=full, r=r, Tn=2048)
     shared.clear()
+    torch.cuda.empty_cache()
+    # the closed-form scale sweep of the adapter fit (not part of the forward path)
+    out["fit_sweep_4096x4096_r16"] = time_fit_sweep(lordba, dev, workloads.HIDDEN, workloads.HIDDEN, 16)
     torch.cuda.empty_cache()
     return out
 
@@ -787,6 +826,23 @@ def run_dense_lora_context(args):
     return 0
 
 
+def run_fit(args):
+    """lordba_fit_scales alone: one line with microseconds per sweep on a 4096 x 4096 target."""
+    import torch
+    from paper_2605_24058_b200 import lordba
+    torch.cuda.set_device(0)
+    ensure_library()
+    lordba.load()
+    res = time_fit_sweep(lordba, torch.device("cuda", 0), workloads.HIDDEN, workloads.HIDDEN, args.rank,
+                         sweeps=max(1, min(args.steps, 50)))
+    print(json.dumps({"metric": "closed-form scale sweep of the adapter fit, 4096 x 4096 float32 target, r=%d" % args.rank,
+                      "value": res["us_per_sweep"], "unit": "us per sweep", "higher_is_better": False,
+                      "roofline": {"bound": "hbm", "achieved": res["gbs"], "unit": "GB/s", "frac": res["frac"],
+                                   "peak_kind": res["peak_kind"], "algorithmic_bytes_per_launch": res["alg_bytes"]},
+                      "config": {"workload": "fit", "rank": args.rank}, "detail": res}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -804,7 +860,7 @@ def main():
                          "has been busy for about 60 ms); a small number keeps a run under a profiler short")
     ap.add_argument("--no-workloads", action="store_true",
                     help="headline only: skip the `workloads` key (configs 2 to 4 and the widened rows)")
-    ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full", "multi", "lora-dense"],
+    ap.add_argument("--workload", default="attn", choices=["attn", "gate", "down", "layer", "decode", "full", "multi", "lora-dense", "fit"],
                     help="attn = the headline configuration (default); the others time one supplementary "
                          "workload alone: one MLP projection, a layer's seven projections in one batched call "
                          "(prefill, or decode with --tokens 1..64), or all 224 projections in one call")
@@ -836,6 +892,8 @@ def main():
         return run_reference(args)
     if args.workload == "lora-dense":
         return run_dense_lora_context(args)
+    if args.workload == "fit":
+        return run_fit(args)
     if not headline:
         return run_workload(args)
     return run_gpu(args)

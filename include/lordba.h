@@ -111,7 +111,9 @@ typedef struct lordba_proj {
  * LORDBA_PROJ_ELL(ell) in its flags, 1 <= ell <= LORDBA_MAX_ELL, takes s_in as ell x d_in,
  * s_r as ell x r and s_out as ell x d_out (row-major, envelope e in row e), and the call adds
  *     sum_e  s_out[e] * ( B_sign ( s_r[e] * ( A_sign ( s_in[e] * x[t,:] ) ) ) )
- * to y[t,:] with one rounding.  Flags without this field mean ell = 1.
+ * to y[t,:] with one rounding.  Flags without this field mean ell = 1.  Every envelope count at
+ * every rank runs on the tensor cores (streaming kernel); the cost is about that of one envelope
+ * at rank ell * r.
  */
 #define LORDBA_MAX_ELL 8
 #define LORDBA_PROJ_ELL(ell) ((((ell) - 1) & 0xf) << 8)

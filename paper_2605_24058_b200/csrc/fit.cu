@@ -34,6 +34,7 @@ namespace {
 constexpr int kFitThreads = 256;
 constexpr int kColsPerBlock = 128;      // columns of T per CTA of the column pass
 constexpr int kMaxRowChunks = 16;       // partial sums of the column pass
+constexpr int kParts = 8;               // partial sums of the Gram matrices and of h (added in a fixed order by their readers)
 
 // r sign bits of row j of B_sign (role-1 stream: bit j*r + k), bit 1 = +1
 __device__ __forceinline__ uint64_t b_bits(const uint32_t *__restrict__ pb, int64_t n_words, int64_t j, int r)
@@ -71,17 +72,20 @@ __device__ __forceinline__ uint64_t a_bits(const uint32_t *__restrict__ pa, int6
 
 // ---- W[i,k] = sum_j T[i,j] gamma_j B_sign[j,k] ----------------------------------------------
 // A CTA owns 8 * RB rows of T (a warp RB of them) and walks the columns 128 at a time: the chunk's
-// signed scales gamma_j B_sign[j,k] are expanded once into shared memory and serve every row, a lane
-// takes the columns lane, lane + 32, ... and keeps RB x RP partial sums, joined by a shuffle tree at
-// the end (fixed order).
+// signed scales gamma_j B_sign[j,k] are expanded once into shared memory and serve every row; a
+// lane takes four consecutive columns (one 16-byte load per row when the rows allow it) and keeps
+// RB x RP partial sums, joined by a shuffle tree at the end (fixed order).
 constexpr int kRowCols = 128;
 
 template <int RP, int RB>
 __global__ void __launch_bounds__(kFitThreads)
 fit_row_pass_kernel(const float *__restrict__ T, int64_t ld, const uint32_t *__restrict__ pb,
-                    const float *__restrict__ gamma, int64_t d_in, int64_t d_out, int r, float *__restrict__ W)
+                    const float *__restrict__ gamma, int64_t d_in, int64_t d_out, int r, int vec4,
+                    float *__restrict__ W)
 {
     constexpr int kStride = RP + 4;                    // floats per column: 16-byte reads without bank conflicts
+    // column c of the chunk sits at slot (c % 4) * 32 + c / 4, so that the four columns of lane l are
+    // the slots l, 32 + l, 64 + l, 96 + l: consecutive lanes read consecutive slots
     __shared__ __align__(16) float S[kRowCols * kStride];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t row0 = ((int64_t)blockIdx.x * (kFitThreads / 32) + warp) * RB;
@@ -92,33 +96,44 @@ fit_row_pass_kernel(const float *__restrict__ T, int64_t ld, const uint32_t *__r
 #pragma unroll
         for (int k = 0; k < RP; ++k) acc[b][k] = 0.0f;
     for (int64_t j0 = 0; j0 < d_out; j0 += kRowCols) {
+        // this chunk's rows of T first: the loads fly while the signs are expanded
+        float t[RB][4];
+        const int64_t jl = j0 + 4 * lane;
+#pragma unroll
+        for (int b = 0; b < RB; ++b) {
+            const bool row_ok = row0 + b < d_in;
+            if (vec4 && row_ok && jl + 4 <= d_out) {
+                const float4 v = __ldcs(reinterpret_cast<const float4 *>(T + (row0 + b) * ld + jl));
+                t[b][0] = v.x; t[b][1] = v.y; t[b][2] = v.z; t[b][3] = v.w;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) t[b][i] = (row_ok && jl + i < d_out) ? T[(row0 + b) * ld + jl + i] : 0.0f;
+            }
+        }
         __syncthreads();
         if (threadIdx.x < kRowCols) {
-            const int64_t j = j0 + threadIdx.x;
+            const int c = threadIdx.x;
+            const int64_t j = j0 + c;
             const bool in = j < d_out;
             const uint64_t bits = in ? b_bits(pb, n_words, j, r) : 0ull;
             const float g = in ? __ldg(gamma + j) : 0.0f;
+            float *dst = S + ((c & 3) * 32 + (c >> 2)) * kStride;
 #pragma unroll
-            for (int k = 0; k < RP; ++k)
-                S[threadIdx.x * kStride + k] = (k < r) ? (((bits >> k) & 1ull) ? g : -g) : 0.0f;
+            for (int k = 0; k < RP; ++k) dst[k] = (k < r) ? (((bits >> k) & 1ull) ? g : -g) : 0.0f;
         }
         __syncthreads();
 #pragma unroll
-        for (int cc = 0; cc < kRowCols / 32; ++cc) {
-            const int c = cc * 32 + lane;
-            const int64_t j = j0 + c;
-            float t[RB];
-#pragma unroll
-            for (int b = 0; b < RB; ++b) t[b] = (row0 + b < d_in && j < d_out) ? T[(row0 + b) * ld + j] : 0.0f;
+        for (int i = 0; i < 4; ++i) {
+            const float *src = S + (i * 32 + lane) * kStride;
 #pragma unroll
             for (int k4 = 0; k4 < RP / 4; ++k4) {
-                const float4 sv = *reinterpret_cast<const float4 *>(&S[c * kStride + 4 * k4]);
+                const float4 sv = *reinterpret_cast<const float4 *>(src + 4 * k4);
 #pragma unroll
                 for (int b = 0; b < RB; ++b) {
-                    acc[b][4 * k4] = fmaf(t[b], sv.x, acc[b][4 * k4]);
-                    acc[b][4 * k4 + 1] = fmaf(t[b], sv.y, acc[b][4 * k4 + 1]);
-                    acc[b][4 * k4 + 2] = fmaf(t[b], sv.z, acc[b][4 * k4 + 2]);
-                    acc[b][4 * k4 + 3] = fmaf(t[b], sv.w, acc[b][4 * k4 + 3]);
+                    acc[b][4 * k4] = fmaf(t[b][i], sv.x, acc[b][4 * k4]);
+                    acc[b][4 * k4 + 1] = fmaf(t[b][i], sv.y, acc[b][4 * k4 + 1]);
+                    acc[b][4 * k4 + 2] = fmaf(t[b][i], sv.z, acc[b][4 * k4 + 2]);
+                    acc[b][4 * k4 + 3] = fmaf(t[b][i], sv.w, acc[b][4 * k4 + 3]);
                 }
             }
         }
@@ -164,9 +179,9 @@ fit_col_pass_kernel(const float *__restrict__ T, int64_t ld, const uint32_t *__r
         __syncthreads();
         const int n = (int)((i_end - i0 < 64) ? (i_end - i0) : 64);
         if (j < d_out) {
-#pragma unroll 4
+#pragma unroll 16
             for (int il = 0; il < n; ++il) {
-                const float t = T[(i0 + il) * ld + j];
+                const float t = __ldcs(T + (i0 + il) * ld + j);
 #pragma unroll
                 for (int k4 = 0; k4 < RP / 4; ++k4) {
                     const float4 sv = *reinterpret_cast<const float4 *>(&S[il * RP + 4 * k4]);
@@ -193,10 +208,12 @@ fit_gram_kernel(const uint32_t *__restrict__ packed, const float *__restrict__ s
 {
     __shared__ double red[kFitThreads / 32][64];
     const int k = blockIdx.x;
+    const int64_t per = (n + kParts - 1) / kParts;
+    const int64_t e_begin = (int64_t)blockIdx.y * per, e_end = (e_begin + per < n) ? e_begin + per : n;
     double acc[64];
 #pragma unroll
     for (int l = 0; l < 64; ++l) acc[l] = 0.0;
-    for (int64_t e = threadIdx.x; e < n; e += kFitThreads) {
+    for (int64_t e = e_begin + threadIdx.x; e < e_end; e += kFitThreads) {
         const double s = (double)__ldg(scale + e);
         const double s2 = s * s;
         const uint64_t bits = (ROLE == 1) ? b_bits(packed, n_words, e, r) : a_bits(packed, e, r);
@@ -217,8 +234,17 @@ fit_gram_kernel(const uint32_t *__restrict__ packed, const float *__restrict__ s
     if (threadIdx.x < r) {
         double v = 0.0;
         for (int w = 0; w < kFitThreads / 32; ++w) v += red[w][threadIdx.x];
-        G[k * r + threadIdx.x] = v;
+        G[((int64_t)blockIdx.y * r + k) * r + threadIdx.x] = v;       // part blockIdx.y
     }
+}
+
+// sum of the kParts partial r x r matrices (or r-vectors), in a fixed order
+__device__ __forceinline__ double sum_parts(const double *__restrict__ parts, int stride, int e)
+{
+    double v = 0.0;
+#pragma unroll
+    for (int p = 0; p < kParts; ++p) v += parts[(int64_t)p * stride + e];
+    return v;
 }
 
 // ---- alpha_i = <c_i, W[i,:]> / (c_i^T Gq c_i), c_i = B1[i,:] * beta (Eq. alpha-update) ---------
@@ -228,7 +254,7 @@ fit_alpha_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, c
 {
     __shared__ double g[64 * 64];
     __shared__ double b[64];
-    for (int e = threadIdx.x; e < r * r; e += kFitThreads) g[e] = Gq[e];
+    for (int e = threadIdx.x; e < r * r; e += kFitThreads) g[e] = sum_parts(Gq, r * r, e);
     if (threadIdx.x < r) b[threadIdx.x] = (double)beta[threadIdx.x];
     __syncthreads();
     const int64_t i = (int64_t)blockIdx.x * kFitThreads + threadIdx.x;
@@ -253,15 +279,16 @@ fit_gamma_kernel(const uint32_t *__restrict__ pb, const float *__restrict__ Vpar
 {
     __shared__ double g[64 * 64];
     __shared__ double b[64];
-    for (int e = threadIdx.x; e < r * r; e += kFitThreads) g[e] = Gp[e];
+    for (int e = threadIdx.x; e < r * r; e += blockDim.x) g[e] = sum_parts(Gp, r * r, e);
     if (threadIdx.x < r) b[threadIdx.x] = (double)beta[threadIdx.x];
     __syncthreads();
-    const int64_t j = (int64_t)blockIdx.x * kFitThreads + threadIdx.x;
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= d_out) return;
     const uint64_t bits = b_bits(pb, (d_out * r + 31) / 32, j, r);
     double num = 0.0, den = 0.0;
     for (int k = 0; k < r; ++k) {
         double v = 0.0;
+#pragma unroll 8
         for (int c = 0; c < chunks; ++c) v += (double)Vpart[((int64_t)c * r + k) * d_out + j];   // fixed order
         const double dk = ((bits >> k) & 1ull) ? b[k] : -b[k];
         num += dk * v;
@@ -272,7 +299,7 @@ fit_gamma_kernel(const uint32_t *__restrict__ pb, const float *__restrict__ Vpar
     gamma[j] = den > 0.0 ? (float)(num / den) : 0.0f;
 }
 
-// ---- h_k = sum_i alpha_i B1[i,k] W[i,k] (Eq. beta-gram): one CTA, fixed-order tree --------------
+// ---- h_k = sum_i alpha_i B1[i,k] W[i,k] (Eq. beta-gram): kParts CTAs, fixed-order trees ------------
 __global__ void __launch_bounds__(kFitThreads)
 fit_h_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, const float *__restrict__ alpha,
              int64_t d_in, int r, double *__restrict__ h)
@@ -282,7 +309,9 @@ fit_h_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, const
     double acc[64];
 #pragma unroll
     for (int k = 0; k < 64; ++k) acc[k] = 0.0;
-    for (int64_t i = tid; i < d_in; i += kFitThreads) {
+    const int64_t per = (d_in + kParts - 1) / kParts;
+    const int64_t i_begin = (int64_t)blockIdx.x * per, i_end = (i_begin + per < d_in) ? i_begin + per : d_in;
+    for (int64_t i = i_begin + tid; i < i_end; i += kFitThreads) {
         const uint64_t bits = a_bits(pa, i, r);
         const double a = (double)alpha[i];
 #pragma unroll
@@ -300,14 +329,14 @@ fit_h_kernel(const uint32_t *__restrict__ pa, const float *__restrict__ W, const
     if (tid < r) {
         double v = 0.0;
         for (int w = 0; w < kFitThreads / 32; ++w) v += red[w * 64 + tid];
-        h[tid] = v;
+        h[blockIdx.x * r + tid] = v;            // part blockIdx.x
     }
 }
 
 // ---- beta = (Gp o Gq)^+ h (Eq. beta-Schur, Eq. beta-pinv): one CTA of 1024 threads ----------------
 // Shared memory (dynamic): A and E, n rows of n + 1 doubles each (n = r rounded up to even), then the
 // rotations of a round (2 x 64), h (64), the eigen-coefficients (64) and 2 x 32 partial norms.
-constexpr int kBetaThreads = 1024;
+constexpr int kBetaThreads = 1024;      // at most; small systems use fewer (a barrier of 128 threads is cheaper)
 
 __global__ void __launch_bounds__(kBetaThreads)
 fit_beta_kernel(const double *__restrict__ Gp, const double *__restrict__ Gq, const double *__restrict__ hvec, int r,
@@ -318,20 +347,20 @@ fit_beta_kernel(const double *__restrict__ Gp, const double *__restrict__ Gq, co
     const int ns = n + 1;        // padded row length: column walks without bank conflicts
     double *A = sh, *E = A + n * ns, *cs = E + n * ns, *h = cs + 2 * 64, *coef = h + 64, *part = coef + 64;
     __shared__ double off_norm, all_norm;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
 
-    for (int e = tid; e < n * n; e += kBetaThreads) {
+    for (int e = tid; e < n * n; e += nthr) {
         const int p = e / n, q = e - p * n;
-        A[p * ns + q] = (p < r && q < r) ? Gp[p * r + q] * Gq[p * r + q] : 0.0;     // Eq. beta-Schur
+        A[p * ns + q] = (p < r && q < r) ? sum_parts(Gp, r * r, p * r + q) * sum_parts(Gq, r * r, p * r + q) : 0.0;   // Eq. beta-Schur
         E[p * ns + q] = (p == q) ? 1.0 : 0.0;
     }
-    if (tid < 64) h[tid] = (tid < r) ? hvec[tid] : 0.0;
+    if (tid < 64) h[tid] = (tid < r) ? sum_parts(hvec, r, tid) : 0.0;
     __syncthreads();
 
     // cyclic Jacobi, n / 2 disjoint rotations per round (round-robin pairing), at most 40 sweeps
     for (int sweep = 0; sweep < 40; ++sweep) {
         double off = 0.0, all = 0.0;
-        for (int e = tid; e < n * n; e += kBetaThreads) {
+        for (int e = tid; e < n * n; e += nthr) {
             const int p = e / n, q = e - p * n;
             const double v = A[p * ns + q] * A[p * ns + q];
             all += v;
@@ -346,12 +375,14 @@ fit_beta_kernel(const double *__restrict__ Gp, const double *__restrict__ Gq, co
         __syncthreads();
         if (tid == 0) {
             double o = 0.0, a = 0.0;
-            for (int w = 0; w < kBetaThreads / 32; ++w) { o += part[w]; a += part[32 + w]; }
+            for (int w = 0; w < nthr / 32; ++w) { o += part[w]; a += part[32 + w]; }
             off_norm = o;
             all_norm = a;
         }
         __syncthreads();
-        if (off_norm <= 1e-30 * all_norm) break;
+        // off-diagonal mass below 1e-12 of the whole (squares: 1e-24): the rotations left only move
+        // rounding noise (they stall near n eps, which a tighter test would never see)
+        if (off_norm <= 1e-24 * all_norm) break;
         for (int round = 0; round < n - 1; ++round) {
             // pair m of this round: (n-1, round) for m = 0, else ((round+m) % (n-1), (round-m) mod (n-1))
             if (tid < n / 2) {
@@ -371,7 +402,7 @@ fit_beta_kernel(const double *__restrict__ Gp, const double *__restrict__ Gq, co
             }
             __syncthreads();
             // columns: A <- A J, E <- E J (task = row t, pair m)
-            for (int task = tid; task < n * (n / 2); task += kBetaThreads) {
+            for (int task = tid; task < n * (n / 2); task += nthr) {
                 const int t = task / (n / 2), m = task - t * (n / 2);
                 const int p = (m == 0) ? n - 1 : (round + m) % (n - 1);
                 const int q = (m == 0) ? round : (round - m + (n - 1)) % (n - 1);
@@ -385,7 +416,7 @@ fit_beta_kernel(const double *__restrict__ Gp, const double *__restrict__ Gq, co
             }
             __syncthreads();
             // rows: A <- J^T A (task = column t, pair m)
-            for (int task = tid; task < n * (n / 2); task += kBetaThreads) {
+            for (int task = tid; task < n * (n / 2); task += nthr) {
                 const int t = task / (n / 2), m = task - t * (n / 2);
                 const int p = (m == 0) ? n - 1 : (round + m) % (n - 1);
                 const int q = (m == 0) ? round : (round - m + (n - 1)) % (n - 1);
@@ -424,8 +455,8 @@ int padded_rank(int r) { return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64; }
 struct FitWorkspace {
     float *W;          // d_in x r
     float *Vpart;      // chunks x r x d_out
-    double *Gq, *Gp;   // r x r each
-    double *h;         // r
+    double *Gq, *Gp;   // kParts partial r x r matrices each
+    double *h;         // kParts partial r-vectors
     int chunks;
     int64_t rows_per_chunk;
     size_t bytes;
@@ -443,9 +474,9 @@ FitWorkspace carve(void *base, int64_t d_in, int64_t d_out, int r)
     char *p = static_cast<char *>(base);
     w.W = reinterpret_cast<float *>(p + off); off += up((size_t)d_in * r * 4);
     w.Vpart = reinterpret_cast<float *>(p + off); off += up((size_t)w.chunks * r * d_out * 4);
-    w.Gq = reinterpret_cast<double *>(p + off); off += up((size_t)r * r * 8);
-    w.Gp = reinterpret_cast<double *>(p + off); off += up((size_t)r * r * 8);
-    w.h = reinterpret_cast<double *>(p + off); off += up((size_t)r * 8);
+    w.Gq = reinterpret_cast<double *>(p + off); off += up((size_t)kParts * r * r * 8);
+    w.Gp = reinterpret_cast<double *>(p + off); off += up((size_t)kParts * r * r * 8);
+    w.h = reinterpret_cast<double *>(p + off); off += up((size_t)kParts * r * 8);
     w.bytes = off;
     return w;
 }
@@ -461,8 +492,9 @@ void launch_row(const float *T, int64_t ld, const uint32_t *pb, const float *gam
                 float *W, cudaStream_t s)
 {
     const int rows_per_block = (kFitThreads / 32) * RB;
+    const int vec4 = (reinterpret_cast<uintptr_t>(T) % 16 == 0 && ld % 4 == 0) ? 1 : 0;
     fit_row_pass_kernel<RP, RB><<<(unsigned)((d_in + rows_per_block - 1) / rows_per_block), kFitThreads, 0, s>>>(
-        T, ld, pb, gamma, d_in, d_out, r, W);
+        T, ld, pb, gamma, d_in, d_out, r, vec4, W);
 }
 
 template <int RP>
@@ -491,12 +523,12 @@ int launch_fit_scales(const float *target, int64_t ld, const uint32_t *pa, const
         // rows of T through B2^T diag(gamma), and Q Q^T
         if (axes & (LORDBA_FIT_ALPHA | LORDBA_FIT_BETA)) {
             switch (rp) {
-                case 8:  launch_row<8, 4>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
-                case 16: launch_row<16, 4>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
-                case 32: launch_row<32, 2>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
+                case 8:  launch_row<8, 2>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
+                case 16: launch_row<16, 2>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
+                case 32: launch_row<32, 1>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
                 default: launch_row<64, 1>(target, ld, pb, s_out, d_in, d_out, r, w.W, stream); break;
             }
-            fit_gram_kernel<1><<<r, kFitThreads, 0, stream>>>(pb, s_out, d_out, r, b_words, w.Gq);
+            fit_gram_kernel<1><<<dim3(r, kParts), kFitThreads, 0, stream>>>(pb, s_out, d_out, r, b_words, w.Gq);
             count_launch(2);
         }
         if (axes & LORDBA_FIT_ALPHA) {
@@ -505,12 +537,15 @@ int launch_fit_scales(const float *target, int64_t ld, const uint32_t *pa, const
             count_launch();
         }
         if (axes & (LORDBA_FIT_BETA | LORDBA_FIT_GAMMA)) {
-            fit_gram_kernel<0><<<r, kFitThreads, 0, stream>>>(pa, s_in, d_in, r, 0, w.Gp);
+            fit_gram_kernel<0><<<dim3(r, kParts), kFitThreads, 0, stream>>>(pa, s_in, d_in, r, 0, w.Gp);
             count_launch();
         }
         if (axes & LORDBA_FIT_BETA) {
-            fit_h_kernel<<<1, kFitThreads, 0, stream>>>(pa, w.W, s_in, d_in, r, w.h);
-            fit_beta_kernel<<<1, kBetaThreads, beta_smem(r), stream>>>(w.Gp, w.Gq, w.h, r, s_r);
+            fit_h_kernel<<<kParts, kFitThreads, 0, stream>>>(pa, w.W, s_in, d_in, r, w.h);
+            const int n_even = (r + 1) & ~1;
+            int beta_threads = 128;              // one task per thread and phase when it fits: n * n / 2 tasks
+            while (beta_threads < n_even * n_even / 2 && beta_threads < kBetaThreads) beta_threads *= 2;
+            fit_beta_kernel<<<1, beta_threads, beta_smem(r), stream>>>(w.Gp, w.Gq, w.h, r, s_r);
             count_launch(2);
         }
         if (axes & LORDBA_FIT_GAMMA) {

@@ -44,6 +44,13 @@
 //     values (an adapter exported with fp16 scales), as one half, which halves
 //     the tensor-core work of that product.  z stays a bf16 pair (its range is
 //     not bounded by 65504) and the second product is unchanged.
+//   * Multi-envelope adapters (Eq. 4: several scale triples over one pair of
+//     carriers): the first product takes the envelopes EG at a time (as many as
+//     keep EG x padded rank <= 64 partial sums per token row in registers), x
+//     fragments and sign bits shared by the envelopes of a pass; an adapter with
+//     more envelopes streams its x items once per group.  The second product
+//     walks all envelopes with the same +-1 fragments and accumulates
+//     sum_e s_out[e] * v_e on top of y in float32: one rounding.
 //
 // Warps split the d_in axis for the first product (fixed-order reduction
 // through shared memory, hence deterministic) and the d_out axis for the
@@ -52,7 +59,8 @@
 //
 // Every mbarrier wait is bounded: after ~1 s it records a code in the device
 // status word, raises the CTA's abort flag (all later waits return at once) and
-// the kernel runs to its end.
+// the kernel runs to its end; a CTA whose first product is incomplete writes
+// nothing, so every element of y is either its old value or the right new one.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>

@@ -83,6 +83,7 @@ typedef enum {
                               /* 128-token tiles (rank > 32: 32 tiles, else eight per SM), and  */
                               /* for widths that are not multiples of 64 from 128 tokens up     */
                               /* (rank a multiple of 8); else FMA.  lordba_query_variant tells  */
+                              /* which one a given call gets                                   */
     LORDBA_VARIANT_FMA = 1,   /* CUDA-core float32 FMA kernel (always used for LORDBA_F32)  */
     LORDBA_VARIANT_TC = 2,    /* tcgen05/TMA cluster kernel; LORDBA_EUNSUPPORTED if the     */
                               /* shape or alignment rules it out                            */

@@ -463,6 +463,7 @@ def supplementary_workloads(lordba, dev, stream, sampler):
     run("attn_T2048_r16_ell2", 20, 5, shapes=[(H, H)], r=16, Tn=2048, ell=2)
     run("attn_T2048_r16_ell4", 20, 5, shapes=[(H, H)], r=16, Tn=2048, ell=4)
     run("attn_T2048_r4_ell2", 20, 5, shapes=[(H, H)], r=4, Tn=2048, ell=2)
+    run("layer_T2048_r32_ell2", 8, 4, shapes=layer, r=32, Tn=2048, ell=2)
     run("multi_8x256_r16", 20, 5, shapes=[(H, H)] * 8, r=16, Tn=256, segments=8)
     run("multi_8x256_r32", 20, 5, shapes=[(H, H)] * 8, r=32, Tn=256, segments=8)
     # config 3: decode, one batched call per layer (latency bound: the figure is us per call)

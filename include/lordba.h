@@ -79,8 +79,8 @@ typedef enum {
 /* Kernel families the forward entry points can be pinned to (default AUTO). */
 typedef enum {
     LORDBA_VARIANT_AUTO = 0,  /* the library's choice: streaming kernel where the shape allows  */
-                              /* it; tcgen05 kernel for rank > 16 once a call holds enough     */
-                              /* 128-token tiles (rank > 32: 32 tiles, else eight per SM), and  */
+                              /* it; tcgen05 kernel for rank (x envelopes) > 16 once a call has */
+                              /* enough 128-token tiles (> 32: 32 tiles, else eight per SM), and */
                               /* for widths that are not multiples of 64 from 128 tokens up     */
                               /* (rank a multiple of 8); else FMA.  lordba_query_variant tells  */
                               /* which one a given call gets                                   */
@@ -113,8 +113,9 @@ typedef struct lordba_proj {
  * s_r as ell x r and s_out as ell x d_out (row-major, envelope e in row e), and the call adds
  *     sum_e  s_out[e] * ( B_sign ( s_r[e] * ( A_sign ( s_in[e] * x[t,:] ) ) ) )
  * to y[t,:] with one rounding.  Flags without this field mean ell = 1.  Every envelope count at
- * every rank runs on the tensor cores (streaming kernel); the cost is about that of one envelope
- * at rank ell * r.
+ * every rank runs on the tensor cores (streaming kernel; two envelopes with ell * r <= 64 also
+ * in the tcgen05 kernel, which the library takes for them by the same rule as for one envelope
+ * of rank ell * r); the cost is about that of one envelope at rank ell * r.
  */
 #define LORDBA_MAX_ELL 8
 #define LORDBA_PROJ_ELL(ell) ((((ell) - 1) & 0xf) << 8)

@@ -158,8 +158,10 @@ FamilySelector make_selector(const lordba_proj *projs, int n, int64_t T, const i
             const int64_t rows = rows_of(tokens, T, i);
             if (rows == 0) continue;
             if (tiles == 0) all_ok = true;
-            all_ok = all_ok && projs[i].r > 16 && tc_supported(projs[i], rows, dtype);
-            all_high = all_high && projs[i].r > 32;
+            // (what counts is the width of the intermediate: envelopes x rank)
+            const int width = (((projs[i].flags >> 8) & 0xf) + 1) * projs[i].r;
+            all_ok = all_ok && width > 16 && tc_supported(projs[i], rows, dtype);
+            all_high = all_high && width > 32;
             tiles += (rows + 127) / 128;
         }
         sel.use_tc = all_ok && tiles >= (all_high ? 32 : 8 * 148);

@@ -27,6 +27,12 @@
 //               tile (already in the slot) += s_out * V in fp32, rounded once to
 //               bf16 in place, TMA-stored from the same slot.
 //
+// Two-envelope adapters (Def. 1 / Eq. 4, ell = 2, ell * r <= 64) run in the instantiation L = 2:
+// both envelopes use the same carriers, so W1 carries every sign under each envelope's s_in
+// (rows e r + k hi, ell r + e r + k lo) and U has 2 ell r columns; z is one hi/lo operand pair per
+// envelope; stage 2 runs per envelope over the same W2 into ell accumulators, and the epilogue
+// adds s_out[e] * V_e over the envelopes before the one rounding.
+//
 // The roles are decoupled by mbarriers only, so each one's per-chunk latency is
 // a ceiling for the whole pipeline; the single MMA-issuing thread in particular
 // carries its ring positions and descriptor words instead of recomputing them.
@@ -57,9 +63,10 @@ constexpr int kGenThreads = kGenGroups * kGenGroupThreads;   // warps 2-9
 constexpr int kEpiThreads = 256;          // warps 10-17
 constexpr int kThreads = 64 + kGenThreads + kEpiThreads;
 constexpr int kMaxTcBatch = 96;          // 96 x 320 bytes of descriptors: inside the 32 KiB of kernel parameters
-constexpr int kTmemCols = 256;
-constexpr int kTmemU = 0;               // stage-1 accumulator columns [0, 2r)
-constexpr int kTmemV = 128;             // stage-2 accumulators: [128,192) and [192,256)
+constexpr int kMaxTcEll = 2;            // envelopes per adapter this kernel takes (ell * r <= kMaxRank)
+constexpr int kTmemU = 0;               // stage-1 accumulator columns [0, 2 ell r)
+constexpr int kTmemV = 128;             // stage-2 accumulators: two buffers of ell x 64 columns
+__host__ __device__ inline uint32_t tmem_cols(int ell) { return ell > 1 ? 512u : 256u; }
 constexpr int kSmemBudget = 227 * 1024;
 
 // Element type of x and y, and how s_in enters the first product (same meaning as in the
@@ -88,6 +95,7 @@ struct TcBatch {
     int n_proj;
     int total_tiles;       // projections may differ in their token counts (tile_start of each)
     int r;                 // rank, multiple of 8
+    int ell;               // envelopes per adapter (1 or 2): scale triples that share the carriers
     int kp;                // r rounded up to 16 (K extent of the stage-2 MMA)
     int cluster;           // CTAs per cluster
     int slots;             // ring depth
@@ -105,39 +113,41 @@ struct SmemPlan {
     int slot_data;          // bytes reserved for the x / y box of a slot (multiple of 1024)
     int slot_stride;        // + the slot's raw scale values and sign bytes
     int op_bytes, off_ops;  // one generated operand tile; start of the operand ring
-    int off_zhi, off_zlo, z_bytes;
+    int off_z, z_bytes;     // per envelope: z hi tile, then z lo tile
+    int raw_sign;           // offset of the sign bytes in a slot's raw area (behind the scale rows)
     int off_rx, off_bar, off_misc, total;
 };
 
 __host__ __device__ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-__host__ __device__ inline int aux_operand_bytes(int r, int kp)
+__host__ __device__ inline int aux_operand_bytes(int r, int kp, int ell)
 {
-    const int w1 = 2 * r * 128;              // 2r rows x 64 bf16
+    const int w1 = 2 * ell * r * 128;        // 2 ell r rows x 64 bf16
     const int w2 = kChunk * kp * 2;          // 64 rows x kp bf16
     return w1 > w2 ? w1 : w2;
 }
 
-__host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile_rows, int cluster)
+__host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile_rows, int cluster, int ell)
 {
     SmemPlan s;
     // The MMA reads 128 rows (16 KiB) from the start of a slot whatever tile_rows is; what lies
     // beyond the box (this slot's raw area, the next slot) only reaches accumulator rows that
     // nobody reads.  `total` is padded so that this read stays inside the allocation.
     s.slot_data = round_up(tile_rows * kChunk * 2, 1024);
-    // behind the box: 256 B of raw scale values and up to 512 B of raw sign bytes
-    s.slot_stride = s.slot_data + round_up(256 + 8 * kMaxRank, 1024);
+    // behind the box: 256 B of raw scale values per envelope and up to 512 B of raw sign bytes
+    // (8 r bytes; ell * r <= kMaxRank)
+    s.raw_sign = 256 * ell;
+    s.slot_stride = s.slot_data + round_up(s.raw_sign + 8 * r, 1024);
     // The generated operands live in a short ring of their own (the MMA is done with one within
     // a microsecond), so that the data ring can be deep enough to cover the load latency at
     // any rank.
-    s.op_bytes = round_up(aux_operand_bytes(r, kp), 1024);
+    s.op_bytes = round_up(aux_operand_bytes(r, kp, ell), 1024);
     s.off_ops = slots * s.slot_stride;
     s.z_bytes = (kTileM / 8) * (kp / 8) * 128;
-    s.off_zhi = s.off_ops + kOps * s.op_bytes;
-    s.off_zlo = s.off_zhi + s.z_bytes;
-    s.off_rx = s.off_zlo + s.z_bytes;
+    s.off_z = s.off_ops + kOps * s.op_bytes;
+    s.off_rx = s.off_z + 2 * ell * s.z_bytes;
     // the exchange buffer for partial u exists only when a cluster splits the feature axes
-    s.off_bar = s.off_rx + (cluster > 1 ? kTileM * r * 4 : 0);
+    s.off_bar = s.off_rx + (cluster > 1 ? kTileM * ell * r * 4 : 0);
     s.off_misc = s.off_bar + (3 * slots + 2 * kOps + 8) * 8;
     s.total = s.off_misc + 16;
     const int last_read_end = (slots - 1) * s.slot_stride + kTileM * kChunk * 2;
@@ -314,6 +324,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t r[32])
                    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr));
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t r[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr));
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
@@ -367,6 +385,8 @@ __device__ __forceinline__ void split_range(int n, int parts, int idx, int &begi
 
 // ------------------------------------------------------------------------------------ the kernel
 
+// L: envelopes per adapter (scale triples over the same carriers), 1 or 2 (= B.ell).
+template <int L>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_forward_kernel(const __grid_constant__ TcBatch B)
 {
@@ -376,6 +396,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     const uint32_t sm_base = smem_u32(sm);
 
     const int r = B.r, kp = B.kp, S = B.slots, C = B.cluster;
+    const int RT = L * r;                  // columns of u over all envelopes
     const int tile_rows = B.tile_rows;
     // Programmatic dependent launch, same protocol as the streaming kernel.  A launch that must
     // see what ran before it sets up, waits for it, and only then lets its successor in.  A launch
@@ -385,7 +406,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     // one CTA per SM the successor's CTAs start as this grid's CTAs leave: no idle tail between
     // the launches of one call.
     if (!B.wait_prev) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const SmemPlan plan = make_plan(r, kp, S, tile_rows, C);
+    const SmemPlan plan = make_plan(r, kp, S, tile_rows, C, L);
     const uint32_t box_bytes = (uint32_t)tile_rows * kChunk * 2;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t crank = cluster_ctarank();
@@ -409,9 +430,11 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
 
     const int kt8 = kp / 8;                 // 16-byte chunks per row of a stage-2 operand
     const int r8 = r / 8;
+    const int rt8 = RT / 8;
     const bool half_io = B.io != kIoBf16;       // x, y and W1 are IEEE halves
     const bool lo_pass = B.io != kIoF16Exact;   // W1 and U carry low parts of s_in
     const uint32_t sign_bytes = 8u * r;     // sign bytes next to one 64-column chunk, either stage
+    const uint32_t raw_bytes = 256u * L + sign_bytes;   // + one 64-entry scale row per envelope
 
     // ---- one-time setup ---------------------------------------------------------------------
     if (tid == 0) {
@@ -425,7 +448,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             mbar_init(bar_op_empty(o), 1);
         }
         mbar_init(bar_u_full, 1);
-        mbar_init(bar_z_full, (uint32_t)(tile_rows * r8));   // one arrive per (row, 8-wide piece), all owners
+        mbar_init(bar_z_full, (uint32_t)(tile_rows * rt8));  // one arrive per (row, 8-wide piece), all owners
         mbar_init(bar_rx_full, (uint32_t)(2 * tile_rows));   // one arrive per (token row, column half)
         mbar_init(bar_v_full(0), 1);
         mbar_init(bar_v_full(1), 1);
@@ -436,12 +459,12 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+                     ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols(L)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // stage-2 A operands start as zeros (K padding beyond r and rows beyond tile_rows stay zero)
-    for (int i = tid; i < 2 * plan.z_bytes / 16; i += kThreads)
-        reinterpret_cast<uint4 *>(sm + plan.off_zhi)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < 2 * L * plan.z_bytes / 16; i += kThreads)
+        reinterpret_cast<uint4 *>(sm + plan.off_z)[i] = make_uint4(0, 0, 0, 0);
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -492,9 +515,11 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     const uint32_t slot = sm_base + s * plan.slot_stride;
                     const uint32_t rawdst = slot + plan.slot_data;
                     if ((c + 1) * kChunk <= P.d_in) {
-                        mbar_arrive_expect_tx(bar_raw(s), 256u + sign_bytes);
-                        bulk_load(rawdst, P.s_in + (size_t)c * kChunk, 256u, bar_raw(s));
-                        bulk_load(rawdst + 256u, reinterpret_cast<const uint8_t *>(P.packed_A) + (size_t)c * sign_bytes,
+                        mbar_arrive_expect_tx(bar_raw(s), raw_bytes);
+#pragma unroll
+                        for (int e = 0; e < L; ++e)
+                            bulk_load(rawdst + 256u * e, P.s_in + (size_t)e * P.d_in + (size_t)c * kChunk, 256u, bar_raw(s));
+                        bulk_load(rawdst + plan.raw_sign, reinterpret_cast<const uint8_t *>(P.packed_A) + (size_t)c * sign_bytes,
                                   sign_bytes, bar_raw(s));
                     } else {
                         mbar_arrive(bar_raw(s));
@@ -509,9 +534,11 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     const uint32_t slot = sm_base + s * plan.slot_stride;
                     const uint32_t rawdst = slot + plan.slot_data;
                     if ((c + 1) * kChunk <= P.d_out) {
-                        mbar_arrive_expect_tx(bar_raw(s), 256u + sign_bytes);
-                        bulk_load(rawdst, P.s_out + (size_t)c * kChunk, 256u, bar_raw(s));
-                        bulk_load(rawdst + 256u, reinterpret_cast<const uint8_t *>(P.packed_B) + (size_t)c * sign_bytes,
+                        mbar_arrive_expect_tx(bar_raw(s), raw_bytes);
+#pragma unroll
+                        for (int e = 0; e < L; ++e)
+                            bulk_load(rawdst + 256u * e, P.s_out + (size_t)e * P.d_out + (size_t)c * kChunk, 256u, bar_raw(s));
+                        bulk_load(rawdst + plan.raw_sign, reinterpret_cast<const uint8_t *>(P.packed_B) + (size_t)c * sign_bytes,
                                   sign_bytes, bar_raw(s));
                     } else {
                         mbar_arrive(bar_raw(s));
@@ -529,7 +556,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             if (lane == 0) {
                 // N of stage 1: hi and lo rows, or the hi rows alone rounded up to the next legal N
                 // (rows past r then hold stale operand data and feed accumulator columns nobody reads)
-                const uint32_t idesc1 = instr_desc(kTileM, lo_pass ? 2 * r : (r + 15) / 16 * 16, half_io);
+                const uint32_t idesc1 = instr_desc(kTileM, lo_pass ? 2 * RT : (RT + 15) / 16 * 16, half_io);
                 const uint32_t idesc2 = instr_desc(kTileM, kChunk, false);      // z and W2 are always bf16
                 const int ksteps2 = kp / 16;
                 // descriptor words (layout above): low = address >> 4 | (lbo >> 4) << 16,
@@ -540,8 +567,8 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 const uint32_t op_lo = ((base18 + plan.off_ops) >> 4) | (8u << 16);
                 const uint32_t w1_hi = 64u | (1u << 14);
                 const uint32_t z_hi = (uint32_t)(kt8 * 8) | (1u << 14);
-                const uint32_t zhi_lo = ((base18 + plan.off_zhi) >> 4) | (8u << 16);
-                const uint32_t zlo_lo = ((base18 + plan.off_zlo) >> 4) | (8u << 16);
+                const uint32_t zhi_lo = ((base18 + plan.off_z) >> 4) | (8u << 16);          // envelope 0, hi tile
+                const uint32_t z_units = (uint32_t)plan.z_bytes >> 4;                       // hi -> lo, lo -> next envelope
                 const uint32_t slot_units = (uint32_t)plan.slot_stride >> 4, op_units = (uint32_t)plan.op_bytes >> 4;
                 uint32_t s = it % S, ph = (it / S) & 1u, o = it % kOps, oph = (it / kOps) & 1u;
                 for (int c = kb; c < ke; ++c, ++it) {
@@ -573,16 +600,21 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                     ok = mbar_wait<false>(wctx, bar_v_empty(vb), vph ^ 1u, kDevMmaWaitTimeout) && ok;
                     tc_fence_after();
                     const uint32_t b_lo = op_lo + o * op_units;           // W2, no swizzle
-                    const uint32_t d = tmem_base + kTmemV + vb * kChunk;
+                    // one accumulator per envelope: V_e = Z_e,hi W2^T + Z_e,lo W2^T over the same W2
                     if (ok) {
 #pragma unroll
-                        for (int ks = 0; ks < kMaxRank / 16; ++ks)
-                            if (ks < ksteps2)
-                                mma_bf16_words(d, zhi_lo + 16u * ks, z_hi, b_lo + 16u * ks, z_hi, idesc2, ks > 0 ? 1u : 0u);
+                        for (int e = 0; e < L; ++e) {
+                            const uint32_t d = tmem_base + kTmemV + (vb * L + e) * kChunk;
+                            const uint32_t zh_lo = zhi_lo + 2u * e * z_units, zl_lo = zh_lo + z_units;
 #pragma unroll
-                        for (int ks = 0; ks < kMaxRank / 16; ++ks)
-                            if (ks < ksteps2)
-                                mma_bf16_words(d, zlo_lo + 16u * ks, z_hi, b_lo + 16u * ks, z_hi, idesc2, 1u);
+                            for (int ks = 0; ks < kMaxRank / 16; ++ks)
+                                if (ks < ksteps2)
+                                    mma_bf16_words(d, zh_lo + 16u * ks, z_hi, b_lo + 16u * ks, z_hi, idesc2, ks > 0 ? 1u : 0u);
+#pragma unroll
+                            for (int ks = 0; ks < kMaxRank / 16; ++ks)
+                                if (ks < ksteps2)
+                                    mma_bf16_words(d, zl_lo + 16u * ks, z_hi, b_lo + 16u * ks, z_hi, idesc2, 1u);
+                        }
                     }
                     mma_commit(bar_v_full(vb));
                     mma_commit(bar_op_empty(o));
@@ -608,40 +640,51 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 mbar_wait<false>(wctx, bar_op_empty(o), ((it / kOps) & 1u) ^ 1u, kDevMmaWaitTimeout);
                 uint8_t *aux = sm + plan.off_ops + o * plan.op_bytes;
                 float *raw_scale = reinterpret_cast<float *>(sm + s * plan.slot_stride + plan.slot_data);
-                uint8_t *raw_sign = reinterpret_cast<uint8_t *>(raw_scale) + 256;
+                uint8_t *raw_sign = reinterpret_cast<uint8_t *>(raw_scale) + plan.raw_sign;
                 if ((c + 1) * kChunk > P.d_in) {
                     // ragged last chunk: guarded loads (the sign block itself is always complete)
-                    if (g < kChunk) raw_scale[g] = (c * kChunk + g < P.d_in) ? __ldg(P.s_in + c * kChunk + g) : 0.0f;
+                    for (int idx = g; idx < L * kChunk; idx += kGenGroupThreads) {
+                        const int e = idx >> 6, col = c * kChunk + (idx & 63);
+                        raw_scale[idx] = (col < P.d_in) ? __ldg(P.s_in + (size_t)e * P.d_in + col) : 0.0f;
+                    }
                     for (int w = g; w < 2 * r; w += kGenGroupThreads)
                         reinterpret_cast<uint32_t *>(raw_sign)[w] = __ldg(P.packed_A + (size_t)c * 2 * r + w);
                     asm volatile("bar.sync %0, %1;" ::"r"(2 + group), "n"(kGenGroupThreads) : "memory");
                 }
-                // s_in of this thread's 8 columns, split into bf16 hi + bf16 lo
-                const float4 sa = *reinterpret_cast<const float4 *>(raw_scale + cc * 8);
-                const float4 sb = *reinterpret_cast<const float4 *>(raw_scale + cc * 8 + 4);
-                const float sv[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
-                uint32_t hi[4], lo[4];
+                // s_in of this thread's 8 columns (every envelope's), split into bf16 hi + bf16 lo
+                uint32_t hi[L][4], lo[L][4];
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    if (half_io) {
-                        hi[p] = pack2_f16(sv[2 * p], sv[2 * p + 1]);
-                        const float2 hf = unpack2_f16(hi[p]);
-                        lo[p] = pack2_f16(sv[2 * p] - hf.x, sv[2 * p + 1] - hf.y);
-                    } else {
-                        const float ah = bf16_round(sv[2 * p]), bh = bf16_round(sv[2 * p + 1]);
-                        hi[p] = pack2_bf16(ah, bh);
-                        lo[p] = pack2_bf16(sv[2 * p] - ah, sv[2 * p + 1] - bh);
+                for (int e = 0; e < L; ++e) {
+                    const float4 sa = *reinterpret_cast<const float4 *>(raw_scale + e * kChunk + cc * 8);
+                    const float4 sb = *reinterpret_cast<const float4 *>(raw_scale + e * kChunk + cc * 8 + 4);
+                    const float sv[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        if (half_io) {
+                            hi[e][p] = pack2_f16(sv[2 * p], sv[2 * p + 1]);
+                            const float2 hf = unpack2_f16(hi[e][p]);
+                            lo[e][p] = pack2_f16(sv[2 * p] - hf.x, sv[2 * p + 1] - hf.y);
+                        } else {
+                            const float ah = bf16_round(sv[2 * p]), bh = bf16_round(sv[2 * p + 1]);
+                            hi[e][p] = pack2_bf16(ah, bh);
+                            lo[e][p] = pack2_bf16(sv[2 * p] - ah, sv[2 * p + 1] - bh);
+                        }
                     }
                 }
+                // W1 rows: envelope e, rank k -> hi row e r + k, lo row ell r + e r + k (the same signs
+                // under every envelope's scales)
                 uint8_t *w1 = aux;
                 for (int k = kg0 * 8 + rsub; k < r; k += kGenGroupThreads / 8) {
                     const uint4 m = sign_masks(raw_sign[k * 8 + cc]);
-                    const int row_hi = k, row_lo = r + k;
-                    *reinterpret_cast<uint4 *>(w1 + (row_hi >> 3) * 1024 + cc * 128 + (row_hi & 7) * 16) =
-                        make_uint4(hi[0] ^ m.x, hi[1] ^ m.y, hi[2] ^ m.z, hi[3] ^ m.w);
-                    if (lo_pass)
-                        *reinterpret_cast<uint4 *>(w1 + (row_lo >> 3) * 1024 + cc * 128 + (row_lo & 7) * 16) =
-                            make_uint4(lo[0] ^ m.x, lo[1] ^ m.y, lo[2] ^ m.z, lo[3] ^ m.w);
+#pragma unroll
+                    for (int e = 0; e < L; ++e) {
+                        const int row_hi = e * r + k, row_lo = RT + row_hi;
+                        *reinterpret_cast<uint4 *>(w1 + (row_hi >> 3) * 1024 + cc * 128 + (row_hi & 7) * 16) =
+                            make_uint4(hi[e][0] ^ m.x, hi[e][1] ^ m.y, hi[e][2] ^ m.z, hi[e][3] ^ m.w);
+                        if (lo_pass)
+                            *reinterpret_cast<uint4 *>(w1 + (row_lo >> 3) * 1024 + cc * 128 + (row_lo & 7) * 16) =
+                                make_uint4(lo[e][0] ^ m.x, lo[e][1] ^ m.y, lo[e][2] ^ m.z, lo[e][3] ^ m.w);
+                    }
                 }
                 fence_proxy_async();
                 mbar_arrive(bar_op_full(o));
@@ -654,10 +697,13 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 mbar_wait<false>(wctx, bar_op_empty(o), ((it / kOps) & 1u) ^ 1u, kDevMmaWaitTimeout);
                 uint8_t *aux = sm + plan.off_ops + o * plan.op_bytes;
                 float *raw_scale = reinterpret_cast<float *>(sm + s * plan.slot_stride + plan.slot_data);
-                uint8_t *raw_sign = reinterpret_cast<uint8_t *>(raw_scale) + 256;
+                uint8_t *raw_sign = reinterpret_cast<uint8_t *>(raw_scale) + plan.raw_sign;
                 if ((c + 1) * kChunk > P.d_out) {
                     const int64_t n_words = ((int64_t)P.d_out * r + 31) / 32;
-                    if (g < kChunk) raw_scale[g] = (c * kChunk + g < P.d_out) ? __ldg(P.s_out + c * kChunk + g) : 0.0f;
+                    for (int idx = g; idx < L * kChunk; idx += kGenGroupThreads) {
+                        const int e = idx >> 6, col = c * kChunk + (idx & 63);
+                        raw_scale[idx] = (col < P.d_out) ? __ldg(P.s_out + (size_t)e * P.d_out + col) : 0.0f;
+                    }
                     for (int w = g; w < 2 * r; w += kGenGroupThreads) {
                         const int64_t gw = (int64_t)c * 2 * r + w;
                         reinterpret_cast<uint32_t *>(raw_sign)[w] = (gw < n_words) ? __ldg(P.packed_B + gw) : 0u;
@@ -698,11 +744,13 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             if (C == 1) {
                 // no exchange: this thread's pieces of u go straight to z = s_r * u as bf16 hi + lo
                 if (warp_has_rows) {
-                    for (int p = chalf; p < r8; p += 2) {
+                    // piece p = columns 8p .. 8p+7 of u = envelope p / r8, ranks 8 (p % r8) ..; s_r is
+                    // ell x r row-major, so its flat index is the column of u
+                    for (int p = chalf; p < rt8; p += 2) {
                         float h[8], l[8];
                         tmem_ld8(tlane + kTmemU + p * 8, h);          // warp-collective
                         if (lo_pass) {
-                            tmem_ld8(tlane + kTmemU + r + p * 8, l);
+                            tmem_ld8(tlane + kTmemU + RT + p * 8, l);
                         } else {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) l[i] = 0.0f;
@@ -718,9 +766,10 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                                 zh[q] = pack2_bf16(h0, h1);
                                 zl[q] = pack2_bf16(z0 - h0, z1 - h1);
                             }
-                            const uint32_t off = (uint32_t)((row >> 3) * (kt8 * 128) + p * 128 + (row & 7) * 16);
-                            *reinterpret_cast<uint4 *>(sm + plan.off_zhi + off) = make_uint4(zh[0], zh[1], zh[2], zh[3]);
-                            *reinterpret_cast<uint4 *>(sm + plan.off_zlo + off) = make_uint4(zl[0], zl[1], zl[2], zl[3]);
+                            const int env = (L == 1) ? 0 : p / r8, pe = p - env * r8;
+                            const uint32_t off = (uint32_t)(env * 2 * plan.z_bytes + (row >> 3) * (kt8 * 128) + pe * 128 + (row & 7) * 16);
+                            *reinterpret_cast<uint4 *>(sm + plan.off_z + off) = make_uint4(zh[0], zh[1], zh[2], zh[3]);
+                            *reinterpret_cast<uint4 *>(sm + plan.off_z + plan.z_bytes + off) = make_uint4(zl[0], zl[1], zl[2], zl[3]);
                             fence_proxy_async();
                             mbar_arrive(bar_z_full);
                         }
@@ -732,12 +781,12 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 const uint32_t owner = row_valid ? (uint32_t)(row / rows_per) : 0u;
                 const int row_local = row - (int)owner * rows_per;
                 const uint32_t rx_remote = mapa(sm_base + plan.off_rx, owner) +
-                                           (uint32_t)(((int)crank * rows_per + row_local) * r) * 4u;
-                for (int p = chalf; p < r8; p += 2) {
+                                           (uint32_t)(((int)crank * rows_per + row_local) * RT) * 4u;
+                for (int p = chalf; p < rt8; p += 2) {
                     float h[8], l[8];
                     tmem_ld8(tlane + kTmemU + p * 8, h);          // warp-collective
                     if (lo_pass) {
-                        tmem_ld8(tlane + kTmemU + r + p * 8, l);
+                        tmem_ld8(tlane + kTmemU + RT + p * 8, l);
                     } else {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) l[i] = 0.0f;
@@ -758,14 +807,14 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
             mbar_wait<true>(wctx, bar_rx_full, tphase, kDevClusterWaitTimeout);
             {
                 const float *rx = reinterpret_cast<const float *>(sm + plan.off_rx);
-                for (int task = e; task < rows_per * r8; task += kEpiThreads) {
-                    const int row_local = task / r8, p = task - row_local * r8;
+                for (int task = e; task < rows_per * rt8; task += kEpiThreads) {
+                    const int row_local = task / rt8, p = task - row_local * rt8;
                     float u[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) u[i] = 0.0f;
                     for (int src = 0; src < C; ++src) {
-                        const float4 a = *reinterpret_cast<const float4 *>(rx + (src * rows_per + row_local) * r + p * 8);
-                        const float4 b = *reinterpret_cast<const float4 *>(rx + (src * rows_per + row_local) * r + p * 8 + 4);
+                        const float4 a = *reinterpret_cast<const float4 *>(rx + (src * rows_per + row_local) * RT + p * 8);
+                        const float4 b = *reinterpret_cast<const float4 *>(rx + (src * rows_per + row_local) * RT + p * 8 + 4);
                         u[0] += a.x; u[1] += a.y; u[2] += a.z; u[3] += a.w;
                         u[4] += b.x; u[5] += b.y; u[6] += b.z; u[7] += b.w;
                     }
@@ -779,10 +828,12 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                         zl[q] = pack2_bf16(z0 - h0, z1 - h1);
                     }
                     const int grow = (int)crank * rows_per + row_local;          // row within the tile
-                    const uint32_t off = (uint32_t)((grow >> 3) * (kt8 * 128) + p * 128 + (grow & 7) * 16);
+                    const int env = (L == 1) ? 0 : p / r8, pe = p - env * r8;
+                    const uint32_t off = (uint32_t)(env * 2 * plan.z_bytes + (grow >> 3) * (kt8 * 128) + pe * 128 + (grow & 7) * 16);
                     for (int dst = 0; dst < C; ++dst) {
-                        st_cluster_v4(mapa(sm_base + plan.off_zhi, dst) + off, zh[0], zh[1], zh[2], zh[3]);
-                        st_cluster_v4(mapa(sm_base + plan.off_zlo, dst) + off, zl[0], zl[1], zl[2], zl[3]);
+                        const uint32_t zb = mapa(sm_base + plan.off_z, dst) + off;
+                        st_cluster_v4(zb, zh[0], zh[1], zh[2], zh[3]);
+                        st_cluster_v4(zb + plan.z_bytes, zl[0], zl[1], zl[2], zl[3]);
                     }
                     asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");
                     for (int dst = 0; dst < C; ++dst) mbar_arrive_remote(mapa(bar_z_full, dst));
@@ -809,7 +860,53 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                 tc_fence_after();
                 uint8_t *ytile = sm + s * plan.slot_stride;
                 const float *so = reinterpret_cast<const float *>(ytile + plan.slot_data);
-                if (warp_has_rows) {
+                if (warp_has_rows && L == 2) {
+                    // two envelopes: y += s_out[0] * V_0 + s_out[1] * V_1, 16 columns at a time
+#pragma unroll
+                    for (int qq = 0; qq < 4; ++qq) {
+                        uint32_t v0[16], v1[16];
+                        tmem_ld16(tlane + kTmemV + (2 * vb) * kChunk + qq * 16, v0);       // warp-collective
+                        tmem_ld16(tlane + kTmemV + (2 * vb + 1) * kChunk + qq * 16, v1);
+                        tmem_wait_ld();
+                        if (qq == 3) {
+                            tc_fence_before();
+                            mbar_arrive(bar_v_empty(vb));
+                        }
+                        if (row_valid) {
+#pragma unroll
+                            for (int q = 0; q < 2; ++q) {
+                                const int ch = qq * 2 + q;                     // 16-byte chunk of the row
+                                uint4 *py = reinterpret_cast<uint4 *>(ytile + row * 128 + ((ch ^ (row & 7)) * 16));
+                                const uint4 yv = *py;
+                                const float4 s0 = *reinterpret_cast<const float4 *>(so + ch * 8);
+                                const float4 s1 = *reinterpret_cast<const float4 *>(so + ch * 8 + 4);
+                                const float4 t0 = *reinterpret_cast<const float4 *>(so + kChunk + ch * 8);
+                                const float4 t1 = *reinterpret_cast<const float4 *>(so + kChunk + ch * 8 + 4);
+                                const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
+                                const float sc0[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                                const float sc1[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+                                uint32_t ow[4];
+#pragma unroll
+                                for (int k2 = 0; k2 < 4; ++k2) {
+                                    float y0, y1;
+                                    if (half_io) {
+                                        const float2 yf = unpack2_f16(yw[k2]);
+                                        y0 = yf.x; y1 = yf.y;
+                                    } else {
+                                        y0 = __uint_as_float(yw[k2] << 16);
+                                        y1 = __uint_as_float(yw[k2] & 0xffff0000u);
+                                    }
+                                    float o0 = fmaf(sc0[2 * k2], __uint_as_float(v0[q * 8 + 2 * k2]), y0);
+                                    float o1 = fmaf(sc0[2 * k2 + 1], __uint_as_float(v0[q * 8 + 2 * k2 + 1]), y1);
+                                    o0 = fmaf(sc1[2 * k2], __uint_as_float(v1[q * 8 + 2 * k2]), o0);
+                                    o1 = fmaf(sc1[2 * k2 + 1], __uint_as_float(v1[q * 8 + 2 * k2 + 1]), o1);
+                                    ow[k2] = half_io ? pack2_f16(o0, o1) : pack2_bf16(o0, o1);
+                                }
+                                *py = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                            }
+                        }
+                    }
+                } else if (warp_has_rows) {
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
                         uint32_t v[32];
@@ -885,7 +982,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols(L)) : "memory");
     }
     if (!B.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
@@ -929,23 +1026,31 @@ struct LaunchShape { int cluster, tile_rows, slots, smem, max_clusters; };
 
 constexpr int kMaxSlots = 32;
 
-// Co-resident clusters for a cluster size and shared-memory footprint (cached: the query is slow).
-int max_active_clusters(int cluster, int smem)
+const void *kernel_for(int ell)
+{
+    return ell == 2 ? reinterpret_cast<const void *>(&tc_forward_kernel<2>)
+                    : reinterpret_cast<const void *>(&tc_forward_kernel<1>);
+}
+
+// Co-resident clusters for an instantiation, a cluster size and a shared-memory footprint (cached:
+// the query is slow).
+int max_active_clusters(int ell, int cluster, int smem)
 {
     static std::mutex mu;
-    static int cache_cluster[64], cache_smem[64], cache_val[64], n_cached = 0;
+    static int cache_ell[64], cache_cluster[64], cache_smem[64], cache_val[64], n_cached = 0;
     static bool attr_set = false;
     std::lock_guard<std::mutex> lock(mu);
     if (!attr_set) {
-        if (cudaFuncSetAttribute(tc_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemBudget) != cudaSuccess) {
-            cudaGetLastError();
-            return 0;
-        }
+        for (int l = 1; l <= kMaxTcEll; ++l)
+            if (cudaFuncSetAttribute(kernel_for(l), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return 0;
+            }
         attr_set = true;
     }
     for (int i = 0; i < n_cached; ++i)
-        if (cache_cluster[i] == cluster && cache_smem[i] == smem) return cache_val[i];
+        if (cache_ell[i] == ell && cache_cluster[i] == cluster && cache_smem[i] == smem) return cache_val[i];
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(cluster, 1, 1);
@@ -956,11 +1061,12 @@ int max_active_clusters(int cluster, int smem)
     attr.val.clusterDim.x = cluster; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr; cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, tc_forward_kernel, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, kernel_for(ell), &cfg) != cudaSuccess) {
         cudaGetLastError();
         n = 0;
     }
     if (n_cached < 64) {
+        cache_ell[n_cached] = ell;
         cache_cluster[n_cached] = cluster; cache_smem[n_cached] = smem; cache_val[n_cached] = n;
         ++n_cached;
     }
@@ -968,15 +1074,15 @@ int max_active_clusters(int cluster, int smem)
 }
 
 // Deepest ring that fits next to the fixed buffers, and how many clusters can be co-resident.
-bool plan_launch(int r, int kp, int cluster, int tile_rows, LaunchShape *out)
+bool plan_launch(int r, int kp, int ell, int cluster, int tile_rows, LaunchShape *out)
 {
     int slots = 0;
     for (int s = kMaxSlots; s >= 2; --s) {
-        if (make_plan(r, kp, s, tile_rows, cluster).total + 1024 <= kSmemBudget) { slots = s; break; }
+        if (make_plan(r, kp, s, tile_rows, cluster, ell).total + 1024 <= kSmemBudget) { slots = s; break; }
     }
     if (slots < 2) return false;
-    const int smem = make_plan(r, kp, slots, tile_rows, cluster).total + 1024;
-    const int n = max_active_clusters(cluster, smem);
+    const int smem = make_plan(r, kp, slots, tile_rows, cluster, ell).total + 1024;
+    const int n = max_active_clusters(ell, cluster, smem);
     if (n < 1) return false;
     out->cluster = cluster; out->tile_rows = tile_rows; out->slots = slots; out->smem = smem;
     out->max_clusters = n;
@@ -988,14 +1094,15 @@ bool plan_launch(int r, int kp, int cluster, int tile_rows, LaunchShape *out)
 // the feature axes over a cluster and by shortening the tile; many tokens use tall tiles and small
 // clusters.
 template <typename TilesFor>
-bool choose_shape(int r, int kp, int64_t tokens, int64_t full_tiles, int min_chunks, TilesFor tiles_for, LaunchShape *best)
+bool choose_shape(int r, int kp, int ell, int64_t tokens, int64_t full_tiles, int min_chunks, TilesFor tiles_for,
+                  LaunchShape *best)
 {
     double best_cost = 1e300;
     bool found = false;
     // Plenty of full-height tiles (two waves or more): no cluster, nothing to exchange.
     {
         LaunchShape solo;
-        if (plan_launch(r, kp, 1, kTileM, &solo) && full_tiles >= 2 * (int64_t)solo.max_clusters) {
+        if (plan_launch(r, kp, ell, 1, kTileM, &solo) && full_tiles >= 2 * (int64_t)solo.max_clusters) {
             *best = solo;
             return true;
         }
@@ -1003,7 +1110,7 @@ bool choose_shape(int r, int kp, int64_t tokens, int64_t full_tiles, int min_chu
     for (int c = 8; c >= 1; c /= 2) {
         if (c > min_chunks) continue;
         LaunchShape probe;
-        if (!plan_launch(r, kp, c, kTileM, &probe)) continue;
+        if (!plan_launch(r, kp, ell, c, kTileM, &probe)) continue;
         const int cap = probe.max_clusters;
         // waves of `cap` clusters needed with full-height tiles, then the tile height that fills them
         const int64_t waves = (full_tiles + cap - 1) / cap;
@@ -1012,7 +1119,7 @@ bool choose_shape(int r, int kp, int64_t tokens, int64_t full_tiles, int min_chu
         if (rows > kTileM) rows = kTileM;
         if (rows < c) rows = c;
         LaunchShape shape;
-        if (!plan_launch(r, kp, c, (int)rows, &shape)) continue;
+        if (!plan_launch(r, kp, ell, c, (int)rows, &shape)) continue;
         const int64_t tiles = tiles_for(rows);
         const int64_t w = (tiles + shape.max_clusters - 1) / shape.max_clusters;
         // cost model: time ~ waves * rows of work per cluster / CTAs sharing it, plus a fixed
@@ -1029,8 +1136,12 @@ bool choose_shape(int r, int kp, int64_t tokens, int64_t full_tiles, int min_chu
 bool tc_supported(const lordba_proj &p, int64_t T, int dtype)
 {
     if ((dtype != LORDBA_BF16 && dtype != LORDBA_F16) || T < 1) return false;
-    if (((p.flags >> 8) & 0xf) != 0) return false;          // multi-envelope adapters: other kernels
-    if (p.r % 8 != 0 || p.r < 8 || p.r > kMaxRank) return false;
+    // one envelope, or two whose ranks together fit the accumulator (their scale rows travel as
+    // bulk copies too: every row must start on a 16-byte boundary)
+    const int ell = ((p.flags >> 8) & 0xf) + 1;
+    if (ell > kMaxTcEll) return false;
+    if (p.r % 8 != 0 || p.r < 8 || ell * p.r > kMaxRank) return false;
+    if (ell > 1 && (p.d_in % 4 || p.d_out % 4)) return false;
     if (p.d_in < kChunk || p.d_out < kChunk) return false;
     if (p.d_in > (1 << 30) || p.d_out > (1 << 30) || T > (1 << 30)) return false;
     if (reinterpret_cast<uintptr_t>(p.x) % 16 || reinterpret_cast<uintptr_t>(p.y) % 16) return false;
@@ -1061,10 +1172,12 @@ int launch_forward_tc(const lordba_proj *projs, const int64_t *tokens, int64_t T
             sms = v;
     }
 
-    // one launch per element / scale kind, rank value and kMaxTcBatch projections
+    auto ell_of = [](const lordba_proj &q) { return ((q.flags >> 8) & 0xf) + 1; };
+    // one launch per element / scale kind, envelope count, rank value and kMaxTcBatch projections
     int16_t all[kMaxCallProjs];
     for (int io = (dtype == LORDBA_BF16 ? kIoBf16 : kIoF16); io <= (dtype == LORDBA_BF16 ? kIoBf16 : kIoF16Exact); ++io)
-    for (int r = 8; r <= kMaxRank; r += 8) {
+    for (int ell = 1; ell <= kMaxTcEll; ++ell)
+    for (int r = 8; ell * r <= kMaxRank; r += 8) {
         // all projections of this kind and rank, in order of falling cost per tile (a y chunk
         // costs about 1.7 x chunks): tiles go to the persistent CTAs round-robin in index order,
         // so a CTA's later tiles are cheaper than its earlier ones, and the last launch of the
@@ -1073,7 +1186,8 @@ int launch_forward_tc(const lordba_proj *projs, const int64_t *tokens, int64_t T
         int64_t total_full_tiles = 0;
         for (int i = 0; i < n; ++i) {
             const int64_t rows = rows_of(tokens, T, i);
-            if (rows > 0 && projs[i].r == r && io_of(projs[i]) == io && fsel.family(projs[i], rows) == LORDBA_VARIANT_TC) {
+            if (rows > 0 && projs[i].r == r && ell_of(projs[i]) == ell && io_of(projs[i]) == io &&
+                fsel.family(projs[i], rows) == LORDBA_VARIANT_TC) {
                 all[total++] = (int16_t)i;
                 total_full_tiles += (rows + kTileM - 1) / kTileM;
             }
@@ -1130,7 +1244,7 @@ int launch_forward_tc(const lordba_proj *projs, const int64_t *tokens, int64_t T
                 for (int k = 0; k < m; ++k) t += (rows_of(tokens, T, all[first + k]) + tile_rows - 1) / tile_rows;
                 return t;
             };
-            if (!choose_shape(r, kp, tok_sum, full_tiles, min_chunks, tiles_for, &shape)) return LORDBA_ECUDA;
+            if (!choose_shape(r, kp, ell, tok_sum, full_tiles, min_chunks, tiles_for, &shape)) return LORDBA_ECUDA;
 
             TcBatch b;
             std::memset(&b, 0, sizeof(b));
@@ -1154,6 +1268,7 @@ int launch_forward_tc(const lordba_proj *projs, const int64_t *tokens, int64_t T
             b.n_proj = m;
             b.total_tiles = (int)tile_count;
             b.r = r;
+            b.ell = ell;
             b.kp = kp;
             b.io = io;
             b.status = status;
@@ -1169,7 +1284,7 @@ int launch_forward_tc(const lordba_proj *projs, const int64_t *tokens, int64_t T
 
             LaunchRec rec;
             std::memset(&rec, 0, sizeof(rec));
-            rec.func = reinterpret_cast<const void *>(&tc_forward_kernel);
+            rec.func = kernel_for(ell);
             rec.grid[0] = (unsigned)(n_clusters * shape.cluster); rec.grid[1] = 1; rec.grid[2] = 1;
             rec.block = kThreads;
             rec.smem = (uint32_t)shape.smem;

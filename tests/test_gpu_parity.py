@@ -431,6 +431,68 @@ def test_multi_envelope_forward(oracle, dtype, T, d_in, d_out, r, ell):
     assert_close(torch_to_f64(d.y), want, dtype, "ell=%d r=%d %s" % (ell, r, dtype))
 
 
+TC_ELL_SHAPES = [
+    # T, d_in, d_out, r  (two envelopes; ell * r <= 64).  Few tokens: the feature axes are split over a
+    # cluster and the partial sums of both envelopes cross it; widths that are not multiples of 64
+    # end in a ragged chunk; 2048 + 40 tokens: full tiles, one CTA per tile, and a short last tile
+    (300, 1024, 768, 32), (70, 256, 192, 8), (200, 512, 512, 24), (130, 1000, 520, 16), (1, 512, 512, 32),
+    (2048 + 40, 4096, 1024, 32), (1500, 1024, 4096, 16),
+]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16", "f16-exact"])
+@pytest.mark.parametrize("T,d_in,d_out,r", TC_ELL_SHAPES)
+def test_two_envelopes_on_the_tcgen05_kernel(oracle, dtype, T, d_in, d_out, r):
+    """Two-envelope adapters (Def. 1 / Eq. 4) with the tcgen05 kernel pinned: every element against the
+    oracle, in bfloat16, in float16, and in float16 with input scales that are float16 values."""
+    io = "bf16" if dtype == "bf16" else "f16"
+    if io != "bf16" and T > 1000:
+        pytest.skip("full-size cases are checked in bf16 only")
+    base, s_in, s_r, s_out = _ell_inputs(d_in, d_out, r, T, io, 2, seed=400 + r + d_in % 97)
+    flags = 0
+    if dtype == "f16-exact":
+        s_in = s_in.astype(np.float16).astype(np.float32)
+        flags = lordba.PROJ_SCALES_F16
+    d = DeviceProj(base)
+    t_in, t_r, t_out = (torch.from_numpy(v).to(d.x.device) for v in (s_in, s_r, s_out))
+    p = lordba.make_proj(d.x, d.packed_A, d.packed_B, t_in, t_r, t_out, d.y, r, flags)
+    code = lordba.BF16 if io == "bf16" else lordba.F16
+    lordba.set_variant(lordba.VARIANT_TC)
+    assert lordba.query_variant([p], T, code) == [lordba.VARIANT_TC]
+    n0 = lordba.launch_count()
+    lordba.adapter_forward_batched([p], T, code)
+    assert lordba.launch_count() - n0 == 1
+    want = oracle.adapter_forward_ell(base.x_f64(), base.A_sign, base.B_sign, s_in.astype(np.float64),
+                                      s_r.astype(np.float64), s_out.astype(np.float64), base.y_f64())
+    assert_close(torch_to_f64(d.y), want, io, "tcgen05 ell=2 r=%d %s" % (r, dtype))
+    assert lordba.device_status() == 0
+
+
+def test_two_envelope_segments_and_mixed_counts_on_the_tcgen05_kernel(oracle):
+    """One pinned tcgen05 call with per-projection token counts whose projections have one and two
+    envelopes at several ranks: one launch per (envelope count, rank), every element checked."""
+    specs = [(1024, 512, 32, 2, 300), (1024, 512, 32, 1, 77), (512, 768, 16, 2, 0), (768, 1024, 16, 2, 150),
+             (512, 512, 64, 1, 130), (1024, 1024, 8, 2, 200)]
+    T = max(t for *_, t in specs)
+    devs, wants, keep = [], [], []
+    for i, (d_in, d_out, r, ell, rows) in enumerate(specs):
+        base, s_in, s_r, s_out = _ell_inputs(d_in, d_out, r, T, "bf16", ell, seed=760 + i)
+        d = DeviceProj(base)
+        ts = [torch.from_numpy(v if ell > 1 else v[0]).to(d.x.device) for v in (s_in, s_r, s_out)]
+        keep.append(ts)
+        devs.append((d, lordba.make_proj(d.x, d.packed_A, d.packed_B, ts[0], ts[1], ts[2], d.y, r)))
+        want = base.y_f64().copy()
+        want[:rows] = oracle.adapter_forward_ell(base.x_f64()[:rows], base.A_sign, base.B_sign, s_in.astype(np.float64),
+                                                 s_r.astype(np.float64), s_out.astype(np.float64), base.y_f64()[:rows])
+        wants.append(want)
+    lordba.set_variant(lordba.VARIANT_TC)
+    n0 = lordba.launch_count()
+    lordba.adapter_forward_segments([p for _, p in devs], [t for *_, t in specs], lordba.BF16)
+    assert lordba.launch_count() - n0 == 5          # (2,32) (1,32) (2,16) (1,64) (2,8); the empty one launches nothing
+    for (d, _), want, spec in zip(devs, wants, specs):
+        assert_close(torch_to_f64(d.y), want, "bf16", "tcgen05 segments %s" % (spec,))
+
+
 def test_multi_envelope_batched_with_mixed_envelope_counts(oracle):
     """One batched call whose projections differ in envelope count and rank: one launch per kind,
     every element against the oracle; and the zero-envelope embedding (an extra envelope with
@@ -738,6 +800,12 @@ def test_query_variant_shows_the_fallbacks():
     p = lordba.make_proj(x, d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, y, 64)
     assert lordba.query_variant([p], 4096, lordba.BF16) == [lordba.VARIANT_TC]      # 32 tiles of 128 tokens
     assert lordba.query_variant([p], [2048], lordba.BF16) == [lordba.VARIANT_MMA]
+    # two envelopes at rank 32 count as rank 64: the same rule
+    two = lambda v: torch.stack([v, v]).contiguous()
+    d32 = DeviceProj(workloads.make_projection(1024, 512, 32, 1, "bf16", seed=6))
+    p2 = lordba.make_proj(x, d32.packed_A, d32.packed_B, two(d32.s_in), two(d32.s_r), two(d32.s_out), y, 32)
+    assert lordba.query_variant([p2], 4096, lordba.BF16) == [lordba.VARIANT_TC]
+    assert lordba.query_variant([p2], [2048], lordba.BF16) == [lordba.VARIANT_MMA]
     lordba.set_variant(lordba.VARIANT_TC)
     with pytest.raises(lordba.LordbaError) as e:
         lordba.query_variant([f32.proj()], T, lordba.F32)      # a pinned family that cannot take the call

@@ -66,10 +66,7 @@ constexpr int kMaxTcBatch = 96;          // 96 x 320 bytes of descriptors: insid
 constexpr int kMaxTcEll = 2;            // envelopes per adapter this kernel takes (ell * r <= kMaxRank)
 constexpr int kTmemU = 0;               // stage-1 accumulator columns [0, 2 ell r)
 constexpr int kTmemV = 128;             // stage-2 accumulators: two buffers of ell x 64 columns
-// z = s_r * u of a lone CTA (no cluster) lives in TMEM too, behind the stage-2 accumulators: per
-// envelope kp / 2 columns of bf16 pairs for the hi parts, then as many for the lo parts
-__host__ __device__ inline uint32_t tmem_z_col(int ell) { return (uint32_t)(kTmemV + 2 * ell * 64); }
-constexpr uint32_t kTmemCols = 512;     // one CTA per SM: all of it
+__host__ __device__ inline uint32_t tmem_cols(int ell) { return ell > 1 ? 512u : 256u; }
 constexpr int kSmemBudget = 227 * 1024;
 
 // Element type of x and y, and how s_in enters the first product (same meaning as in the
@@ -148,8 +145,7 @@ __host__ __device__ inline SmemPlan make_plan(int r, int kp, int slots, int tile
     s.off_ops = slots * s.slot_stride;
     s.z_bytes = (kTileM / 8) * (kp / 8) * 128;
     s.off_z = s.off_ops + kOps * s.op_bytes;
-    // (a lone CTA keeps z in TMEM; with a cluster z arrives from the owners of its rows, in shared memory)
-    s.off_rx = s.off_z + (cluster > 1 ? 2 * ell * s.z_bytes : 0);
+    s.off_rx = s.off_z + 2 * ell * s.z_bytes;
     // the exchange buffer for partial u exists only when a cluster splits the feature axes
     s.off_bar = s.off_rx + (cluster > 1 ? kTileM * ell * r * 4 : 0);
     s.off_misc = s.off_bar + (3 * slots + 2 * kOps + 8) * 8;
@@ -303,16 +299,6 @@ __device__ __forceinline__ void mma_bf16_words(uint32_t d_tmem, uint32_t a_lo, u
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}"
                  ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
-// the same with the A operand in tensor memory (row m in lane m, elements 2c and 2c+1 of the K axis
-// in 32-bit column c)
-__device__ __forceinline__ void mma_bf16_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
-                                                uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile("{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %5, 0;\n"
-                 "mov.b64 db, {%2, %3};\n"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}"
-                 ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
-}
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -346,13 +332,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t r[16])
                    "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
                  : "r"(taddr));
 }
-// four 32-bit columns of this warp's 32 lanes (lane = thread), warp-collective
-__device__ __forceinline__ void tmem_st4(uint32_t taddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
-                 ::"r"(taddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
@@ -480,31 +459,18 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+                     ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols(L)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // stage-2 A operands start as zeros (K padding beyond r and rows beyond tile_rows stay zero)
-    if (C > 1)
-        for (int i = tid; i < 2 * L * plan.z_bytes / 16; i += kThreads)
-            reinterpret_cast<uint4 *>(sm + plan.off_z)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < 2 * L * plan.z_bytes / 16; i += kThreads)
+        reinterpret_cast<uint4 *>(sm + plan.off_z)[i] = make_uint4(0, 0, 0, 0);
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     cluster_sync_all();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_z = tmem_base + tmem_z_col(L);
-    if (C == 1 && kp > r && warp >= 2 + kGenThreads / 32) {
-        // K padding of z (ranks r .. kp-1) in TMEM: zero once; nothing writes it afterwards
-        const uint32_t zl = tmem_z + ((uint32_t)((warp & 3) * 32) << 16);
-        for (int e = 0; e < L; ++e)
-            for (int pe = r8; pe < kt8; ++pe) {
-                tmem_st4(zl + e * kp + pe * 4, 0u, 0u, 0u, 0u);
-                tmem_st4(zl + e * kp + kp / 2 + pe * 4, 0u, 0u, 0u, 0u);
-            }
-        tmem_wait_st();
-        tc_fence_before();
-    }
     if (B.wait_prev) {
         // nothing before this line touched global memory
         asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -518,7 +484,17 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     uint32_t vit = 0;       // stage-2 chunk counter (TMEM accumulator double buffer)
     uint32_t tile_n = 0;    // tiles done by this cluster (phase of the per-tile barriers)
 
-    for (int item = cid; item < B.total_tiles; item += n_clusters, ++tile_n) {
+    // The launch's tiles are in order of falling cost and go to the clusters round-robin, wave by
+    // wave: after the full waves cluster 0 carries the most and the last cluster the least, so
+    // the last wave (the cheapest tiles, often a partial wave) is dealt from the other end.  Only
+    // for three to five waves: with two the ends carry the same, and with many (the launches of a
+    // full model's call, which also hand their SMs to the next launch as they finish) it measured
+    // 1 - 2 % behind.
+    const int last_wave = (B.total_tiles - 1) / n_clusters;
+    const bool deal_back = last_wave > 1 && last_wave <= 4;
+    for (int wave = 0; wave <= last_wave; ++wave, ++tile_n) {
+        const int item = wave * n_clusters + ((wave == last_wave && deal_back) ? n_clusters - 1 - cid : cid);
+        if (item >= B.total_tiles) break;
         // the projection of this tile: the last one whose first tile is not beyond it (a binary
         // search, seven uniform constant loads; a linear walk through the large parameter block was
         // measured at 6 % of a tile's time)
@@ -639,19 +615,6 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
 #pragma unroll
                         for (int e = 0; e < L; ++e) {
                             const uint32_t d = tmem_base + kTmemV + (vb * L + e) * kChunk;
-                            if (C == 1) {
-                                // z in TMEM: 8 columns per K step of 16
-                                const uint32_t zh_t = tmem_z + e * kp, zl_t = zh_t + kp / 2;
-#pragma unroll
-                                for (int ks = 0; ks < kMaxRank / 16; ++ks)
-                                    if (ks < ksteps2)
-                                        mma_bf16_tmem_a(d, zh_t + 8u * ks, b_lo + 16u * ks, z_hi, idesc2, ks > 0 ? 1u : 0u);
-#pragma unroll
-                                for (int ks = 0; ks < kMaxRank / 16; ++ks)
-                                    if (ks < ksteps2)
-                                        mma_bf16_tmem_a(d, zl_t + 8u * ks, b_lo + 16u * ks, z_hi, idesc2, 1u);
-                                continue;
-                            }
                             const uint32_t zh_lo = zhi_lo + 2u * e * z_units, zl_lo = zh_lo + z_units;
 #pragma unroll
                             for (int ks = 0; ks < kMaxRank / 16; ++ks)
@@ -803,26 +766,23 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
                             for (int i = 0; i < 8; ++i) l[i] = 0.0f;
                         }
                         tmem_wait_ld();
-                        // (rows past tile_rows carry whatever the padding rows of the x box gave: they
-                        // feed accumulator rows that nobody reads)
-                        uint32_t zh[4], zl[4];
+                        if (row_valid) {
+                            uint32_t zh[4], zl[4];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float z0 = (h[2 * q] + l[2 * q]) * __ldg(P.s_r + p * 8 + 2 * q);
-                            const float z1 = (h[2 * q + 1] + l[2 * q + 1]) * __ldg(P.s_r + p * 8 + 2 * q + 1);
-                            const float h0 = bf16_round(z0), h1 = bf16_round(z1);
-                            zh[q] = pack2_bf16(h0, h1);
-                            zl[q] = pack2_bf16(z0 - h0, z1 - h1);
+                            for (int q = 0; q < 4; ++q) {
+                                const float z0 = (h[2 * q] + l[2 * q]) * __ldg(P.s_r + p * 8 + 2 * q);
+                                const float z1 = (h[2 * q + 1] + l[2 * q + 1]) * __ldg(P.s_r + p * 8 + 2 * q + 1);
+                                const float h0 = bf16_round(z0), h1 = bf16_round(z1);
+                                zh[q] = pack2_bf16(h0, h1);
+                                zl[q] = pack2_bf16(z0 - h0, z1 - h1);
+                            }
+                            const int env = (L == 1) ? 0 : p / r8, pe = p - env * r8;
+                            const uint32_t off = (uint32_t)(env * 2 * plan.z_bytes + (row >> 3) * (kt8 * 128) + pe * 128 + (row & 7) * 16);
+                            *reinterpret_cast<uint4 *>(sm + plan.off_z + off) = make_uint4(zh[0], zh[1], zh[2], zh[3]);
+                            *reinterpret_cast<uint4 *>(sm + plan.off_z + plan.z_bytes + off) = make_uint4(zl[0], zl[1], zl[2], zl[3]);
+                            fence_proxy_async();
+                            mbar_arrive(bar_z_full);
                         }
-                        // ranks 8 pe .. 8 pe + 7 of envelope env = 4 columns of bf16 pairs in this
-                        // thread's TMEM lane: the A operand of stage 2 is read from there
-                        const int env = (L == 1) ? 0 : p / r8, pe = p - env * r8;
-                        const uint32_t zc = tmem_z + ((uint32_t)(quad * 32) << 16) + env * kp + pe * 4;
-                        tmem_st4(zc, zh[0], zh[1], zh[2], zh[3]);               // warp-collective
-                        tmem_st4(zc + kp / 2, zl[0], zl[1], zl[2], zl[3]);
-                        tmem_wait_st();
-                        tc_fence_before();
-                        if (row_valid) mbar_arrive(bar_z_full);
                     }
                     tc_fence_before();
                 }
@@ -1032,7 +992,7 @@ tc_forward_kernel(const __grid_constant__ TcBatch B)
     cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols(L)) : "memory");
     }
     if (!B.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
 }

@@ -812,6 +812,23 @@ def test_query_variant_shows_the_fallbacks():
     assert e.value.status == 2
 
 
+def test_tcgen05_last_wave_dealt_from_the_other_end(oracle):
+    """A launch of between three and five waves of tiles deals its last wave to the persistent CTAs
+    in reverse order: 148 * 3 + 40 tiles of 128 tokens and a short one, two projections of
+    different cost, every element against the oracle (a tile done twice or not at all would show)."""
+    T = 128 * (74 * 3 + 20) + 5
+    projs = [workloads.make_projection(512, 256, 64, T, "bf16", seed=9100),
+             workloads.make_projection(256, 256, 64, T, "bf16", seed=9101)]
+    devs = [DeviceProj(p) for p in projs]
+    lordba.set_variant(lordba.VARIANT_TC)
+    n0 = lordba.launch_count()
+    lordba.adapter_forward_batched([d.proj() for d in devs], T, lordba.BF16)
+    assert lordba.launch_count() - n0 == 1
+    for p, d in zip(projs, devs):
+        assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16", "tcgen05 four waves " + str(p.meta["seed"]))
+    assert lordba.device_status() == 0
+
+
 @pytest.mark.parametrize("r", [32, 64])
 @pytest.mark.parametrize("pin", [False, True])
 def test_segments_on_the_tcgen05_kernel(oracle, r, pin):

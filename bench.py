@@ -521,9 +521,10 @@ def run_gpu(args):
     # Consecutive steps work on different buffer sets, so every step but the first of a graph is
     # declared independent of the ones before it (LORDBA_PROJ_OVERLAP): its loads may start while
     # the previous step's last tiles are still being written.
-    def step(i, dependent=False):
+    def step(i, dependent=False, x_ready=False):
         lordba.adapter_forward(xs[i % n_sets], packed_A, packed_B, s_in, s_r, s_out, ys[i % n_sets], R,
-                               overlap=(i % n_sets != 0) and not args.no_overlap and not dependent)
+                               overlap=(i % n_sets != 0) and not args.no_overlap and not dependent,
+                               x_ready=x_ready)
 
     # correctness of the configuration being timed: sampled rows against the oracle (rank 0)
     parity = None
@@ -588,6 +589,11 @@ def run_gpu(args):
         dep_region = timed(dep, args.steps, args.warmup)
         sampler.recording = False
         dep_ms = float(np.median(dep_region)) / args.steps
+        # and the chain an adapter call sits in inside a model: it follows the base projection
+        # that produced y, while x (the base projection's own input) and the adapter were final
+        # before that: LORDBA_PROJ_X_READY on every step, no step declared independent
+        depx = GraphSteps(lambda i: step(i, dependent=True, x_ready=True), n_sets, stream)
+        depx_ms = float(np.median(timed(depx, args.steps, args.warmup))) / args.steps
 
         # the same independent steps issued one by one from the host, no graph: a prepared call
         # (tensor maps encoded once) against the plain entry point, in microseconds per call
@@ -678,6 +684,10 @@ def run_gpu(args):
             "dependent_steps": {"ms_per_step": dep_ms, "value": world * T / (dep_ms * 1e-3), "unit": UNIT,
                                 "roofline_frac": alg_bytes / (dep_ms * 1e-3) / 1e9 / peak,
                                 "steps": args.steps, "repeats": int(len(dep_region))},
+            "dependent_steps_x_ready": {"ms_per_step": depx_ms, "unit": UNIT, "value": world * T / (depx_ms * 1e-3),
+                                        "roofline_frac": alg_bytes / (depx_ms * 1e-3) / 1e9 / peak,
+                                        "promise": "LORDBA_PROJ_X_READY: every call waits for the previous one "
+                                                   "before it touches y; x and the adapter were final earlier"},
             "eager_calls": eager,
         }
         if extra is not None:

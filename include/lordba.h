@@ -103,7 +103,7 @@ typedef struct lordba_proj {
     void           *y;          /* [device] T x d_out, pitch ldy, updated in place */
     int64_t d_in, d_out, ldx, ldy;
     int32_t r;
-    int32_t flags;              /* LORDBA_PROJ_OVERLAP, LORDBA_PROJ_SCALES_F16, LORDBA_PROJ_ELL(ell); other bits 0 */
+    int32_t flags;              /* LORDBA_PROJ_OVERLAP, _X_READY, _SCALES_F16, LORDBA_PROJ_ELL(ell); other bits 0 */
 } lordba_proj;
 
 /*
@@ -133,6 +133,19 @@ typedef struct lordba_proj {
  * kernel acts on the flag; elsewhere it is accepted and ignored.
  */
 #define LORDBA_PROJ_OVERLAP 1
+
+/*
+ * lordba_proj.flags: a weaker promise for a call that does depend on its predecessor, as an
+ * adapter call does that follows the base projection which produced y (Eq. 2: y = W x, then
+ * y += Delta-W x).  With LORDBA_PROJ_X_READY on every projection of a call made WITHOUT
+ * LORDBA_PROJ_OVERLAP the caller guarantees that x, the packed carriers and the three scale
+ * vectors were final before the previous piece of work on the stream began (the base projection
+ * reads x itself, so this is the normal case); only y may still be in the making.  The call then
+ * requests x and runs the first product (Eq. 8, u = A_sign (s_in * x)) while its predecessor
+ * finishes, and touches y only once the predecessor is complete.  Only the streaming kernel acts
+ * on the flag; elsewhere, and together with LORDBA_PROJ_OVERLAP, it is accepted and ignored.
+ */
+#define LORDBA_PROJ_X_READY 4
 
 /*
  * lordba_proj.flags: the caller states that every entry of s_in is exactly representable as an

@@ -123,7 +123,7 @@ int validate_proj(const lordba_proj &p, int64_t T, int dtype)
 {
     if (!known_dtype(dtype)) return LORDBA_EUNSUPPORTED;
     if (T < 0 || p.d_in < 1 || p.d_out < 1 || p.ldx < p.d_in || p.ldy < p.d_out) return LORDBA_EINVAL;
-    if ((p.flags & ~(LORDBA_PROJ_OVERLAP | LORDBA_PROJ_SCALES_F16 | 0xf00)) != 0) return LORDBA_EINVAL;
+    if ((p.flags & ~(LORDBA_PROJ_OVERLAP | LORDBA_PROJ_SCALES_F16 | LORDBA_PROJ_X_READY | 0xf00)) != 0) return LORDBA_EINVAL;
     if (((p.flags >> 8) & 0xf) + 1 > LORDBA_MAX_ELL) return LORDBA_EUNSUPPORTED;
     if (p.r < 1 || p.r > kMaxRank) return LORDBA_EUNSUPPORTED;
     if (T == 0) return LORDBA_OK;   // nothing is touched: the pointers may be anything

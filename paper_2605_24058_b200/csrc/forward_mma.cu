@@ -111,6 +111,9 @@ struct MmaParams {
     int slots;         // ring depth
     int wait_prev;     // 1: the previous kernel of the stream must be complete before any global access
     int skip_item;     // -1; the test-hooks build can name one item whose copy request is left out
+    int x_ready;       // 1 (only with wait_prev): x and the adapter were final before the previous kernel began,
+                       // so the x items are requested and the first product runs before the wait for it;
+                       // y is touched only afterwards
     int gate_y;        // g > 0: the y items that fit the ring at the start are requested only once x item
                        // g - 1 has landed, so that the x items, which the first product waits for, do not
                        // share the memory system with them from the start (0: everything is requested at once)
@@ -388,7 +391,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (prm.wait_prev) {
+        if (prm.wait_prev && !prm.x_ready) {
             // everything before this line overlapped the previous kernel; nothing after it may
             asm volatile("griddepcontrol.wait;" ::: "memory");
             asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -410,7 +413,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         tma_load_2d(slot + plan.off_bits, is_x ? &P.pa_map : &P.pb_map, 0, col0 * r / 512, bar_full(s));
     };
     const int n_first = n_items < S ? n_items : S;
-    const int n_eager = (prm.gate_y && n_xi < n_first) ? n_xi : n_first;
+    const int n_eager = ((prm.gate_y || prm.x_ready) && n_xi < n_first) ? n_xi : n_first;
     if (tid == kConsumerThreads)
         for (int it = 0; it < n_eager; ++it) issue_item(it, it);     // n_eager <= n_first <= S
     __syncthreads();
@@ -421,6 +424,12 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             // item n_first is the first to reuse a slot: slot 0, first release phase
             int s = 0;
             uint32_t eph = 0;
+            if (prm.x_ready) {
+                // what was requested so far is x and the adapter; from here on y, which the
+                // previous kernel may have written: wait for it, then let the successor in
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+            }
             if (n_eager < n_first &&
                 mbar_wait(wctx, bar_full(prm.gate_y - 1 < n_eager ? prm.gate_y - 1 : n_eager - 1), 0u, kDevTmaWaitTimeout))
                 for (int it = n_eager; it < n_first; ++it) issue_item(it, it);
@@ -607,6 +616,8 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         // A wait that gave up during the first product left u incomplete: this CTA then writes
         // nothing (its rows of y keep their old values) and only drains its items.
         const bool u_complete = !__any_sync(0xffffffffu, *abort_flag != 0);
+        // (every thread that is going to write y has seen the previous kernel complete)
+        if (prm.x_ready) asm volatile("griddepcontrol.wait;" ::: "memory");
         uint16_t *yrow0 = P.y + (t0 + g) * P.ldy;
         uint16_t *yrow1 = yrow0 + 8 * P.ldy;
         const bool vec32 = P.y_vec32 != 0;
@@ -970,6 +981,9 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 // and fewer, fuller CTAs leave room for the neighbouring calls' CTAs.
                 const int64_t rows = kTile;
                 const bool overlaps_neighbours = (*launches == 0) ? all_overlap : batch_checked;
+                // the first launch of a call that waits for its predecessor may still start on x
+                bool x_ready = !overlaps_neighbours && *launches == 0;
+                for (int k = 0; k < m; ++k) x_ready = x_ready && (sel[k]->flags & LORDBA_PROJ_X_READY);
                 int64_t tiles = 0, all_tiles = 0;      // widest projection (grid.x), and the sum
                 for (int k = 0; k < m; ++k) {
                     const int64_t tk = (sel_T[k] + rows - 1) / rows;
@@ -1019,6 +1033,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 std::memset(&prm, 0, sizeof(prm));
                 prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
                 prm.wait_prev = !overlaps_neighbours;
+                prm.x_ready = x_ready;
                 prm.skip_item = test_skip_item();
                 prm.gate_y = prm.wait_prev ? 2 : 0;   // (measured: a call that waits for its predecessor, 12.1 -> 11.8 us; later items lose it again)
                 prm.ell = ell;

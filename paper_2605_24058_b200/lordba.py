@@ -20,6 +20,7 @@ F32, BF16, F16 = 0, 1, 2
 VARIANT_AUTO, VARIANT_FMA, VARIANT_TC, VARIANT_MMA = 0, 1, 2, 3
 PROJ_OVERLAP = 1
 PROJ_SCALES_F16 = 2
+PROJ_X_READY = 4
 MAX_ELL = 8
 MAX_PROJS = 4096
 FIT_ALPHA, FIT_BETA, FIT_GAMMA, FIT_ALL = 1, 2, 4, 7
@@ -217,12 +218,14 @@ def make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, flags: int = 0
 
 
 def adapter_forward(x, packed_A, packed_B, s_in, s_r, s_out, y, r: int, stream=None,
-                    overlap: bool = False, scales_f16: bool = False) -> None:
+                    overlap: bool = False, scales_f16: bool = False, x_ready: bool = False) -> None:
     """y += adapter(x) in place, through lordba_adapter_forward{,_f32} (dense rows)
     or lordba_adapter_forward_ex (row-strided x / y, float16, or a flag: overlap=True is the
     caller's promise LORDBA_PROJ_OVERLAP that this call is independent of the run of calls before
-    it, scales_f16=True the statement LORDBA_PROJ_SCALES_F16 that s_in holds float16 values)."""
-    flags = (PROJ_OVERLAP if overlap else 0) | (PROJ_SCALES_F16 if scales_f16 else 0)
+    it, scales_f16=True the statement LORDBA_PROJ_SCALES_F16 that s_in holds float16 values,
+    x_ready=True the promise LORDBA_PROJ_X_READY that only y can still be in the making)."""
+    flags = ((PROJ_OVERLAP if overlap else 0) | (PROJ_SCALES_F16 if scales_f16 else 0) |
+             (PROJ_X_READY if x_ready else 0))
     p = make_proj(x, packed_A, packed_B, s_in, s_r, s_out, y, r, flags)
     T = x.shape[0]
     lib = load()

@@ -75,7 +75,8 @@ def test_bad_arguments_return_codes_without_launching(lib):
     assert call(_proj(lordba, d_in=0)) == EINVAL
     assert call(_proj(lordba, ldx=63)) == EINVAL
     assert call(_proj(lordba, ldy=10)) == EINVAL
-    assert call(_proj(lordba, flags=6)) == EINVAL
+    assert call(_proj(lordba, flags=8)) == EINVAL
+    assert call(_proj(lordba, flags=0x1000)) == EINVAL
     assert call(_proj(lordba, r=0)) == EUNSUP
     assert call(_proj(lordba, r=65)) == EUNSUP
     assert call(_proj(lordba), dt=9) == EUNSUP
@@ -127,7 +128,8 @@ def test_float16_arguments_and_inputs_without_launching(lib):
     assert call(_proj(lordba, flags=lordba.PROJ_SCALES_F16), T=0) == 0
     assert call(_proj(lordba, flags=lordba.PROJ_SCALES_F16 | lordba.PROJ_OVERLAP), T=0) == 0
     assert call(_proj(lordba, x=0x1001)) == EALIGN                    # 2-byte elements
-    assert call(_proj(lordba, flags=4), T=0) == EINVAL
+    assert call(_proj(lordba, flags=lordba.PROJ_X_READY), T=0) == 0
+    assert call(_proj(lordba, flags=8), T=0) == EINVAL
     assert lib.lordba_scales_from_f16(0x1000, 0x2000, -1, None) == EINVAL
     assert lib.lordba_scales_from_f16(None, 0x2000, 4, None) == EINVAL
     assert lib.lordba_scales_from_f16(0x1001, 0x2000, 4, None) == EALIGN

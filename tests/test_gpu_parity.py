@@ -532,6 +532,62 @@ def test_multi_envelope_with_one_envelope_equals_plain_call(oracle):
     assert torch.equal(a.y, b.y)
 
 
+# ---------------------------------------------------------------- the x-ready promise
+
+@pytest.mark.parametrize("T,d_in,d_out,r", [(2048, 4096, 4096, 16), (300, 1024, 768, 32), (2048, 11008, 4096, 16), (40, 512, 512, 8)])
+def test_x_ready_chain_on_one_y(oracle, T, d_in, d_out, r):
+    """LORDBA_PROJ_X_READY (Eq. 2: the adapter call follows the work that produced y): three calls
+    in a row update the SAME y from three inputs and adapters that were final beforehand, the second
+    and third with the promise, so each starts on its x while its predecessor still writes y and
+    must not touch y before that one is complete.  The result equals, bit for bit and on every one
+    of 10 rounds, that of the same chain without the promise (a call that read y early would lose an
+    update), which is checked against the oracle chain element by element."""
+    ps = [workloads.make_projection(d_in, d_out, r, T, "bf16", seed=9300 + i) for i in range(3)]
+    ds = [DeviceProj(p) for p in ps]
+    y0 = ds[0].y.clone()
+    want = ps[0].y_f64()
+    bound = np.zeros_like(want)
+    for p in ps:
+        # each call rounds y to bfloat16 once and the oracle chain does the same between the calls.
+        # Where the two sides round an intermediate y to different neighbours they leave that call
+        # a whole bfloat16 step apart (2^-7 |y|, twice the bound of a single call), and every
+        # call adds its own share, relative to what y holds after it
+        want = oracle.adapter_forward(p.x_f64(), p.A_sign, p.B_sign, p.s_in.astype(np.float64), p.s_r.astype(np.float64),
+                                      p.s_out.astype(np.float64), want)
+        bound += 2.0 ** -7 * np.abs(want) + 2.0 ** -12 * np.sqrt(np.mean(want ** 2))
+        want = torch.from_numpy(want).to(torch.bfloat16).to(torch.float64).numpy()
+
+    def chain(promise):
+        y = y0.clone()
+        torch.cuda.current_stream().synchronize()
+        for i, d in enumerate(ds):
+            lordba.adapter_forward(d.x, d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, y, r, x_ready=promise and i > 0)
+        return y
+
+    plain = chain(False)
+    for rnd in range(10):
+        assert torch.equal(chain(True), plain), "round %d differs from the chain without the promise" % rnd
+    err = np.abs(torch_to_f64(plain) - want)
+    assert np.all(err <= bound), float((err / bound).max())
+    assert lordba.device_status() == 0
+
+
+def test_x_ready_after_other_work_and_with_the_other_flags(oracle):
+    """The promise after a kernel that is not the library's (y filled by a copy just before the
+    call), on a batched call, and next to LORDBA_PROJ_OVERLAP (then ignored): every element."""
+    T = 300
+    ps = [workloads.make_projection(1024, 768, 16, T, "bf16", seed=9400 + i) for i in range(3)]
+    ds = [DeviceProj(p) for p in ps]
+    for d in ds:
+        d.y.copy_(d.y.clone())                     # y "produced" on the stream right before the call
+    flags = [lordba.PROJ_X_READY, lordba.PROJ_X_READY, lordba.PROJ_X_READY | lordba.PROJ_OVERLAP]
+    projs = [lordba.make_proj(d.x, d.packed_A, d.packed_B, d.s_in, d.s_r, d.s_out, d.y, 16, f) for d, f in zip(ds, flags)]
+    lordba.adapter_forward_batched(projs[:2], T, lordba.BF16)
+    lordba.adapter_forward_batched(projs[2:], T, lordba.BF16)
+    for p, d in zip(ps, ds):
+        assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16", "x-ready " + str(p.meta["seed"]))
+
+
 # ---------------------------------------------------------------- multi-adapter batches (segments)
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])

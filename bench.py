@@ -308,7 +308,7 @@ class DeviceWorkload:
     envelopes) over Tn tokens, n_sets rotating sets of x / y buffers, one library call per step."""
 
     def __init__(self, lordba, dev, shapes, r, Tn, ell=1, dtype="bf16", scales_f16=False, segments=0,
-                 overlap=True, seed=1234, mem_cap=40e9, shared=None):
+                 overlap=True, x_ready=False, seed=1234, mem_cap=40e9, shared=None):
         import torch
         self.torch, self.lordba = torch, lordba
         self.shapes, self.r, self.Tn, self.ell, self.segments = shapes, r, Tn, ell, segments
@@ -319,6 +319,11 @@ class DeviceWorkload:
         # an adapter exported with half-precision scales: values rounded to float16, declared to the library
         exported = (lambda s: s.to(torch.float16).to(torch.float32)) if scales_f16 else (lambda s: s)
         self.base_flags = lordba.PROJ_SCALES_F16 if scales_f16 else 0
+        # x_ready (with overlap=False): every call waits for the previous one before it touches y;
+        # x and the adapter are declared final before that (LORDBA_PROJ_X_READY)
+        self.x_ready = x_ready and not overlap
+        if self.x_ready:
+            self.base_flags |= lordba.PROJ_X_READY
 
         def rand_signs(rows, cols):
             return torch.randint(0, 2, (rows, cols), device=dev, generator=gen, dtype=torch.int8) * 2 - 1
@@ -391,7 +396,9 @@ def time_workload(w: DeviceWorkload, stream, steps: int, warmup: int, min_repeat
             "p90_us": float(np.percentile(ms, 90)) / steps * 1e3, "gbs": achieved, "frac": achieved / peak,
             "peak_kind": "of " + peak_kind, "variant": w.variant(), "launches_per_call": launches_per_step,
             "steps": steps, "repeats": int(len(ms)), "buffer_sets": w.n_sets, "alg_bytes": w.alg_bytes,
-            "step_dependency": "declared independent" if w.overlap_ok else "each call waits for the previous one"}
+            "step_dependency": "declared independent" if w.overlap_ok else
+                               "each call waits for the previous one before it touches y (x declared ready)" if w.x_ready
+                               else "each call waits for the previous one"}
 
 
 def time_fit_sweep(lordba, dev, N, M, r, sweeps=10):
@@ -469,6 +476,11 @@ def supplementary_workloads(lordba, dev, stream, sampler):
     # config 3: decode, one batched call per layer (latency bound: the figure is us per call)
     for Tn in (1, 8, 32, 64):
         run("decode_layer_T%d_r16" % Tn, 32, 8, shapes=layer, r=16, Tn=Tn)
+    # the same call as it sits in a decoding model: every call waits for the one before it (its
+    # latency, not its throughput), without and with the promise that only y is still in the making
+    for Tn in (1, 8, 64):
+        run("decode_layer_T%d_r16_dependent" % Tn, 32, 8, shapes=layer, r=16, Tn=Tn, overlap=False)
+        run("decode_layer_T%d_r16_x_ready" % Tn, 32, 8, shapes=layer, r=16, Tn=Tn, overlap=False, x_ready=True)
     # config 4: all 224 projections in one call over the rank sweep (one 15.8 GB buffer set, shared)
     shared = {}
     for r in (8, 16, 32, 64):

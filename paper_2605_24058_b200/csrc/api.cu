@@ -70,7 +70,8 @@ int launch_record(const LaunchRec &rec, const void *arg0, const void *arg1, cuda
     unsigned na = 0;
     if (rec.cluster > 1) {
         attr[na].id = cudaLaunchAttributeClusterDimension;
-        attr[na].val.clusterDim.x = rec.cluster; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        attr[na].val.clusterDim.x = rec.cluster_z ? 1 : rec.cluster; attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = rec.cluster_z ? rec.cluster : 1;
         ++na;
     }
     if (rec.pdl) {

@@ -111,6 +111,9 @@ struct MmaParams {
     int slots;         // ring depth
     int wait_prev;     // 1: the previous kernel of the stream must be complete before any global access
     int skip_item;     // -1; the test-hooks build can name one item whose copy request is left out
+    int xsplit;        // C > 1 (single-envelope launches of few tiles): the CTAs are launched as clusters of C
+                       // along grid z; CTA c of a cluster takes every x item of its share of the d_in axis
+                       // only, and the partial sums of u go round the cluster through distributed shared memory
     int x_ready;       // 1 (only with wait_prev): x and the adapter were final before the previous kernel began,
                        // so the x items are requested and the first product runs before the wait for it;
                        // y is touched only afterwards
@@ -127,13 +130,14 @@ struct SmemPlan {
     int off_scale;     // slot offset of the item's float32 scales
     int off_bits;      // slot offset of the item's sign bytes
     int slot_bytes;    // multiple of 1024 (swizzle atom)
-    int off_red, off_zh, off_zl, off_bar, total;
+    int off_red, off_zh, off_zl, off_ux, off_bar, total;
 };
 
 // nw: consumer warps = 64-column groups per item; cwy: columns of a y item
 // eg: envelopes (scale triples) per pass of the first product: eg rows of scales per x item, eg
 // partial sums; ell: all envelopes of the adapter: ell rows of scales per y item, ell z tiles
-__host__ __device__ inline SmemPlan make_plan(int nw, int rp, int r, int slots, int eg, int ell, int cwy)
+// xsplit: CTAs of a cluster that share the first product (1: none): one tile of partial u per CTA
+__host__ __device__ inline SmemPlan make_plan(int nw, int rp, int r, int slots, int eg, int ell, int cwy, int xsplit = 1)
 {
     SmemPlan s;
     s.off_scale = nw * kBlockBytes;
@@ -144,7 +148,8 @@ __host__ __device__ inline SmemPlan make_plan(int nw, int rp, int r, int slots, 
     s.off_red = slots * s.slot_bytes;
     s.off_zh = s.off_red + eg * nw * kTile * rp * 4;
     s.off_zl = s.off_zh + ell * kTile * ks * 8 * 4;
-    s.off_bar = s.off_zl + ell * kTile * ks * 8 * 4;
+    s.off_ux = s.off_zl + ell * kTile * ks * 8 * 4;
+    s.off_bar = s.off_ux + (xsplit > 1 ? xsplit * kTile * ks * 16 * 4 : 0);
     s.total = s.off_bar + (2 * kMaxSlots + 2) * 8 + 1024;    // + slack to align the base to 1 KiB
     return s;
 }
@@ -161,6 +166,30 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// ---- cluster helpers (launches whose CTAs share the first product) ----
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t v; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(v)); return v;
+}
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank)
+{
+    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f2(uint32_t addr, float a, float b)
+{
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
+// arrive on a barrier of any CTA of the cluster (address from mapa), release at cluster scope
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
 {
@@ -210,6 +239,28 @@ __device__ __forceinline__ bool mbar_wait(const WaitCtx &w, uint32_t bar, uint32
     uint32_t spins = 0;
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0) {
+            if (*w.abort_flag) return false;
+            if (clock64() - start > kWaitLimitCycles) {
+                atomicCAS(w.status, 0, code);
+                *w.abort_flag = 1;
+                return false;
+            }
+        }
+    }
+}
+
+// The same for a barrier on which other CTAs of the cluster arrive (acquire at cluster scope).
+__device__ __forceinline__ bool mbar_wait_cluster(const WaitCtx &w, uint32_t bar, uint32_t parity, int code)
+{
+    const long long start = clock64();
+    uint32_t spins = 0;
+    for (;;) {
+        uint32_t ok;
+        asm volatile("{\n.reg .pred p;\n"
+                     "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+                     "selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
         if ((++spins & 63u) == 0) {
             if (*w.abort_flag) return false;
             if (clock64() - start > kWaitLimitCycles) {
@@ -358,11 +409,17 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     const int d_in = P.d_in, d_out = P.d_out;
     const int ell = (EGT == 1) ? 1 : prm.ell;
     const int n_groups = (EGT == 1) ? 1 : (ell + EG - 1) / EG;
-    const SmemPlan plan = make_plan(NW, RP, r, S, EG, ell, cwy);
+    // CTAs of a cluster along grid z share the first product (single-envelope launches only)
+    const int xsplit = (EGT == 1) ? prm.xsplit : 1;
+    const SmemPlan plan = make_plan(NW, RP, r, S, EG, ell, cwy, xsplit);
     const uint32_t sm_base = smem_u32(smem);
 
-    // items: all x chunks (once per envelope group), then this CTA's share of the y chunks
-    const int n_x = (d_in + cwx - 1) / cwx;
+    // items: the x chunks (once per envelope group; with a cluster this CTA's share of them, a
+    // contiguous range), then this CTA's share of the y chunks
+    const int n_x_all = (d_in + cwx - 1) / cwx;
+    const int xrank = xsplit > 1 ? (int)cluster_ctarank() : 0;
+    const int x_first = (int)((int64_t)xrank * n_x_all / xsplit);
+    const int n_x = (int)((int64_t)(xrank + 1) * n_x_all / xsplit) - x_first;
     const int n_xi = n_groups * n_x;
     const int n_yc = (d_out + cwy - 1) / cwy;
     const int yc_begin = (int)((int64_t)blockIdx.z * n_yc / gridDim.z);
@@ -372,6 +429,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     const uint32_t bar0 = sm_base + plan.off_bar;
     auto bar_full = [&](int s) { return bar0 + 8u * s; };
     auto bar_empty = [&](int s) { return bar0 + 8u * (kMaxSlots + s); };
+    const uint32_t bar_ux = bar0 + 8u * (2 * kMaxSlots + 1);    // partial sums of the whole cluster have arrived
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + plan.off_bar + 2 * kMaxSlots * 8);
     const WaitCtx wctx{abort_flag, prm.status};
 
@@ -389,6 +447,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             mbar_init(bar_full(s), 1);
             mbar_init(bar_empty(s), kConsumerWarps);
         }
+        if (xsplit > 1) mbar_init(bar_ux, (uint32_t)xsplit);   // one arrival per CTA of the cluster
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (prm.wait_prev && !prm.x_ready) {
@@ -401,7 +460,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
         const bool is_x = it < n_xi;
         const int cw = is_x ? cwx : cwy;
         const int grp = is_x ? it / n_x : 0;       // the envelope group this pass over x belongs to
-        const int col0 = is_x ? (it - grp * n_x) * cwx : (yc_begin + (it - n_xi)) * cwy;
+        const int col0 = is_x ? (x_first + it - grp * n_x) * cwx : (yc_begin + (it - n_xi)) * cwy;
         // a box is always whole: what lies past the tensor (columns, envelopes) is filled with zeros and counted
         const uint32_t bytes = (uint32_t)(cw / kGroup) * kBlockBytes + (uint32_t)(is_x ? EG : ell) * cw * 4u +
                                (uint32_t)cw * r / 8u;
@@ -417,6 +476,9 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     if (tid == kConsumerThreads)
         for (int it = 0; it < n_eager; ++it) issue_item(it, it);     // n_eager <= n_first <= S
     __syncthreads();
+    // every CTA of the cluster has initialised its barriers before any of them arrives on another's
+    // (all CTAs of a cluster have the same tile and projection: none has left above)
+    if (xsplit > 1) cluster_sync_all();
 
     if (warp == kConsumerWarps) {
         // ================= producer warp: one lane refills the slots as they are released ========
@@ -431,7 +493,8 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                 asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
             }
             if (n_eager < n_first &&
-                mbar_wait(wctx, bar_full(prm.gate_y - 1 < n_eager ? prm.gate_y - 1 : n_eager - 1), 0u, kDevTmaWaitTimeout))
+                (n_eager == 0 || prm.gate_y == 0 ||
+                 mbar_wait(wctx, bar_full(prm.gate_y - 1 < n_eager ? prm.gate_y - 1 : n_eager - 1), 0u, kDevTmaWaitTimeout)))
                 for (int it = n_eager; it < n_first; ++it) issue_item(it, it);
             for (int it = n_first; it < n_items; ++it) {
                 if (!mbar_wait(wctx, bar_empty(s), eph, kDevTmaWaitTimeout)) break;
@@ -469,7 +532,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
 
         for (int xc = 0; xc < n_x; ++xc, ++it) {
             const bool ok = __all_sync(0xffffffffu, mbar_wait(wctx, bar_full(s), sph, kDevMmaWaitTimeout));
-            const int cwv = (d_in - xc * cwx < cwx) ? (d_in - xc * cwx) : cwx;
+            const int cwv = (d_in - (x_first + xc) * cwx < cwx) ? (d_in - (x_first + xc) * cwx) : cwx;
             if (gcol < cwv && ok) {
                 const uint8_t *slot = smem + s * plan.slot_bytes;
                 // this lane's columns: gcol + 16q .. +7 (piece A) and gcol + 16q + 8 .. +15 (piece B);
@@ -562,6 +625,55 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             }
         }
         consumer_sync<kConsumerThreads>();
+        if (EGT == 1 && xsplit > 1) {
+            // This CTA's sums cover its share of d_in only.  Every pair of them goes to every CTA of
+            // the cluster (its own included), followed by one arrival on that CTA's barrier; once
+            // all CTAs have arrived here, the shares are added in the order of the CTAs' ranks.
+            // A CTA whose own share is incomplete (a wait gave up) sends nothing: the others'
+            // waits then give up too, and no CTA of the cluster writes to y.
+            const bool whole = !*abort_flag;
+            const uint32_t ux0 = sm_base + plan.off_ux;
+            for (int idx = tid; idx < kTile * ZP; idx += kConsumerThreads) {
+                const int tok = idx / ZP, pr = idx - tok * ZP;
+                float u0 = 0.0f, u1 = 0.0f;
+                if (2 * pr < RP) {
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float2 v = *reinterpret_cast<const float2 *>(red + ((w * kTile + tok) * RP + 2 * pr));
+                        u0 += v.x;
+                        u1 += v.y;
+                    }
+                }
+                if (whole) {
+                    const uint32_t off = (uint32_t)(((xrank * kTile + tok) * ZP + pr) * 8);
+                    for (int dst = 0; dst < xsplit; ++dst) st_cluster_f2(mapa(ux0, dst) + off, u0, u1);
+                }
+            }
+            // all of this CTA's stores, then one arrival per destination: the fences and the
+            // barrier order every thread's stores before the arriving thread's release
+            asm volatile("fence.acq_rel.cluster;" ::: "memory");
+            consumer_sync<kConsumerThreads>();
+            if (tid == 0 && whole)
+                for (int dst = 0; dst < xsplit; ++dst) mbar_arrive_remote(mapa(bar_ux, dst));
+            const bool got = mbar_wait_cluster(wctx, bar_ux, 0u, kDevMmaWaitTimeout);
+            const float *ux = reinterpret_cast<const float *>(smem + plan.off_ux);
+            for (int idx = tid; idx < kTile * ZP; idx += kConsumerThreads) {
+                const int tok = idx / ZP, pr = idx - tok * ZP;
+                float u0 = 0.0f, u1 = 0.0f;
+                for (int src = 0; src < xsplit && got; ++src) {
+                    const float2 v = *reinterpret_cast<const float2 *>(ux + ((src * kTile + tok) * ZP + pr) * 2);
+                    u0 += v.x;
+                    u1 += v.y;
+                }
+                const int k = 2 * pr;
+                const float z0 = (k < r) ? u0 * __ldg(P.s_r + k) : 0.0f;
+                const float z1 = (k + 1 < r) ? u1 * __ldg(P.s_r + k + 1) : 0.0f;
+                uint32_t hi, lo;
+                split2(z0, z1, hi, lo);
+                zH[idx] = hi;
+                zL[idx] = lo;
+            }
+        } else
         for (int idx = tid; idx < EG * kTile * ZP; idx += kConsumerThreads) {
             const int env = idx / (kTile * ZP), rem = idx - env * (kTile * ZP);
             const int genv = grp * EG + env;           // envelope of the adapter
@@ -998,14 +1110,49 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 // wave of tiles, or a call that may overlap its neighbours.  One's start-up and
                 // first-load latency then hide behind the other's streaming.  A lone single-wave
                 // call keeps one CTA with 16 consumer warps per SM.
-                const int nw = (all_tiles > sms || overlaps_neighbours) ? 8 : kMaxWarps;
+                // Few tiles of a single-envelope launch with a long d_in (a decode-sized call on a
+                // layer or a down projection): the CTAs that split a tile's y items also share its
+                // first product, as clusters of 4 or 8 along grid z.  Each CTA streams its part of
+                // d_in only and the partial sums go round the cluster, instead of every CTA repeating
+                // the product over all of d_in, which was most of such a call's time (layer at 1 to 8
+                // tokens: 11.3 -> 7.3 us per call that waits for its predecessor; down projection
+                // alone 10.8 -> 7.6 us).  Small CTAs (512-column items), one per SM.  Not below 16 x
+                // items (a 4096-wide projection alone measured 5 % behind: the exchange costs what
+                // the shorter product saves) nor with room for fewer than 4 CTAs per tile.
+                int xsplit = 1;
+                int64_t max_din = 0;
+                for (int k = 0; k < m; ++k)
+                    if (sel[k]->d_in > max_din) max_din = sel[k]->d_in;
+                if (egt == 1 && max_din >= 16 * 8 * kGroup) {
+                    const int64_t room = sms / all_tiles;
+                    xsplit = room >= 8 ? 8 : room >= 4 ? 4 : 1;
+                    if (xsplit > 1) want_splits = room / xsplit * xsplit;
+                }
+                const int nw = (all_tiles > sms || overlaps_neighbours || xsplit > 1) ? 8 : kMaxWarps;
                 const int max_chunk = nw * kGroup;
                 const int smem_budget = (nw == kMaxWarps) ? kSmemBudget : kSmemBudgetHalf;
                 int cw = max_chunk;
-                while (cw > min_cw && (min_dout + cw - 1) / cw < want_splits) cw /= 2;
-                int64_t splits = (min_dout + cw - 1) / cw;
-                if (splits > want_splits) splits = want_splits;
-                if (splits > 64) splits = 64;
+                int64_t splits;
+                if (xsplit > 1) {
+                    // the widest items with which no CTA of the launch gets more y items than it must
+                    // (an item costs about the same time whatever its width)
+                    splits = want_splits > 64 ? 64 : want_splits;
+                    auto y_items = [&](int w) {
+                        int64_t worst = 0;
+                        for (int k = 0; k < m; ++k) {
+                            const int64_t c = ((sel[k]->d_out + w - 1) / w + splits - 1) / splits;
+                            if (c > worst) worst = c;
+                        }
+                        return worst;
+                    };
+                    for (int w = max_chunk / 2; w >= min_cw; w /= 2)
+                        if (y_items(w) < y_items(cw)) cw = w;
+                } else {
+                    while (cw > min_cw && (min_dout + cw - 1) / cw < want_splits) cw /= 2;
+                    splits = (min_dout + cw - 1) / cw;
+                    if (splits > want_splits) splits = want_splits;
+                    if (splits > 64) splits = 64;
+                }
 
                 MmaBatch b;
                 std::memset(&b, 0, sizeof(b));
@@ -1034,13 +1181,14 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 prm.rows = (int)rows; prm.cwy = cw; prm.status = status;
                 prm.wait_prev = !overlaps_neighbours;
                 prm.x_ready = x_ready;
+                prm.xsplit = xsplit;
                 prm.skip_item = test_skip_item();
-                prm.gate_y = prm.wait_prev ? 2 : 0;   // (measured: a call that waits for its predecessor, 12.1 -> 11.8 us; later items lose it again)
+                prm.gate_y = (prm.wait_prev && xsplit == 1) ? 2 : 0;   // (measured: a call that waits for its predecessor, 12.1 -> 11.8 us; later items lose it again)
                 prm.ell = ell;
                 ++*launches;
                 int slots = kMaxSlots;
-                while (slots > 2 && make_plan(nw, rp, max_r, slots, eg, ell, cw).total > smem_budget) --slots;
-                const SmemPlan plan = make_plan(nw, rp, max_r, slots, eg, ell, cw);
+                while (slots > 2 && make_plan(nw, rp, max_r, slots, eg, ell, cw, xsplit).total > smem_budget) --slots;
+                const SmemPlan plan = make_plan(nw, rp, max_r, slots, eg, ell, cw, xsplit);
                 if (plan.total > kSmemBudget) return LORDBA_ECUDA;
                 prm.slots = slots;
                 LaunchRec rec;
@@ -1057,6 +1205,8 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 // touch no global data before griddepcontrol.wait, which returns once that kernel has
                 // completed and its writes are visible.
                 rec.pdl = 1;
+                rec.cluster = xsplit > 1 ? (uint32_t)xsplit : 0;
+                rec.cluster_z = xsplit > 1 ? 1 : 0;
                 rec.n_args = 2;
                 rec.arg_bytes[0] = sizeof(MmaBatch);
                 rec.arg_bytes[1] = sizeof(MmaParams);

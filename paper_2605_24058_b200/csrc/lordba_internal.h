@@ -55,7 +55,7 @@ struct LaunchRec {
     uint32_t n_args;       // 1 or 2 argument blocks
     uint32_t arg_bytes[2];
     uint32_t total_bytes;  // this record + its argument blocks in plan storage (multiple of 64)
-    uint32_t pad_;
+    uint32_t cluster_z;    // 1: the cluster lies along grid z instead of grid x
 };
 
 struct LaunchSink {

@@ -116,6 +116,45 @@ def test_config3_decode_layer_batched(oracle, T, vname, variant):
                      "config3/T=%d/%s/%s" % (T, p.name, vname))
 
 
+@pytest.mark.parametrize("T,d_in,d_out,r,dtype", [
+    (1, 11008, 4096, 16, "bf16"), (8, 11008, 4096, 16, "bf16"), (33, 11008, 4096, 16, "bf16"),
+    (100, 11008, 4096, 16, "bf16"), (300, 11008, 4096, 16, "bf16"), (500, 11008, 4096, 16, "bf16"),
+    (8, 8192, 1024, 64, "bf16"), (40, 8192 + 256, 512, 8, "bf16"), (8, 16384, 2048, 32, "f16"),
+    (20, 11008, 4096, 12, "bf16"), (64, 11008, 4096, 16, "f16"),
+])
+def test_few_tokens_long_d_in_shared_first_product(oracle, T, d_in, d_out, r, dtype):
+    """Few token tiles and a long d_in: the CTAs of a tile share the first product (Eq. 8, u = A_sign
+    (s_in x)) as a cluster, each summing its part of d_in, parts added in a fixed order.  Every
+    element against the oracle; twice the same bits; also with the x-ready promise."""
+    p = workloads.make_projection(d_in, d_out, r, T, dtype, seed=9500 + T + r)
+    a, b, c = DeviceProj(p), DeviceProj(p), DeviceProj(p)
+    code = lordba.BF16 if dtype == "bf16" else lordba.F16
+    assert lordba.query_variant([a.proj()], T, code) == [lordba.VARIANT_MMA]
+    a.forward()
+    b.forward()
+    lordba.adapter_forward(c.x, c.packed_A, c.packed_B, c.s_in, c.s_r, c.s_out, c.y, r, x_ready=True)
+    assert_close(torch_to_f64(a.y), oracle_forward(oracle, p), dtype, "shared first product T=%d r=%d" % (T, r))
+    assert torch.equal(a.y, b.y) and torch.equal(a.y, c.y)
+    assert lordba.device_status() == 0
+
+
+def test_few_tokens_segments_with_shared_first_product(oracle):
+    """Per-projection token counts in a decode-sized batched call (one projection empty, one with
+    fewer tiles than the others): the clusters of a projection's missing tiles leave together."""
+    lengths = [40, 0, 7, 33]
+    ps = [workloads.make_projection(11008, 4096, 16, 40, "bf16", seed=9600 + i) for i in range(4)]
+    ds = [DeviceProj(p) for p in ps]
+    y0 = [d.y.clone() for d in ds]
+    lordba.adapter_forward_segments([d.proj() for d in ds], lengths, lordba.BF16)
+    for p, d, n, y in zip(ps, ds, lengths, y0):
+        rows = np.arange(n)
+        if n:
+            assert_close(torch_to_f64(d.y[:n]), oracle_forward(oracle, p, rows=rows), "bf16", "segment of %d" % n,
+                         scale_from=oracle_forward(oracle, p))
+        assert torch.equal(d.y[n:], y[n:])
+    assert lordba.device_status() == 0
+
+
 @pytest.mark.parametrize("r", [8, 16, 32, 64])
 def test_config4_one_layer_with_outliers(oracle, r):
     """One layer of the 32-layer set at a reduced T that still spans several token tiles and a

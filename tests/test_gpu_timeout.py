@@ -84,5 +84,28 @@ def test_a_wait_that_runs_out_is_reported_and_nothing_wrong_is_written(oracle, h
         assert_close(torch_to_f64(d.y), want, "bf16", "after the timeout")
 
 
+def test_a_wait_that_runs_out_in_a_cluster_stops_the_whole_cluster(oracle, hooks):
+    """Eight token rows of a down projection: the CTAs of the tile share the first product as
+    clusters.  With one CTA's first copy request left out, that CTA sends its partial sums to
+    nobody, every CTA of every cluster gives up its wait for them, the status word reports it and
+    y is untouched; the same call afterwards is correct."""
+    T, d_in, d_out, r = 8, 11008, 4096, 16
+    p = workloads.make_projection(d_in, d_out, r, T, "bf16", seed=901)
+    d = DeviceProj(p)
+    y0 = d.y.clone()
+    hooks.lordba_set_variant(lordba.VARIANT_MMA)
+    assert _status(hooks) == (0, 0)
+    hooks.lordba_test_skip_item(0)
+    assert _forward(hooks, d, T) == 0
+    rc, code = _status(hooks)
+    assert rc == ETIMEOUT and code in (1, 2, 3, 4)
+    assert _status(hooks) == (0, 0)
+    assert torch.equal(d.y, y0)
+    hooks.lordba_test_skip_item(-1)
+    assert _forward(hooks, d, T) == 0
+    assert _status(hooks) == (0, 0)
+    assert_close(torch_to_f64(d.y), oracle_forward(oracle, p), "bf16", "after the timeout in a cluster")
+
+
 def test_product_library_has_no_hooks():
     assert not hasattr(lordba.load(), "lordba_test_skip_item")

@@ -54,8 +54,16 @@
 //
 // Warps split the d_in axis for the first product (fixed-order reduction
 // through shared memory, hence deterministic) and the d_out axis for the
-// second.  gridDim.z > 1 splits the y items over several CTAs that each repeat
-// the first product: used when a call has too few tokens to fill the GPU.
+// second.  gridDim.z > 1 splits the y items over several CTAs: used when a call
+// has too few tokens to fill the GPU.  Each of them repeats the first product,
+// or, where d_in is long, they share it as clusters of 4 or 8 along grid z: a
+// CTA streams only its part of d_in, stores its 16 x r partial sums into every
+// cluster CTA's shared memory, arrives once on each one's barrier, and every
+// CTA adds the parts in rank order once all have arrived (MmaParams::xsplit).
+//
+// A call that waits for its predecessor only because of y (the caller's promise
+// LORDBA_PROJ_X_READY) requests its x items and runs the first product before
+// it waits; the y items and everything that writes come after the wait.
 //
 // Every mbarrier wait is bounded: after ~1 s it records a code in the device
 // status word, raises the CTA's abort flag (all later waits return at once) and

@@ -189,10 +189,12 @@ __device__ __forceinline__ void st_cluster_f2(uint32_t addr, float a, float b)
 {
     asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
-// arrive on a barrier of any CTA of the cluster (address from mapa), release at cluster scope
+// arrive on a barrier of any CTA of the cluster (address from mapa).  Relaxed: the stores that the
+// arrival publishes were fenced at cluster scope by the threads that made them, before the CTA
+// barrier that precedes this arrival.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all()
 {
@@ -657,12 +659,12 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
                     for (int dst = 0; dst < xsplit; ++dst) st_cluster_f2(mapa(ux0, dst) + off, u0, u1);
                 }
             }
-            // all of this CTA's stores, then one arrival per destination: the fences and the
-            // barrier order every thread's stores before the arriving thread's release
+            // all of this CTA's stores, each thread's fenced at cluster scope, then the CTA barrier,
+            // then one arrival per destination
             asm volatile("fence.acq_rel.cluster;" ::: "memory");
             consumer_sync<kConsumerThreads>();
-            if (tid == 0 && whole)
-                for (int dst = 0; dst < xsplit; ++dst) mbar_arrive_remote(mapa(bar_ux, dst));
+            // (one thread per destination: an arrival with release is a round trip through the cluster)
+            if (tid < xsplit && whole) mbar_arrive_remote(mapa(bar_ux, tid));
             const bool got = mbar_wait_cluster(wctx, bar_ux, 0u, kDevMmaWaitTimeout);
             const float *ux = reinterpret_cast<const float *>(smem + plan.off_ux);
             for (int idx = tid; idx < kTile * ZP; idx += kConsumerThreads) {

@@ -393,10 +393,14 @@ enum IoKind {
 // items once per group of EG, the y items once.
 // EGT = 0 stands for "one envelope per pass, several envelopes in all" (rank above 32), EGT = 1 for
 // the single-envelope adapter, whose code carries no envelope loops at all.
-template <int RP, int NW, int EGT, int IO, bool GEN>
+// EGT_ = -1 is the single-envelope kernel whose CTAs share the first product as clusters
+// (MmaParams::xsplit), an instantiation of its own so that the others carry none of that code.
+template <int RP, int NW, int EGT_, int IO, bool GEN>
 __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 2)
 mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant__ MmaParams prm)
 {
+    constexpr bool kClusters = (EGT_ == -1);
+    constexpr int EGT = kClusters ? 1 : EGT_;
     constexpr int EG = (EGT == 0) ? 1 : EGT;
     constexpr bool kHalf = (IO != kIoBf16);     // x, y and the first product's operands are halves
     constexpr bool kLoPass = (IO != kIoF16Exact);
@@ -420,7 +424,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     const int ell = (EGT == 1) ? 1 : prm.ell;
     const int n_groups = (EGT == 1) ? 1 : (ell + EG - 1) / EG;
     // CTAs of a cluster along grid z share the first product (single-envelope launches only)
-    const int xsplit = (EGT == 1) ? prm.xsplit : 1;
+    const int xsplit = kClusters ? prm.xsplit : 1;
     const SmemPlan plan = make_plan(NW, RP, r, S, EG, ell, cwy, xsplit);
     const uint32_t sm_base = smem_u32(smem);
 
@@ -635,7 +639,7 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
             }
         }
         consumer_sync<kConsumerThreads>();
-        if (EGT == 1 && xsplit > 1) {
+        if (kClusters && xsplit > 1) {
             // This CTA's sums cover its share of d_in only.  Every pair of them goes to every CTA of
             // the cluster (its own included), followed by one arrival on that CTA's barrier; once
             // all CTAs have arrived here, the shares are added in the order of the CTAs' ranks.
@@ -998,8 +1002,19 @@ const void *kernel_rank(int rp, int eg)
         case 32 * 16 + 2: return kernel_one<32, NW, 2, IO, GEN>();
         case 64 * 16 + 1: return kernel_one<64, NW, 1, IO, GEN>();
         case 64 * 16 + 0: return kernel_one<64, NW, 0, IO, GEN>();
-        default: return nullptr;
+        default: break;
     }
+    // single envelope, CTAs sharing the first product as clusters: small CTAs only
+    if (NW == 8 && eg == -1) {
+        switch (rp) {
+            case 8:  return kernel_one<8, 8, -1, IO, GEN>();
+            case 16: return kernel_one<16, 8, -1, IO, GEN>();
+            case 32: return kernel_one<32, 8, -1, IO, GEN>();
+            case 64: return kernel_one<64, 8, -1, IO, GEN>();
+            default: break;
+        }
+    }
+    return nullptr;
 }
 
 template <int IO>
@@ -1203,9 +1218,10 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 prm.slots = slots;
                 LaunchRec rec;
                 std::memset(&rec, 0, sizeof(rec));
-                rec.func = io == kIoBf16 ? kernel_io<kIoBf16>(rp, nw, egt, gen != 0)
-                           : io == kIoF16 ? kernel_io<kIoF16>(rp, nw, egt, gen != 0)
-                                          : kernel_io<kIoF16Exact>(rp, nw, egt, gen != 0);
+                const int inst = xsplit > 1 ? -1 : egt;      // (the instantiation with the cluster exchange)
+                rec.func = io == kIoBf16 ? kernel_io<kIoBf16>(rp, nw, inst, gen != 0)
+                           : io == kIoF16 ? kernel_io<kIoF16>(rp, nw, inst, gen != 0)
+                                          : kernel_io<kIoF16Exact>(rp, nw, inst, gen != 0);
                 if (!rec.func) return LORDBA_ECUDA;
                 rec.grid[0] = (unsigned)tiles; rec.grid[1] = (unsigned)m; rec.grid[2] = (unsigned)splits;
                 rec.block = nw * 32 + 32;

@@ -1135,20 +1135,20 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 // wave of tiles, or a call that may overlap its neighbours.  One's start-up and
                 // first-load latency then hide behind the other's streaming.  A lone single-wave
                 // call keeps one CTA with 16 consumer warps per SM.
-                // Few tiles of a single-envelope launch with a long d_in (a decode-sized call on a
-                // layer or a down projection): the CTAs that split a tile's y items also share its
-                // first product, as clusters of 4 or 8 along grid z.  Each CTA streams its part of
-                // d_in only and the partial sums go round the cluster, instead of every CTA repeating
-                // the product over all of d_in, which was most of such a call's time (layer at 1 to 8
-                // tokens: 11.3 -> 7.3 us per call that waits for its predecessor; down projection
-                // alone 10.8 -> 7.6 us).  Small CTAs (512-column items), one per SM.  Not below 16 x
-                // items (a 4096-wide projection alone measured 5 % behind: the exchange costs what
-                // the shorter product saves) nor with room for fewer than 4 CTAs per tile.
+                // Few tiles of a single-envelope launch (a decode-sized call, a short prompt): the CTAs
+                // that split a tile's y items also share its first product, as clusters of 4 or 8 along
+                // grid z.  Each CTA streams its part of d_in only and the partial sums go round the
+                // cluster, instead of every CTA repeating the product over all of d_in, which was most
+                // of such a call's time (layer at 1 to 8 tokens: 11.3 -> 5.8 us per call that waits
+                // for its predecessor; a 4096-wide projection alone at 8 to 256 tokens 5.9 - 6.7 ->
+                // 4.5 - 5.6 us).  Small CTAs (512-column items), one per SM.  Only with room for at
+                // least 4 CTAs per tile: clusters of 2 measured behind the repeated product
+                // (layer at 128 tokens, waiting: 13.6 against 12.8 us).
                 int xsplit = 1;
                 int64_t max_din = 0;
                 for (int k = 0; k < m; ++k)
                     if (sel[k]->d_in > max_din) max_din = sel[k]->d_in;
-                if (egt == 1 && max_din >= 16 * 8 * kGroup) {
+                if (egt == 1 && max_din >= 4 * 8 * kGroup) {
                     const int64_t room = sms / all_tiles;
                     xsplit = room >= 8 ? 8 : room >= 4 ? 4 : 1;
                     if (xsplit > 1) want_splits = room / xsplit * xsplit;

@@ -814,7 +814,7 @@ def test_f16_mixed_scale_kinds_on_the_tcgen05_kernel(oracle):
 
 # ---------------------------------------------------------------- prepared calls and the kernel query
 
-@pytest.mark.parametrize("kind", ["layer_r16", "layer_r64", "segments_r16", "mixed_families"])
+@pytest.mark.parametrize("kind", ["layer_r16", "layer_r64", "segments_r16", "mixed_families", "decode_r16"])
 def test_planned_call_equals_plain_call(oracle, kind):
     """lordba_plan_init + lordba_adapter_forward_planned launch what the plain call launches: the
     same number of kernels, bit-identical y, and y matches the oracle; a plan can be replayed."""
@@ -830,6 +830,10 @@ def test_planned_call_equals_plain_call(oracle, kind):
     elif kind == "segments_r16":
         projs = [workloads.make_projection(1024, 768, 16, T, "bf16", seed=8200 + i) for i in range(3)]
         tokens = [T, 0, 77]
+    elif kind == "decode_r16":
+        T = 8                                             # few tiles: launched as clusters that share the first product
+        projs = workloads.config3(T)
+        tokens = T
     else:
         # three kernel families in one call: widths that are not multiples of 64 (the tcgen05 kernel
         # takes them from 128 tokens up), a row pitch of 1001 elements (only the CUDA-core kernel),

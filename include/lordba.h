@@ -312,7 +312,7 @@ int lordba_query_variant(const lordba_proj *projs, int n_proj, int64_t T, const 
  * A plan holds device addresses: it belongs to the device that was current at lordba_plan_init
  * (LORDBA_EINVAL on another one), stays valid while the buffers it names are, and may be replayed
  * any number of times, from any stream; it holds no resources and needs no release.
- * LORDBA_PROJ_OVERLAP in the projections' flags is part of the plan.
+ * LORDBA_PROJ_OVERLAP and LORDBA_PROJ_X_READY in the projections' flags are part of the plan.
  */
 size_t lordba_plan_bytes(const lordba_proj *projs, int n_proj, int64_t T, const int64_t *tokens, int dtype);
 int lordba_plan_init(void *plan, size_t plan_bytes, const lordba_proj *projs, int n_proj, int64_t T,

@@ -138,6 +138,25 @@ def test_few_tokens_long_d_in_shared_first_product(oracle, T, d_in, d_out, r, dt
     assert lordba.device_status() == 0
 
 
+def test_shared_first_product_gives_the_same_bits_every_time():
+    """The partial sums cross the cluster in whatever order the CTAs finish and are added in rank
+    order: 40 runs of a decode-sized layer call (different launch timing every time, the previous
+    run's kernels still draining) give one result."""
+    T = 8
+    projs = workloads.config3(T)
+    first = None
+    for run in range(40):
+        devs = [DeviceProj(p) for p in projs]
+        lordba.adapter_forward_batched([d.proj() for d in devs], T, lordba.BF16)
+        ys = [d.y for d in devs]
+        if first is None:
+            first = ys
+        else:
+            for a, b in zip(first, ys):
+                assert torch.equal(a, b), "run %d differs" % run
+    assert lordba.device_status() == 0
+
+
 def test_few_tokens_segments_with_shared_first_product(oracle):
     """Per-projection token counts in a decode-sized batched call (one projection empty, one with
     fewer tiles than the others): the clusters of a projection's missing tiles leave together."""

@@ -771,7 +771,7 @@ def run_workload(args):
     shapes = {"attn": [(H, H)], "multi": [(H, H)] * max(n_seg, 1), "gate": [(H, F)], "down": [(F, H)],
               "layer": layer, "decode": layer, "full": layer * workloads.N_LAYERS}[args.workload]
     w = DeviceWorkload(lordba, dev, shapes, r, Tn, ell=args.ell, dtype=args.dtype, scales_f16=args.scales_f16,
-                       segments=n_seg, overlap=not args.no_overlap)
+                       segments=n_seg, overlap=not (args.no_overlap or args.x_ready), x_ready=args.x_ready)
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
     sampler = ClockSampler(0)
@@ -896,6 +896,9 @@ def main():
                     help="element type of x and y (supplementary workloads; the default workload is bf16)")
     ap.add_argument("--scales-f16", action="store_true",
                     help="scales rounded to float16 values and declared so (an adapter exported in fp16)")
+    ap.add_argument("--x-ready", action="store_true",
+                    help="supplementary workloads: every step waits for the previous one before it touches y, "
+                         "x and the adapter declared final earlier (LORDBA_PROJ_X_READY)")
     ap.add_argument("--no-overlap", action="store_true",
                     help="every step waits for the previous one to finish (no LORDBA_PROJ_OVERLAP)")
     args = ap.parse_args()

@@ -905,7 +905,7 @@ def main():
     global FIXED_REPEATS
     FIXED_REPEATS = args.repeats if args.repeats and args.repeats > 0 else None
     headline = not (args.workload != "attn" or args.ell != 1 or args.rank != R or args.tokens != T or
-                    args.dtype != "bf16" or args.scales_f16)
+                    args.dtype != "bf16" or args.scales_f16 or args.x_ready)
     if args.impl == "reference" or headline or args.workload == "lora-dense":
         dflt_steps, dflt_warm = 2000, 100
     elif args.workload == "full":

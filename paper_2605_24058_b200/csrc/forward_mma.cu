@@ -125,6 +125,7 @@ struct MmaParams {
     int x_ready;       // 1 (only with wait_prev): x and the adapter were final before the previous kernel began,
                        // so the x items are requested and the first product runs before the wait for it;
                        // y is touched only afterwards
+    int spread_issue;  // 1: the first requests are issued by one lane each instead of one after the other
     int gate_y;        // g > 0: the y items that fit the ring at the start are requested only once x item
                        // g - 1 has landed, so that the x items, which the first product waits for, do not
                        // share the memory system with them from the start (0: everything is requested at once)
@@ -454,20 +455,24 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     // predecessor just before it exits, so that "this grid is complete" still implies "everything
     // before it is complete".
     if (!prm.wait_prev) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid == kConsumerThreads) {
-        // the producer's first lane prepares the barriers and requests the first items at once;
-        // everybody else meets it at the barrier below
-        for (int s = 0; s < S; ++s) {
-            mbar_init(bar_full(s), 1);
-            mbar_init(bar_empty(s), kConsumerWarps);
+    if (warp == kConsumerWarps) {
+        // the producer warp's first lane prepares the barriers; everybody else meets the warp at the
+        // barrier below
+        if (lane == 0) {
+            for (int s = 0; s < S; ++s) {
+                mbar_init(bar_full(s), 1);
+                mbar_init(bar_empty(s), kConsumerWarps);
+            }
+            if (xsplit > 1) mbar_init(bar_ux, (uint32_t)xsplit);   // one arrival per CTA of the cluster
+            *abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
-        if (xsplit > 1) mbar_init(bar_ux, (uint32_t)xsplit);   // one arrival per CTA of the cluster
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        __syncwarp();
         if (prm.wait_prev && !prm.x_ready) {
             // everything before this line overlapped the previous kernel; nothing after it may
+            // (every lane that is going to request data waits itself)
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+            if (lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         }
     }
     auto issue_item = [&](int it, int s) {       // one thread; s = it % S
@@ -487,8 +492,18 @@ mma_forward_kernel(const __grid_constant__ MmaBatch batch, const __grid_constant
     };
     const int n_first = n_items < S ? n_items : S;
     const int n_eager = ((prm.gate_y || prm.x_ready) && n_xi < n_first) ? n_xi : n_first;
-    if (tid == kConsumerThreads)
-        for (int it = 0; it < n_eager; ++it) issue_item(it, it);     // n_eager <= n_first <= S
+    // The first requests (n_eager <= n_first <= S <= 32).  A tensor copy takes its issuing thread some
+    // 50 ns and the ring's first fill is up to 18 of them: the cluster launches of few tiles, which
+    // are all latency, have one lane of the producer warp issue each item (a decode-sized layer call
+    // that waits for its predecessor: 5.9 -> 5.65 us); everywhere else the items go out in order from
+    // one lane (the other way measured 2 - 7 % behind where the memory system is the limit).
+    if (warp == kConsumerWarps) {
+        if (prm.spread_issue) {
+            if (lane < n_eager) issue_item(lane, lane);
+        } else if (lane == 0) {
+            for (int it = 0; it < n_eager; ++it) issue_item(it, it);
+        }
+    }
     __syncthreads();
     // every CTA of the cluster has initialised its barriers before any of them arrives on another's
     // (all CTAs of a cluster have the same tile and projection: none has left above)
@@ -1207,6 +1222,7 @@ int launch_forward_mma(const lordba_proj *projs, const int64_t *tokens, int64_t 
                 prm.wait_prev = !overlaps_neighbours;
                 prm.x_ready = x_ready;
                 prm.xsplit = xsplit;
+                prm.spread_issue = xsplit > 1 ? 1 : 0;
                 prm.skip_item = test_skip_item();
                 prm.gate_y = (prm.wait_prev && xsplit == 1) ? 2 : 0;   // (measured: a call that waits for its predecessor, 12.1 -> 11.8 us; later items lose it again)
                 prm.ell = ell;
